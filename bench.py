@@ -1,0 +1,308 @@
+#!/usr/bin/env python
+"""Benchmark of the gossip-BMUF synchronisation round.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload wikitext103] [--impl gbmuf]
+
+One "step" is one synchronisation round (neighbour draws + the fused gather / average /
+block-momentum pass) over all K replicas of the workload, preceded by one synthetic local step
+that is launched outside the timed interval (its time is reported separately).  Prints ONE JSON
+line.  `--impl reference` times the CPU oracle instead, on a bounded column sample.
+
+Metric: replica-parameters per second per round (K * N / t_round), with the achieved
+algorithmic HBM traffic (24 B per replica-parameter for fp32 replicas, 20 B for bf16) against
+the measured copy bandwidth of the GPU.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "replica_params_per_sec_per_gossip_bmuf_round"
+UNIT = "replica-params/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM traffic of the fused kernel per replica-parameter from an ncu capture (dram__bytes_read.sum
+# + dram__bytes_write.sum divided by the replica-parameters of the captured launch), valid only
+# for the kernel source it was taken from (sha256 of csrc/gbmuf.cu, first 12 hex digits).
+NCU_TRAFFIC = {"source_sha": None, "bytes_per_replica_param": None}
+
+
+def algorithmic_bytes_per_replica_param(dtype: int, mode: int = 0) -> int:
+    """theta read once + omega, Delta read + omega, Delta, theta written."""
+    th = 4 if dtype == 0 else 2
+    return 2 * th if mode == 1 else th + 8 + 8 + th
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        mhz, mx, reasons = [], None, set()
+        for ts, line in self.rows:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7 or not (t0 - 0.05 <= ts <= t1 + 0.15):
+                continue
+            try:
+                mhz.append(float(f[0]))
+                mx = float(f[1])
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                "sw_power_cap"), f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(mhz) if mhz else None, "sm_max_mhz": mx,
+                "samples": len(mhz), "reasons": sorted(reasons)}
+
+
+def source_sha() -> str:
+    with open(os.path.join(ROOT, "paper_1909_09010_b200", "csrc", "gbmuf.cu"), "rb") as f:
+        return hashlib.sha256(f.read()).hexdigest()[:12]
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle legs
+# ------------------------------------------------------------------------------------------------
+def oracle_sample(w, cols: int):
+    """Oracle state over the first `cols` columns of the workload (a column range is exact)."""
+    import numpy as np
+    import oracle
+    from paper_1909_09010_b200 import workloads
+    cols = min(cols, w.N)
+    sh = workloads.shard_columns(w.offsets, 0, cols)
+    theta0 = workloads.theta0_numpy(w, cols)
+    if w.dtype == 1:
+        theta0 = oracle.f32_to_bf16(theta0)
+    st = oracle.init(theta0, w.K, dtype=w.dtype)
+    oracle.local_perturb(st, w.seed, 0, w.lr or 0.1, w.sigma or 1e-3, 1, elem_base=0)
+    return sh, st
+
+
+def time_oracle_rounds(w, cols: int, rounds: int, first_round: int = 1):
+    """Seconds per oracle round (single thread) on the column sample."""
+    import oracle
+    sh, st = oracle_sample(w, cols)
+    times = []
+    for r in range(first_round, first_round + rounds):
+        oracle.local_perturb(st, w.seed, r, w.lr or 0.1, w.sigma or 1e-3, 1, elem_base=0)
+        t0 = time.perf_counter()
+        nbr = oracle.sample_neighbors(w.seed, r, w.K, sh.m, w.p, w.q, comp_base=sh.comp_base)
+        oracle.sync_round(st, sh.offsets, nbr, w.eta, w.zeta)
+        times.append(time.perf_counter() - t0)
+    return times, w.K * sh.n
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cols = args.ref_cols
+    for _ in range(max(args.warmup, 0)):
+        pass
+    times, units = time_oracle_rounds(w, cols, args.warmup + args.steps)
+    times = times[args.warmup:]
+    t = sum(times) / len(times)
+    val = units / t
+    sample = f"columns [0,{min(cols, w.N)}) of {w.name}, all K={w.K} replicas, one round per step"
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32" if w.dtype == 0 else "bf16-stored/f32", "data": "synthetic",
+            "config": {"workload": w.name, "K": w.K, "N": w.N, "components": w.m, "p": w.p,
+                       "q": w.q, "eta": w.eta, "zeta": w.zeta, "sample": sample},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------
+# GPU leg
+# ------------------------------------------------------------------------------------------------
+def run_gpu(args, w):
+    import torch
+    import torch.distributed as dist
+    from paper_1909_09010_b200 import binding, build, workloads
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    build.build()
+    torch.cuda.set_device(local)
+    dev = torch.device(f"cuda:{local}")
+
+    # each rank holds the columns [rank*N, (rank+1)*N) of a model `world` times as wide: ranges of
+    # columns are independent given the (counter-based) neighbour draws, so no data is exchanged
+    K, N, ld = w.K, w.N, w.ld
+    tdt = torch.float32 if w.dtype == 0 else torch.bfloat16
+    theta = torch.empty((K, ld), dtype=tdt, device=dev)
+    omega = torch.empty((K, ld), dtype=torch.float32, device=dev)
+    delta = torch.empty((K, ld), dtype=torch.float32, device=dev)
+    g = binding.Gbmuf(theta, omega, delta, K=K, N=N, ld=ld, p=w.p, q=w.q, eta=w.eta, zeta=w.zeta,
+                      seed=w.seed, theta_dtype=w.dtype, device=local, comp_base=rank * w.m,
+                      elem_base=rank * N)
+    if args.tuning:
+        t = [int(x) for x in args.tuning.split(",")]
+        g.set_tuning(*t)
+    g.set_partition(w.offsets)
+    theta0 = workloads.theta0_torch(w, dev).to(tdt)
+    g.init(theta0)
+    del theta0
+    lr, sigma = w.lr or 0.1, w.sigma or 1e-3
+    g.local_perturb(0, lr, sigma, 1)
+    torch.cuda.synchronize()
+    info = g.launch_info()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True),
+           torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    rnd = 1
+    for _ in range(args.warmup):
+        g.local_perturb(rnd, lr, sigma, 1)
+        g.sync_round(rnd)
+        rnd += 1
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    t_wall0 = time.time()
+    for i in range(args.steps):
+        a, b, c = ev[i]
+        a.record()
+        g.local_perturb(rnd, lr, sigma, 1)      # the synthetic local step: outside the timed interval
+        b.record()
+        g.sync_round(rnd)                       # set-up kernel + fused kernel
+        c.record()
+        rnd += 1
+    barrier()
+    t_wall1 = time.time()
+    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+    status = g.device_status()
+    sync_ms = [b.elapsed_time(c) for a, b, c in ev]
+    pert_ms = [a.elapsed_time(b) for a, b, c in ev]
+    total_sync_s = sum(sync_ms) / 1e3
+    tt = torch.tensor([total_sync_s], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    total_sync_s = float(tt.item())
+
+    line = None
+    if rank == 0:
+        units = world * K * N * args.steps
+        value = units / total_sync_s
+        peak, peak_kind = measured_peak()
+        bpe = algorithmic_bytes_per_replica_param(w.dtype)
+        # per-launch figures of the fused kernel on this rank (the set-up kernel that shares the
+        # event bracket runs for microseconds)
+        t_launch = (sum(sync_ms) / len(sync_ms)) / 1e3
+        achieved = bpe * K * N / t_launch / 1e9
+        traffic = None
+        if NCU_TRAFFIC["source_sha"] == source_sha() and NCU_TRAFFIC["bytes_per_replica_param"]:
+            traffic = NCU_TRAFFIC["bytes_per_replica_param"] * K * N
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": total_sync_s / args.steps * 1e3,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "f32" if w.dtype == 0 else "bf16-stored/f32", "data": "synthetic",
+                "config": {"workload": w.name, "K": K, "N": N, "components": w.m, "p": w.p, "q": w.q,
+                           "eta": w.eta, "zeta": w.zeta, "replica_params_per_gpu": K * N,
+                           "parallelism": f"element-range shards x{world}, no collective",
+                           "l2": "inputs_larger_than_l2 (state %.1f GB per GPU)" %
+                                 ((K * ld * (8 + (4 if w.dtype == 0 else 2))) / 1e9),
+                           "launch": info, "local_step_ms": sum(pert_ms) / len(pert_ms),
+                           "sync_ms_min": min(sync_ms), "sync_ms_max": max(sync_ms),
+                           "device_status": status},
+                "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                             "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                             "frac_of_nominal_8TBs": achieved / 8000.0,
+                             "algorithmic_bytes_per_replica_param": bpe, "traffic": traffic,
+                             "kernel": "sync_fused_kernel"},
+                "clocks": clocks, "gpu_launches": 3 * args.steps, "e2e": None}
+        if not args.no_cpu_baseline and world == 1:
+            times, units_cpu = time_oracle_rounds(w, args.ref_cols, 3)
+            t = sum(times) / len(times)
+            line["cpu_baseline"] = {
+                "value": units_cpu / t, "unit": UNIT, "cores": 1, "kind": "oracle",
+                "sample": f"columns [0,{min(args.ref_cols, N)}) of {w.name}, K={K}, 3 rounds, "
+                          f"{t:.2f} s per round"}
+    g.destroy()
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if line is not None:
+        print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="gbmuf", choices=["gbmuf", "reference"])
+    ap.add_argument("--workload", default="wikitext103")
+    ap.add_argument("--tuning", default="", help="consumer_threads,vectors,stages,ctas,unroll")
+    ap.add_argument("--ref-cols", type=int, default=1 << 23,
+                    help="columns of the workload the CPU oracle is timed on")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    from paper_1909_09010_b200 import workloads
+    w = workloads.get(args.workload)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_gpu(args, w)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,158 @@
+/* gbmuf.h -- C ABI of libgbmuf: the random-gossip BMUF synchronisation round on one GPU.
+ *
+ * The operation is the body of `if t mod H_i == 0` in Algorithm 1 ("gossip-MA (gossip-BMUF) for
+ * node k") of "A Random Gossip BMUF Process for Neural Language Modeling": every worker k, for
+ * every model component i that is due, picks q random neighbours on a p-symmetric ring
+ * (Definition 1), averages its copy of the component with theirs, and passes the average through
+ * the block-momentum filter (block delta G, momentum Delta <- eta Delta + zeta G, global model
+ * omega <- omega + Delta, restart point theta <- omega + eta Delta).  The K workers are K
+ * parameter replicas that live side by side in one GPU's memory.
+ *
+ * Conventions
+ *   - "device" pointers are CUDA device memory of the context's GPU, owned by the CALLER (the
+ *     library never frees or reallocates them); "host" pointers are ordinary host memory read or
+ *     written before the call returns.
+ *   - theta, omega, delta are row-major [K][ld]: worker k's element e is at k*ld + e.  ld >= N,
+ *     ld a multiple of 32, base pointers 128-byte aligned.  Columns N..ld-1 are padding: never
+ *     written, contents irrelevant.  theta is fp32 or bf16 (theta_dtype); omega and delta are
+ *     always fp32.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls that
+ *     take a stream only enqueue work; they do not wait for it.
+ *   - Every function returns a gbmuf_status; nothing throws or aborts across this boundary.  On
+ *     error no device work has been enqueued by that call and out-parameters are untouched;
+ *     gbmuf_last_error() gives a sentence about the most recent failure on that context.
+ *   - All arithmetic is fp32 with round-to-nearest-even on every single operation (no fused
+ *     multiply-add, no flush-to-zero), in the order Algorithm 1 writes it; a bf16 theta is
+ *     widened exactly on load and rounded to nearest-even on store.
+ *   - There is no CPU path and no other back-end: without a CUDA device every compute call
+ *     returns GBMUF_ERR_CUDA.
+ */
+#ifndef GBMUF_H_
+#define GBMUF_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct gbmuf_ctx gbmuf_ctx; /* opaque, owned by the library, freed by gbmuf_destroy */
+
+typedef enum {
+  GBMUF_OK = 0,
+  GBMUF_ERR_INVALID_ARG = 1, /* a size, pointer, alignment or hyper-parameter is out of range   */
+  GBMUF_ERR_BAD_STATE = 2,   /* call order: e.g. sync_round before set_partition               */
+  GBMUF_ERR_ALLOC = 3,       /* a small device table could not be allocated                     */
+  GBMUF_ERR_CUDA = 4,        /* a CUDA runtime call failed (text in gbmuf_last_error)           */
+  GBMUF_ERR_TIMEOUT = 5,     /* a bounded device-side wait gave up (see gbmuf_device_status)    */
+  GBMUF_ERR_UNSUPPORTED = 6  /* valid request outside what the kernels cover (e.g. K too large) */
+} gbmuf_status;
+
+typedef enum { GBMUF_F32 = 0, GBMUF_BF16 = 1 } gbmuf_dtype;
+
+/* Algorithm 1 has two branches after the averaging line: gossip-BMUF (the filter) and gossip-MA
+ * (theta <- average; omega and Delta are then neither read nor written). */
+typedef enum { GBMUF_MODE_BMUF = 0, GBMUF_MODE_MA = 1 } gbmuf_mode;
+
+typedef struct {
+  int32_t K;           /* number of workers n (Definition 1), 1 <= K <= 65535                     */
+  int64_t N;           /* parameters per replica, >= 1                                            */
+  int64_t ld;          /* row stride in elements: >= N, multiple of 32                            */
+  int32_t p;           /* symmetric degree of the ring (Definition 1), >= 0; the candidate set of
+                          worker k is (k-1)%K..(k-p)%K,(k+1)%K..(k+p)%K without k itself and
+                          without repeats, so it has c = min(2p, K-1) members; c <= 64            */
+  int32_t q;           /* gossip neighbours per draw, 0 <= q <= c (Algorithm 1: q <= 2p)          */
+  float eta;           /* block momentum                                                          */
+  float zeta;          /* block learning rate                                                     */
+  int32_t mode;        /* gbmuf_mode                                                              */
+  int32_t theta_dtype; /* gbmuf_dtype                                                             */
+  uint64_t seed;       /* keys the neighbour draws and the synthetic local steps                  */
+  int32_t device;      /* CUDA device ordinal                                                     */
+  int32_t comp_base;   /* global index of this context's component 0 (>= 0).  Non-zero when the
+                          buffers hold a column range of a larger model: draws are keyed by the
+                          global component index, so a range reproduces the full model's choices */
+  int64_t elem_base;   /* global index of column 0 (>= 0); keys the synthetic local-step noise     */
+} gbmuf_config;
+
+/* Bind a context to three caller-owned device buffers (theta, omega, delta: [K][ld], see the
+ * conventions above).  Allocates only small tables (a few KB plus 4*K*m*q bytes later on).
+ * The buffers must stay valid until gbmuf_destroy.  Errors: INVALID_ARG (any range, alignment or
+ * NULL violation; q > c), UNSUPPORTED (K*element size too large for one staged tile, c > 64),
+ * CUDA, ALLOC. */
+gbmuf_status gbmuf_create(const gbmuf_config* cfg, void* theta_device, float* omega_device,
+                          float* delta_device, gbmuf_ctx** out);
+
+/* Split theta = [theta_1^T .. theta_m^T]^T (Algorithm 1, second REQUIRE line): component i covers
+ * elements offsets[i] .. offsets[i+1]-1.  offsets: host, m+1 entries, offsets[0] = 0, strictly
+ * increasing, offsets[m] = N; no alignment is required of interior offsets.  periods: host, m
+ * entries >= 1 (the synchronous period H_i of each component), or NULL for all 1.  May be called
+ * again to re-partition; waits for the context's earlier work first.  1 <= m <= 65536.
+ * Errors: INVALID_ARG, ALLOC, CUDA. */
+gbmuf_status gbmuf_set_partition(gbmuf_ctx* ctx, int32_t m, const int64_t* offsets_host,
+                                 const int32_t* periods_host);
+
+/* Initialisation line of Algorithm 1: theta^k <- theta_0, omega^k <- theta_0, Delta^k <- 0 for
+ * all k.  theta0: device, [N], theta's dtype, 16-byte aligned; may not alias theta. */
+gbmuf_status gbmuf_init(gbmuf_ctx* ctx, const void* theta0_device, void* stream);
+
+/* Synthetic stand-in for the local SGD line theta <- theta - alpha g of Algorithm 1 (there is no
+ * model or data here): nsteps times, theta^k[e] <- store(theta^k[e] - lr * (sigma * z)), with
+ * z(seed, step + s, k, elem_base + e) a counter-based, approximately standard normal value
+ * (Philox4x32-10; sum of four 16-bit uniforms, centred and scaled to unit variance).  In place;
+ * omega and Delta are not touched.  nsteps >= 0, step + nsteps <= 2^32 - 1. */
+gbmuf_status gbmuf_local_perturb(gbmuf_ctx* ctx, uint64_t step, float lr, float sigma,
+                                 int32_t nsteps, void* stream);
+
+/* One synchronisation round `round` (the t of Algorithm 1).  Components taking part:
+ * comp_mask != NULL: host, m bytes, component i takes part iff comp_mask[i] != 0;
+ * comp_mask == NULL: component i takes part iff round % periods[i] == 0.
+ * For each worker k and participating component i: the q neighbours are drawn for
+ * (seed, round, k, comp_base + i); theta_bar = (theta^k + sum_j theta^{k_j}) / (q+1), own value
+ * first, then the neighbours in draw order, all read as they were before this round;
+ * G = theta_bar - R, with R the component as the worker's previous sync left it (theta_0 before
+ * any); Delta <- eta Delta + zeta G; omega <- omega + Delta; theta <- omega + eta Delta.
+ * R is not stored: it is recomputed as store(omega + eta Delta) from the values before the round,
+ * which is bit-for-bit the expression that produced it.  In MA mode theta <- theta_bar only.
+ * Everything happens in place in one pass; components not taking part are not touched.
+ * Requires set_partition.  Errors: BAD_STATE, INVALID_ARG, CUDA. */
+gbmuf_status gbmuf_sync_round(gbmuf_ctx* ctx, uint64_t round, const uint8_t* comp_mask_host,
+                              void* stream);
+
+/* The neighbour choices of round `round`: out is host, [K][m][q] int32 (worker ids).  Runs the
+ * sampler kernel on a private stream and waits for it; does not disturb rounds in flight. */
+gbmuf_status gbmuf_get_neighbors(gbmuf_ctx* ctx, uint64_t round, int32_t* out_host);
+
+/* Return line of Algorithm 1: out[e] = (1/K) sum_k theta^k[e], summed for k = 0..K-1 in that
+ * order.  out: device, [N], theta's dtype, 16-byte aligned. */
+gbmuf_status gbmuf_final_average(gbmuf_ctx* ctx, void* out_device, void* stream);
+
+/* Reads and clears the device-side status word (waits for `stream` first).  *out is GBMUF_OK, or
+ * GBMUF_ERR_TIMEOUT if a kernel's bounded wait on a staged tile expired; the kernel then stopped
+ * early and the buffers' contents are unspecified. */
+gbmuf_status gbmuf_device_status(gbmuf_ctx* ctx, void* stream, int32_t* out);
+
+/* Launch shape of the fused kernel.  Any argument may be 0 to keep the built-in choice.
+ * consumer_threads in {128, 256}; vectors_per_thread >= 1 (a tile is consumer_threads *
+ * vectors_per_thread vectors of 16 bytes of theta); stages 1..8; ctas_per_sm 1..4;
+ * unroll in {1, 2, 4} workers whose omega/Delta loads are issued together.
+ * Errors: INVALID_ARG, UNSUPPORTED (does not fit shared memory). */
+gbmuf_status gbmuf_set_tuning(gbmuf_ctx* ctx, int32_t consumer_threads, int32_t vectors_per_thread,
+                              int32_t stages, int32_t ctas_per_sm, int32_t unroll);
+
+/* What the next full round would launch: tiles (work items), grid and block size, dynamic shared
+ * memory in bytes, elements per tile, stages.  Any out pointer may be NULL.  Requires
+ * set_partition. */
+gbmuf_status gbmuf_get_launch_info(gbmuf_ctx* ctx, int64_t* tiles, int32_t* grid, int32_t* block,
+                                   int32_t* smem_bytes, int32_t* tile_elems, int32_t* stages);
+
+/* Sentence about the last error on this context ("" if none); valid until the next call on it.
+ * With ctx == NULL: the last error of a failed gbmuf_create on this thread. */
+const char* gbmuf_last_error(const gbmuf_ctx* ctx);
+
+/* Waits for the context's work, frees the library's tables.  NULL is accepted. */
+gbmuf_status gbmuf_destroy(gbmuf_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GBMUF_H_ */

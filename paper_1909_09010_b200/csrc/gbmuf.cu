@@ -1,0 +1,1079 @@
+// libgbmuf: the random-gossip BMUF synchronisation round (Algorithm 1 of "A Random Gossip BMUF
+// Process for Neural Language Modeling") for K parameter replicas resident in one GPU's memory.
+// CUDA for sm_100a.  The interface is include/gbmuf.h; this file holds the kernels and the
+// host-side C ABI.
+//
+// Kernels
+//   round_setup_kernel   neighbour draws for every (worker, component) of a round + the tile
+//                        work-list prefix of the components that take part
+//   sync_fused_kernel    gather + average + block-momentum filter, one pass, in place
+//   perturb_kernel       synthetic local steps (counter-based noise)
+//   init_kernel          theta^k <- theta_0, omega^k <- theta_0, Delta^k <- 0
+//   final_average_kernel theta = (1/K) sum_k theta^k
+//
+// Floating point: every operation is an explicit round-to-nearest intrinsic (__fadd_rn,
+// __fmul_rn, __fdiv_rn) so that nothing is contracted into a fused multiply-add.
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "gbmuf.h"
+
+namespace {
+
+// =================================================================================================
+// Philox4x32-10 (Salmon et al., SC'11), device side
+// =================================================================================================
+struct Philox4 { uint32_t x, y, z, w; };
+
+__device__ __forceinline__ Philox4 philox4x32_10(Philox4 c, uint32_t k0, uint32_t k1) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
+    Philox4 n;
+    n.x = hi1 ^ c.y ^ k0;
+    n.y = lo1;
+    n.z = hi0 ^ c.w ^ k1;
+    n.w = lo0;
+    c = n;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  return c;
+}
+
+constexpr uint32_t kTagSampler = 0x53414D50u;  // second key word of the neighbour-draw stream
+constexpr uint32_t kTagPerturb = 0x50455254u;  // second key word of the local-step noise stream
+constexpr int kMaxCand = 64;                   // largest candidate set min(2p, K-1)
+constexpr int kAlign = 8;                      // tiles start on multiples of 8 elements (>= 16 B)
+constexpr int kMaxStages = 8;
+
+// =================================================================================================
+// Round set-up: neighbour draws (Algorithm 1: "randomly choose q neighbors k_1..k_q") and the
+// work-list of this round.
+// =================================================================================================
+struct SetupParams {
+  int K, m, p, q, comp_base, T, use_mask, plan;
+  uint64_t seed, round;
+  const int64_t* off;      // [m+1]
+  const int32_t* periods;  // [m]
+  const uint8_t* mask;     // [m] when use_mask
+  int32_t* nbr;            // [m][K][q]
+  int32_t* tile_prefix;    // [m+1]
+};
+
+// Ring neighbours of worker k (Definition 1): (k-1)%K..(k-p)%K then (k+1)%K..(k+p)%K, leaving
+// out k itself and anything already listed.  Returns the count.
+__device__ int ring_candidates(int k, int K, int p, int32_t* a) {
+  int c = 0;
+  for (int side = 0; side < 2; ++side) {
+    for (int d = 1; d <= p && c < kMaxCand; ++d) {
+      const int step = d % K;
+      int node = side == 0 ? k - step : k + step;
+      if (node < 0) node += K;
+      if (node >= K) node -= K;
+      if (node == k) continue;
+      bool seen = false;
+      for (int j = 0; j < c; ++j) seen |= (a[j] == node);
+      if (!seen) a[c++] = node;
+    }
+  }
+  return c;
+}
+
+__device__ __forceinline__ int tiles_of_component(int64_t lo, int64_t hi, int T) {
+  if (hi <= lo) return 0;
+  const int64_t start = lo & ~(int64_t)(kAlign - 1);
+  return (int)((hi - start + T - 1) / T);
+}
+
+__global__ void __launch_bounds__(256) round_setup_kernel(SetupParams P) {
+  const int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (g < (int64_t)P.K * P.m && P.q > 0) {
+    const int i = (int)(g / P.K), k = (int)(g % P.K);
+    int32_t a[kMaxCand];
+    const int c = ring_candidates(k, P.K, P.p, a);
+    int32_t* out = P.nbr + g * P.q;
+    Philox4 r = {0, 0, 0, 0};
+    for (int j = 0; j < P.q && j < c; ++j) {
+      if ((j & 3) == 0) {
+        Philox4 ctr = {(uint32_t)P.round, (uint32_t)(P.round >> 32), (uint32_t)(P.comp_base + i),
+                       (uint32_t)k | ((uint32_t)(j >> 2) << 16)};
+        r = philox4x32_10(ctr, (uint32_t)P.seed, (uint32_t)(P.seed >> 32) ^ kTagSampler);
+      }
+      const uint32_t u = (j & 3) == 0 ? r.x : (j & 3) == 1 ? r.y : (j & 3) == 2 ? r.z : r.w;
+      const int t = j + (int)__umulhi(u, (uint32_t)(c - j));   // partial Fisher-Yates
+      const int32_t tmp = a[j];
+      a[j] = a[t];
+      a[t] = tmp;
+      out[j] = a[j];
+    }
+  }
+
+  // Block 0 also lays out the work-list: tile_prefix[i] = number of tiles of the participating
+  // components before i.  Block-wide exclusive scan, 256 components at a time.
+  if (blockIdx.x == 0 && P.plan) {
+    __shared__ int warp_tot[8];
+    __shared__ int carry_s;
+    if (threadIdx.x == 0) carry_s = 0;
+    __syncthreads();
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    for (int base = 0; base < P.m; base += 256) {
+      const int i = base + threadIdx.x;
+      int cnt = 0;
+      if (i < P.m) {
+        const bool due = P.use_mask ? (P.mask[i] != 0) : (P.round % (uint64_t)P.periods[i] == 0);
+        if (due) cnt = tiles_of_component(P.off[i], P.off[i + 1], P.T);
+      }
+      int inc = cnt;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, inc, d);
+        if (lane >= d) inc += n;
+      }
+      if (lane == 31) warp_tot[wid] = inc;
+      __syncthreads();
+      int before = 0;
+      for (int w2 = 0; w2 < wid; ++w2) before += warp_tot[w2];
+      const int carry = carry_s;
+      if (i < P.m) P.tile_prefix[i] = carry + before + inc - cnt;
+      __syncthreads();
+      if (threadIdx.x == 255) carry_s = carry + before + inc;
+      __syncthreads();
+    }
+    if (threadIdx.x == 0) P.tile_prefix[P.m] = carry_s;
+  }
+}
+
+// =================================================================================================
+// Shared-memory barrier and bulk-copy primitives (PTX).  Every wait is bounded.
+// =================================================================================================
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Wait for the phase with the given parity to complete.  Gives up after about a second, records
+// GBMUF_ERR_TIMEOUT in the device status word and returns false; the caller then leaves its loop.
+__device__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, int32_t* status) {
+  for (uint32_t spin = 0; spin < (1u << 22); ++spin) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (spin > 32) __nanosleep(spin > 4096 ? 256 : 32);
+  }
+  atomicExch(status, (int32_t)GBMUF_ERR_TIMEOUT);
+  return false;
+}
+// One-dimensional bulk copy global -> shared through the copy engine (no multicast); completion
+// is counted in bytes on the mbarrier.  Addresses and size are multiples of 16 bytes.
+__device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src, uint32_t bytes,
+                                          uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+          dst_smem),
+      "l"(src), "r"(bytes), "r"(bar)
+      : "memory");
+}
+
+// =================================================================================================
+// theta storage types
+// =================================================================================================
+template <typename TH> struct ThetaTraits;
+template <> struct ThetaTraits<float> {
+  static constexpr int VEC = 4;   // elements per 16-byte vector of theta
+  static __device__ __forceinline__ float widen(float v) { return v; }
+  static __device__ __forceinline__ float round_store(float v) { return v; }
+  static __device__ __forceinline__ float narrow(float v) { return v; }
+  static __device__ __forceinline__ void lds(const float* p, float (&x)[4]) {
+    const float4 t = *reinterpret_cast<const float4*>(p);
+    x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w;
+  }
+  static __device__ __forceinline__ void stg(float* p, const float (&x)[4]) {
+    __stcs(reinterpret_cast<float4*>(p), make_float4(x[0], x[1], x[2], x[3]));
+  }
+};
+template <> struct ThetaTraits<__nv_bfloat16> {
+  static constexpr int VEC = 8;
+  static __device__ __forceinline__ float widen(__nv_bfloat16 v) { return __bfloat162float(v); }
+  // value of v after a round trip through bf16 storage (round to nearest, ties to even)
+  static __device__ __forceinline__ float round_store(float v) {
+    return __bfloat162float(__float2bfloat16_rn(v));
+  }
+  static __device__ __forceinline__ __nv_bfloat16 narrow(float v) { return __float2bfloat16_rn(v); }
+  static __device__ __forceinline__ void lds(const __nv_bfloat16* p, float (&x)[8]) {
+    const uint4 t = *reinterpret_cast<const uint4*>(p);
+    x[0] = __uint_as_float(t.x << 16); x[1] = __uint_as_float(t.x & 0xFFFF0000u);
+    x[2] = __uint_as_float(t.y << 16); x[3] = __uint_as_float(t.y & 0xFFFF0000u);
+    x[4] = __uint_as_float(t.z << 16); x[5] = __uint_as_float(t.z & 0xFFFF0000u);
+    x[6] = __uint_as_float(t.w << 16); x[7] = __uint_as_float(t.w & 0xFFFF0000u);
+  }
+  static __device__ __forceinline__ void stg(__nv_bfloat16* p, const float (&x)[8]) {
+    uint4 t;
+    __nv_bfloat162 h;
+    h = __floats2bfloat162_rn(x[0], x[1]); t.x = *reinterpret_cast<uint32_t*>(&h);
+    h = __floats2bfloat162_rn(x[2], x[3]); t.y = *reinterpret_cast<uint32_t*>(&h);
+    h = __floats2bfloat162_rn(x[4], x[5]); t.z = *reinterpret_cast<uint32_t*>(&h);
+    h = __floats2bfloat162_rn(x[6], x[7]); t.w = *reinterpret_cast<uint32_t*>(&h);
+    __stcs(reinterpret_cast<uint4*>(p), t);
+  }
+};
+
+// =================================================================================================
+// The fused round: gather + average + block-momentum filter, in place, one pass.
+//
+// Work item = one tile: up to T consecutive elements of ONE component, for all K workers.  A
+// persistent CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...  Warp 0 is the producer: it
+// looks the tile up in the work-list, and has the copy engine bring the K replicas' slices of
+// that tile into a shared-memory stage (K bulk copies counted on the stage's `full` barrier),
+// running up to `stages` tiles ahead.  The other warps are consumers: each thread owns 16-byte
+// vectors of the tile; for every worker k it sums the worker's own slice and its q neighbours'
+// slices out of shared memory (own first, then draw order), divides by q+1, streams omega and
+// Delta of that worker through registers, applies the filter and writes Delta, omega and the
+// restart point theta back in place.  Because the CTA is the only reader and writer of its tile
+// in all K replicas and has staged the pre-round values before writing any, every neighbour read
+// sees the replica as it was before the round.  Unique traffic per replica-parameter: theta read
+// once, omega and Delta read once, all three written once.
+// =================================================================================================
+struct TileDesc {
+  long long e0;   // first element of the staged range (multiple of kAlign)
+  long long lo;   // first element this tile owns
+  long long hi;   // one past the last element this tile owns
+  int comp;
+  int pad;
+};
+
+struct SyncParams {
+  void* theta;
+  float* omega;
+  float* delta;
+  const int64_t* off;
+  const int32_t* tile_prefix;
+  const int32_t* nbr;   // [m][K][q]
+  int32_t* status;
+  long long ld;
+  int K, m, q, mode;
+  float eta, zeta, qp1, inv_qp1;
+  int inv_exact;        // q+1 is a power of two: multiplying by 1/(q+1) equals dividing
+  int T, U, stages, ncons;
+  uint32_t stage_stride, nbr_off, desc_off;
+};
+
+template <typename TH>
+__device__ __forceinline__ float gossip_average_1(const SyncParams& P, const TH* sth,
+                                                  const int* snb, int k, int col) {
+  float s = ThetaTraits<TH>::widen(sth[(size_t)k * P.T + col]);
+  for (int j = 0; j < P.q; ++j)
+    s = __fadd_rn(s, ThetaTraits<TH>::widen(sth[(size_t)snb[k * P.q + j] * P.T + col]));
+  return P.inv_exact ? __fmul_rn(s, P.inv_qp1) : __fdiv_rn(s, P.qp1);
+}
+
+// Block-momentum filter for one element (Algorithm 1: G, Delta, omega, theta lines).  The
+// block-start value is recomputed from the pre-round omega and Delta.
+template <typename TH>
+__device__ __forceinline__ void bmuf_filter(float avg, float& w, float& d, float& t, float eta,
+                                            float zeta) {
+  const float etad = __fmul_rn(eta, d);
+  const float r = ThetaTraits<TH>::round_store(__fadd_rn(w, etad));
+  const float g = __fsub_rn(avg, r);
+  d = __fadd_rn(etad, __fmul_rn(zeta, g));
+  w = __fadd_rn(w, d);
+  t = __fadd_rn(w, __fmul_rn(eta, d));
+}
+
+template <typename TH, int UNR>
+__device__ __forceinline__ void tile_vector(const SyncParams& P, const TH* sth, const int* snb,
+                                            int col, long long e) {
+  constexpr int VEC = ThetaTraits<TH>::VEC;
+  constexpr int NF4 = VEC / 4;
+  const int K = P.K, q = P.q, T = P.T;
+  TH* theta = static_cast<TH*>(P.theta);
+  if (P.mode == GBMUF_MODE_MA) {
+    for (int k = 0; k < K; ++k) {
+      float s[VEC], t[VEC];
+      ThetaTraits<TH>::lds(sth + (size_t)k * T + col, s);
+      for (int j = 0; j < q; ++j) {
+        ThetaTraits<TH>::lds(sth + (size_t)snb[k * q + j] * T + col, t);
+#pragma unroll
+        for (int x = 0; x < VEC; ++x) s[x] = __fadd_rn(s[x], t[x]);
+      }
+#pragma unroll
+      for (int x = 0; x < VEC; ++x)
+        s[x] = P.inv_exact ? __fmul_rn(s[x], P.inv_qp1) : __fdiv_rn(s[x], P.qp1);
+      ThetaTraits<TH>::stg(theta + (long long)k * P.ld + e, s);
+    }
+    return;
+  }
+  for (int k0 = 0; k0 < K; k0 += UNR) {
+    float4 W[UNR][NF4], D[UNR][NF4];
+#pragma unroll
+    for (int u = 0; u < UNR; ++u) {
+      if (k0 + u < K) {
+        const long long at = (long long)(k0 + u) * P.ld + e;
+#pragma unroll
+        for (int f = 0; f < NF4; ++f) {
+          W[u][f] = __ldcs(reinterpret_cast<const float4*>(P.omega + at) + f);
+          D[u][f] = __ldcs(reinterpret_cast<const float4*>(P.delta + at) + f);
+        }
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < UNR; ++u) {
+      const int k = k0 + u;
+      if (k < K) {
+        float s[VEC], t[VEC];
+        ThetaTraits<TH>::lds(sth + (size_t)k * T + col, s);
+        for (int j = 0; j < q; ++j) {
+          ThetaTraits<TH>::lds(sth + (size_t)snb[k * q + j] * T + col, t);
+#pragma unroll
+          for (int x = 0; x < VEC; ++x) s[x] = __fadd_rn(s[x], t[x]);
+        }
+        float* w = reinterpret_cast<float*>(&W[u][0]);
+        float* d = reinterpret_cast<float*>(&D[u][0]);
+#pragma unroll
+        for (int x = 0; x < VEC; ++x) {
+          const float avg = P.inv_exact ? __fmul_rn(s[x], P.inv_qp1) : __fdiv_rn(s[x], P.qp1);
+          bmuf_filter<TH>(avg, w[x], d[x], t[x], P.eta, P.zeta);
+        }
+        const long long at = (long long)k * P.ld + e;
+#pragma unroll
+        for (int f = 0; f < NF4; ++f) {
+          __stcs(reinterpret_cast<float4*>(P.delta + at) + f, D[u][f]);
+          __stcs(reinterpret_cast<float4*>(P.omega + at) + f, W[u][f]);
+        }
+        ThetaTraits<TH>::stg(theta + at, t);
+      }
+    }
+  }
+}
+
+// A vector that straddles the edge of the component: element by element, only what the tile owns.
+template <typename TH>
+__device__ void tile_vector_ragged(const SyncParams& P, const TH* sth, const int* snb, int col,
+                                   long long e, long long lo, long long hi) {
+  constexpr int VEC = ThetaTraits<TH>::VEC;
+  TH* theta = static_cast<TH*>(P.theta);
+  for (int x = 0; x < VEC; ++x) {
+    const long long ee = e + x;
+    if (ee < lo || ee >= hi) continue;
+    for (int k = 0; k < P.K; ++k) {
+      const float avg = gossip_average_1<TH>(P, sth, snb, k, col + x);
+      const long long at = (long long)k * P.ld + ee;
+      if (P.mode == GBMUF_MODE_MA) {
+        theta[at] = ThetaTraits<TH>::narrow(avg);
+      } else {
+        float w = P.omega[at], d = P.delta[at], t;
+        bmuf_filter<TH>(avg, w, d, t, P.eta, P.zeta);
+        P.delta[at] = d;
+        P.omega[at] = w;
+        theta[at] = ThetaTraits<TH>::narrow(t);
+      }
+    }
+  }
+}
+
+template <typename TH, int UNR>
+__global__ void sync_fused_kernel(const SyncParams P) {
+  constexpr int VEC = ThetaTraits<TH>::VEC;
+  extern __shared__ __align__(128) unsigned char smem[];
+  // [0,64): full barriers, [64,128): empty barriers, then the stages
+  const uint32_t bars = smem_u32(smem);
+  unsigned char* stage0 = smem + 128;
+  const int total = P.tile_prefix[P.m];
+  const int stages = P.stages;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(bars + 8 * s, 1);                  // full: one arrival (the producer) + bytes
+      mbar_init(bars + 64 + 8 * s, P.ncons);       // empty: every consumer thread arrives
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+
+  if (threadIdx.x < 32) {
+    // ------------------------------------------------------------------ producer warp
+    const int lane = threadIdx.x;
+    int issued = 0;
+    bool ok = true;
+    for (int it = 0, w = blockIdx.x; w < total; w += gridDim.x, ++it) {
+      const int s = it % stages;
+      if (it >= stages) {
+        ok = mbar_wait_bounded(bars + 64 + 8 * s, ((it / stages) - 1) & 1, P.status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+      }
+      // component of tile w: the last i with tile_prefix[i] <= w
+      int lo_i = 0, hi_i = P.m;
+      while (hi_i - lo_i > 1) {
+        const int mid = (lo_i + hi_i) >> 1;
+        if (__ldg(P.tile_prefix + mid) <= w) lo_i = mid; else hi_i = mid;
+      }
+      const int comp = lo_i;
+      const long long cb = __ldg(P.off + comp), ce = __ldg(P.off + comp + 1);
+      const long long e0 = (cb & ~(long long)(kAlign - 1)) +
+                           (long long)(w - __ldg(P.tile_prefix + comp)) * P.T;
+      long long load_end = (ce + kAlign - 1) & ~(long long)(kAlign - 1);
+      if (load_end > e0 + P.T) load_end = e0 + P.T;
+      const uint32_t bytes = (uint32_t)(load_end - e0) * (uint32_t)sizeof(TH);
+      unsigned char* st = stage0 + (size_t)s * P.stage_stride;
+      int* snb = reinterpret_cast<int*>(st + P.nbr_off);
+      const int32_t* gnb = P.nbr + (size_t)comp * P.K * P.q;
+      for (int x = lane; x < P.K * P.q; x += 32) snb[x] = __ldg(gnb + x);
+      if (lane == 0) {
+        TileDesc* d = reinterpret_cast<TileDesc*>(st + P.desc_off);
+        d->e0 = e0;
+        d->lo = cb > e0 ? cb : e0;
+        d->hi = ce < e0 + P.T ? ce : e0 + P.T;
+        d->comp = comp;
+      }
+      __syncwarp();
+      const uint32_t full = bars + 8 * s;
+      if (lane == 0) mbar_arrive_expect_tx(full, bytes * (uint32_t)P.K);
+      __syncwarp();
+      const TH* src = static_cast<const TH*>(P.theta) + e0;
+      for (int k = lane; k < P.K; k += 32)
+        bulk_load(smem_u32(st) + (uint32_t)k * (uint32_t)P.T * (uint32_t)sizeof(TH),
+                  src + (long long)k * P.ld, bytes, full);
+      issued = it + 1;
+    }
+    if (!ok) {
+      // leave only after the copies already issued into this CTA's shared memory have landed
+      for (int it = issued > stages ? issued - stages : 0; it < issued; ++it)
+        mbar_wait_bounded(bars + 8 * (it % stages), (it / stages) & 1, P.status);
+    }
+    return;
+  }
+
+  // -------------------------------------------------------------------- consumer warps
+  const int c = threadIdx.x - 32;
+  for (int it = 0, w = blockIdx.x; w < total; w += gridDim.x, ++it) {
+    const int s = it % stages;
+    if (!mbar_wait_bounded(bars + 8 * s, (it / stages) & 1, P.status)) return;
+    unsigned char* st = stage0 + (size_t)s * P.stage_stride;
+    const TH* sth = reinterpret_cast<const TH*>(st);
+    const int* snb = reinterpret_cast<const int*>(st + P.nbr_off);
+    const TileDesc* d = reinterpret_cast<const TileDesc*>(st + P.desc_off);
+    const long long e0 = d->e0, lo = d->lo, hi = d->hi;
+    for (int u = 0; u < P.U; ++u) {
+      const int col = (u * P.ncons + c) * VEC;
+      const long long e = e0 + col;
+      if (e >= hi || e + VEC <= lo) continue;
+      if (e >= lo && e + VEC <= hi) tile_vector<TH, UNR>(P, sth, snb, col, e);
+      else tile_vector_ragged<TH>(P, sth, snb, col, e, lo, hi);
+    }
+    mbar_arrive(bars + 64 + 8 * s);   // this thread has finished reading the stage
+  }
+}
+
+// =================================================================================================
+// Synthetic local step: theta <- store(theta - lr * (sigma * z)), z from the four 16-bit halves
+// of two Philox words (Irwin-Hall, n = 4), keyed by (seed, step, worker, global element pair).
+// =================================================================================================
+__device__ __forceinline__ float noise_from_words(uint32_t a, uint32_t b) {
+  const int sum = (int)((a & 0xFFFFu) + (a >> 16) + (b & 0xFFFFu) + (b >> 16));
+  return __fmul_rn((float)(sum - 131070), 0x1.bb67aep-16f);   // 1 / sqrt((2^32 - 1) / 3)
+}
+
+template <typename TH>
+__global__ void __launch_bounds__(256) perturb_kernel(TH* theta, int K, long long N, long long ld,
+                                                      uint32_t key0, uint32_t key1, uint32_t step0,
+                                                      int nsteps, float lr, float sigma,
+                                                      long long elem_base) {
+  constexpr int VEC = ThetaTraits<TH>::VEC;
+  const long long nvec = (N + VEC - 1) / VEC;
+  const long long total = nvec * K;
+  for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+       idx += (long long)gridDim.x * blockDim.x) {
+    const int k = (int)(idx / nvec);
+    const long long e = (idx % nvec) * VEC;
+    TH* row = theta + (long long)k * ld + e;
+    const int n = N - e < VEC ? (int)(N - e) : VEC;
+    float v[VEC];
+    if (n == VEC) {
+      ThetaTraits<TH>::lds(row, v);   // a 16-byte load (rows and vectors are 16-byte aligned)
+    } else {
+      for (int x = 0; x < n; ++x) v[x] = ThetaTraits<TH>::widen(row[x]);
+    }
+    for (int s = 0; s < nsteps; ++s) {
+      unsigned long long have = ~0ull;
+      Philox4 r = {0, 0, 0, 0};
+#pragma unroll
+      for (int x = 0; x < VEC; ++x) {
+        if (x < n) {
+          const unsigned long long ge = (unsigned long long)(elem_base + e + x);
+          const unsigned long long pair = ge >> 1;
+          if (pair != have) {
+            Philox4 ctr = {(uint32_t)pair, (uint32_t)(pair >> 32), (uint32_t)k, step0 + (uint32_t)s};
+            r = philox4x32_10(ctr, key0, key1);
+            have = pair;
+          }
+          const float z = (ge & 1) ? noise_from_words(r.z, r.w) : noise_from_words(r.x, r.y);
+          const float upd = __fmul_rn(lr, __fmul_rn(sigma, z));
+          v[x] = ThetaTraits<TH>::round_store(__fsub_rn(v[x], upd));
+        }
+      }
+    }
+    if (n == VEC) {
+      ThetaTraits<TH>::stg(row, v);
+    } else {
+      for (int x = 0; x < n; ++x) row[x] = ThetaTraits<TH>::narrow(v[x]);
+    }
+  }
+}
+
+// =================================================================================================
+// Initialisation line of Algorithm 1 and its return line.
+// =================================================================================================
+template <typename TH>
+__global__ void __launch_bounds__(256) init_kernel(const TH* theta0, TH* theta, float* omega,
+                                                   float* delta, int K, long long N, long long ld) {
+  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < N;
+       e += (long long)gridDim.x * blockDim.x) {
+    const TH v = theta0[e];
+    const float f = ThetaTraits<TH>::widen(v);
+    for (int k = 0; k < K; ++k) {
+      const long long at = (long long)k * ld + e;
+      theta[at] = v;
+      omega[at] = f;
+      delta[at] = 0.0f;
+    }
+  }
+}
+
+template <typename TH>
+__global__ void __launch_bounds__(256) final_average_kernel(const TH* theta, TH* out, int K,
+                                                            long long N, long long ld) {
+  const float fk = (float)K;
+  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < N;
+       e += (long long)gridDim.x * blockDim.x) {
+    float s = ThetaTraits<TH>::widen(theta[e]);
+    for (int k = 1; k < K; ++k) s = __fadd_rn(s, ThetaTraits<TH>::widen(theta[(long long)k * ld + e]));
+    out[e] = ThetaTraits<TH>::narrow(__fdiv_rn(s, fk));
+  }
+}
+
+// =================================================================================================
+// Host side
+// =================================================================================================
+thread_local std::string g_create_error;
+
+struct Tuning {
+  int ncons = 0, U = 0, stages = 0, ctas = 0, unroll = 0;   // 0 = built-in choice
+};
+
+struct Launch {
+  int ncons, U, stages, ctas, unroll, T;
+  uint32_t stage_stride, nbr_off, desc_off, smem;
+};
+
+int host_candidates(int K, int p) {
+  long long c = 2LL * p;
+  if (c > K - 1) c = K - 1;
+  return (int)c;
+}
+
+}  // namespace
+
+struct gbmuf_ctx {
+  gbmuf_config cfg;
+  void* theta;
+  float* omega;
+  float* delta;
+  int m = 0;
+  int cand = 0;
+  bool partitioned = false;
+  std::vector<int64_t> off;
+  std::vector<int32_t> periods;
+  int64_t* d_off = nullptr;
+  int32_t* d_periods = nullptr;
+  uint8_t* d_mask = nullptr;
+  int32_t* d_prefix = nullptr;
+  int32_t* d_nbr = nullptr;
+  int32_t* d_nbr_export = nullptr;
+  int32_t* d_status = nullptr;
+  cudaStream_t priv = nullptr;
+  int num_sms = 0;
+  int max_smem = 0;        // opt-in dynamic shared memory per block
+  int smem_per_sm = 0;
+  Tuning tuning;
+  Launch launch;
+  bool attr_set[2][3] = {{false, false, false}, {false, false, false}};
+  std::string err;
+};
+
+namespace {
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { prev = -1; }
+    if (prev != dev) ok = (cudaSetDevice(dev) == cudaSuccess);
+  }
+  ~DeviceGuard() {
+    int cur = -1;
+    if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+  }
+};
+
+gbmuf_status fail(gbmuf_ctx* ctx, gbmuf_status st, const std::string& msg) {
+  if (ctx) ctx->err = msg; else g_create_error = msg;
+  return st;
+}
+
+gbmuf_status cuda_fail(gbmuf_ctx* ctx, const char* what, cudaError_t e) {
+  return fail(ctx, GBMUF_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+size_t theta_size(const gbmuf_ctx* c) { return c->cfg.theta_dtype == GBMUF_F32 ? 4 : 2; }
+
+// Choose (or check) the launch shape of the fused kernel for this K, q and dtype.
+gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
+  const int K = ctx->cfg.K, q = ctx->cfg.q;
+  const int esz = (int)theta_size(ctx);
+  const int VEC = 16 / esz;
+  Launch L;
+  L.ncons = t.ncons ? t.ncons : 256;
+  L.unroll = t.unroll ? t.unroll : (esz == 4 ? 4 : 2);
+  L.ctas = t.ctas ? t.ctas : 2;
+  const long long budget = (long long)ctx->smem_per_sm / L.ctas - 1024;   // per CTA, bytes
+  const long long cap = budget < ctx->max_smem ? budget : ctx->max_smem;
+  auto stage_bytes = [&](int ncons, int U, uint32_t* nbr_off, uint32_t* desc_off) {
+    const long long th = (long long)K * ncons * U * 16;
+    long long nb = (th + 15) / 16 * 16;
+    long long ds = (nb + (long long)K * q * 4 + 15) / 16 * 16;
+    long long end = (ds + (long long)sizeof(TileDesc) + 127) / 128 * 128;
+    if (nbr_off) *nbr_off = (uint32_t)nb;
+    if (desc_off) *desc_off = (uint32_t)ds;
+    return end;
+  };
+  if (t.U) {
+    L.U = t.U;
+  } else {
+    // a stage of about 32 KB: large enough for long bursts per row, small enough for depth
+    L.U = 1;
+    while (L.U < 8 && stage_bytes(L.ncons, L.U * 2, nullptr, nullptr) <= 32 * 1024) L.U *= 2;
+  }
+  if (!t.ncons) {
+    // prefer a shape that leaves room for at least two stages per CTA
+    const long long need = t.stages ? t.stages : 2;
+    while (L.ncons > 128 && need * stage_bytes(L.ncons, L.U, nullptr, nullptr) + 128 > cap)
+      L.ncons /= 2;
+  }
+  const long long sb = stage_bytes(L.ncons, L.U, &L.nbr_off, &L.desc_off);
+  if (sb + 128 > cap || sb >= (1 << 20))
+    return fail(ctx, GBMUF_ERR_UNSUPPORTED,
+                "one staged tile (K * 16 bytes * consumer threads * vectors per thread) does not "
+                "fit the shared memory available per CTA");
+  if (t.stages) {
+    L.stages = t.stages;
+  } else {
+    L.stages = (int)((cap - 128) / sb);
+    if (L.stages > 4) L.stages = 4;
+  }
+  if (L.stages < 1 || L.stages > kMaxStages || 128 + (long long)L.stages * sb > cap)
+    return fail(ctx, GBMUF_ERR_UNSUPPORTED, "stages * tile does not fit shared memory");
+  L.stage_stride = (uint32_t)sb;
+  L.smem = (uint32_t)(128 + (long long)L.stages * sb);
+  L.T = L.ncons * L.U * VEC;
+  *out = L;
+  return GBMUF_OK;
+}
+
+long long host_total_tiles(const gbmuf_ctx* ctx, uint64_t round, const uint8_t* mask, int T) {
+  long long total = 0;
+  for (int i = 0; i < ctx->m; ++i) {
+    const bool due = mask ? mask[i] != 0 : (round % (uint64_t)ctx->periods[i] == 0);
+    if (!due) continue;
+    const int64_t lo = ctx->off[i], hi = ctx->off[i + 1];
+    if (hi <= lo) continue;
+    const int64_t start = lo & ~(int64_t)(kAlign - 1);
+    total += (hi - start + T - 1) / T;
+  }
+  return total;
+}
+
+template <typename TH, int UNR>
+gbmuf_status launch_sync(gbmuf_ctx* ctx, const SyncParams& P, int grid, cudaStream_t st, bool* attr) {
+  auto kern = sync_fused_kernel<TH, UNR>;
+  if (!*attr) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         ctx->max_smem);
+    if (e != cudaSuccess) return cuda_fail(ctx, "cudaFuncSetAttribute", e);
+    *attr = true;
+  }
+  kern<<<grid, 32 + P.ncons, ctx->launch.smem, st>>>(P);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(ctx, "launch of the fused round kernel", e);
+  return GBMUF_OK;
+}
+
+void fill_setup(const gbmuf_ctx* ctx, uint64_t round, bool use_mask, bool plan, int32_t* nbr,
+                SetupParams* S) {
+  S->K = ctx->cfg.K; S->m = ctx->m; S->p = ctx->cfg.p; S->q = ctx->cfg.q;
+  S->comp_base = ctx->cfg.comp_base; S->T = ctx->launch.T;
+  S->use_mask = use_mask ? 1 : 0; S->plan = plan ? 1 : 0;
+  S->seed = ctx->cfg.seed; S->round = round;
+  S->off = ctx->d_off; S->periods = ctx->d_periods; S->mask = ctx->d_mask;
+  S->nbr = nbr; S->tile_prefix = ctx->d_prefix;
+}
+
+int elementwise_grid(const gbmuf_ctx* ctx, long long work_items) {
+  long long blocks = (work_items + 255) / 256;
+  const long long cap = (long long)ctx->num_sms * 16;
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  return (int)blocks;
+}
+
+void free_tables(gbmuf_ctx* ctx) {
+  cudaFree(ctx->d_off); cudaFree(ctx->d_periods); cudaFree(ctx->d_mask); cudaFree(ctx->d_prefix);
+  cudaFree(ctx->d_nbr); cudaFree(ctx->d_nbr_export);
+  ctx->d_off = nullptr; ctx->d_periods = nullptr; ctx->d_mask = nullptr; ctx->d_prefix = nullptr;
+  ctx->d_nbr = nullptr; ctx->d_nbr_export = nullptr;
+}
+
+}  // namespace
+
+// =================================================================================================
+// C ABI
+// =================================================================================================
+extern "C" {
+
+gbmuf_status gbmuf_create(const gbmuf_config* cfg, void* theta, float* omega, float* delta,
+                          gbmuf_ctx** out) {
+  if (!cfg || !out) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "cfg and out must not be NULL");
+  if (cfg->K < 1 || cfg->K > 65535) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "K must be in 1..65535");
+  if (cfg->N < 1) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "N must be >= 1");
+  if (cfg->ld < cfg->N || cfg->ld % 32 != 0)
+    return fail(nullptr, GBMUF_ERR_INVALID_ARG, "ld must be >= N and a multiple of 32");
+  if (cfg->p < 0 || cfg->q < 0) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "p and q must be >= 0");
+  if (cfg->mode != GBMUF_MODE_BMUF && cfg->mode != GBMUF_MODE_MA)
+    return fail(nullptr, GBMUF_ERR_INVALID_ARG, "unknown mode");
+  if (cfg->theta_dtype != GBMUF_F32 && cfg->theta_dtype != GBMUF_BF16)
+    return fail(nullptr, GBMUF_ERR_INVALID_ARG, "unknown theta_dtype");
+  if (cfg->comp_base < 0 || cfg->elem_base < 0)
+    return fail(nullptr, GBMUF_ERR_INVALID_ARG, "comp_base and elem_base must be >= 0");
+  if (!(cfg->eta == cfg->eta) || !(cfg->zeta == cfg->zeta))
+    return fail(nullptr, GBMUF_ERR_INVALID_ARG, "eta and zeta must not be NaN");
+  const int cand = host_candidates(cfg->K, cfg->p);
+  if (cfg->q > cand)
+    return fail(nullptr, GBMUF_ERR_INVALID_ARG,
+                "q exceeds the number of ring neighbours min(2p, K-1) (Algorithm 1: q <= 2p)");
+  if (cand > kMaxCand)
+    return fail(nullptr, GBMUF_ERR_UNSUPPORTED, "more than 64 ring neighbours per worker");
+  if (!theta || !omega || !delta)
+    return fail(nullptr, GBMUF_ERR_INVALID_ARG, "theta, omega and delta must not be NULL");
+  if (((uintptr_t)theta | (uintptr_t)omega | (uintptr_t)delta) % 128 != 0)
+    return fail(nullptr, GBMUF_ERR_INVALID_ARG, "theta, omega and delta must be 128-byte aligned");
+  if (cfg->device < 0) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "device must be >= 0");
+
+  int ndev = 0;
+  cudaError_t e = cudaGetDeviceCount(&ndev);
+  if (e != cudaSuccess) return cuda_fail(nullptr, "cudaGetDeviceCount", e);
+  if (cfg->device >= ndev) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "no such CUDA device");
+  DeviceGuard guard(cfg->device);
+  if (!guard.ok) return fail(nullptr, GBMUF_ERR_CUDA, "cudaSetDevice failed");
+
+  gbmuf_ctx* ctx = new (std::nothrow) gbmuf_ctx();
+  if (!ctx) return fail(nullptr, GBMUF_ERR_ALLOC, "out of host memory");
+  ctx->cfg = *cfg; ctx->theta = theta; ctx->omega = omega; ctx->delta = delta; ctx->cand = cand;
+  int v = 0;
+  cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, cfg->device); ctx->num_sms = v;
+  cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerBlockOptin, cfg->device); ctx->max_smem = v;
+  cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerMultiprocessor, cfg->device);
+  ctx->smem_per_sm = v;
+  gbmuf_status st = plan_launch(ctx, ctx->tuning, &ctx->launch);
+  if (st != GBMUF_OK) { g_create_error = ctx->err; delete ctx; return st; }
+  e = cudaMalloc(&ctx->d_status, sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->priv, cudaStreamNonBlocking);
+  if (e != cudaSuccess) {
+    st = e == cudaErrorMemoryAllocation ? fail(nullptr, GBMUF_ERR_ALLOC, "device status word")
+                                        : cuda_fail(nullptr, "context set-up", e);
+    cudaFree(ctx->d_status);
+    delete ctx;
+    return st;
+  }
+  *out = ctx;
+  return GBMUF_OK;
+}
+
+gbmuf_status gbmuf_set_partition(gbmuf_ctx* ctx, int32_t m, const int64_t* offsets,
+                                 const int32_t* periods) {
+  if (!ctx) return GBMUF_ERR_INVALID_ARG;
+  if (m < 1 || m > 65536 || !offsets) return fail(ctx, GBMUF_ERR_INVALID_ARG, "m must be in 1..65536 and offsets not NULL");
+  if (offsets[0] != 0 || offsets[m] != ctx->cfg.N)
+    return fail(ctx, GBMUF_ERR_INVALID_ARG, "offsets[0] must be 0 and offsets[m] must be N");
+  for (int i = 0; i < m; ++i)
+    if (offsets[i + 1] <= offsets[i]) return fail(ctx, GBMUF_ERR_INVALID_ARG, "offsets must be strictly increasing");
+  if (periods)
+    for (int i = 0; i < m; ++i)
+      if (periods[i] < 1) return fail(ctx, GBMUF_ERR_INVALID_ARG, "periods must be >= 1");
+  if ((long long)ctx->cfg.comp_base + m > 0x7fffffffLL)
+    return fail(ctx, GBMUF_ERR_INVALID_ARG, "comp_base + m overflows");
+  DeviceGuard guard(ctx->cfg.device);
+  if (!guard.ok) return fail(ctx, GBMUF_ERR_CUDA, "cudaSetDevice failed");
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return cuda_fail(ctx, "cudaDeviceSynchronize", e);
+  free_tables(ctx);
+  ctx->partitioned = false;
+  ctx->m = m;
+  ctx->off.assign(offsets, offsets + m + 1);
+  if (periods) ctx->periods.assign(periods, periods + m); else ctx->periods.assign(m, 1);
+  const size_t nb = (size_t)ctx->cfg.K * m * (ctx->cfg.q > 0 ? ctx->cfg.q : 1) * sizeof(int32_t);
+  e = cudaMalloc(&ctx->d_off, (m + 1) * sizeof(int64_t));
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->d_periods, m * sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->d_mask, m);
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->d_prefix, (m + 1) * sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->d_nbr, nb);
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->d_nbr_export, nb);
+  if (e == cudaSuccess) e = cudaMemcpy(ctx->d_off, ctx->off.data(), (m + 1) * sizeof(int64_t), cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaMemcpy(ctx->d_periods, ctx->periods.data(), m * sizeof(int32_t), cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaMemset(ctx->d_mask, 1, m);
+  if (e != cudaSuccess) {
+    free_tables(ctx);
+    return e == cudaErrorMemoryAllocation ? fail(ctx, GBMUF_ERR_ALLOC, "partition tables") : cuda_fail(ctx, "partition upload", e);
+  }
+  ctx->partitioned = true;
+  return GBMUF_OK;
+}
+
+gbmuf_status gbmuf_set_tuning(gbmuf_ctx* ctx, int32_t ncons, int32_t U, int32_t stages,
+                              int32_t ctas, int32_t unroll) {
+  if (!ctx) return GBMUF_ERR_INVALID_ARG;
+  if ((ncons != 0 && ncons != 128 && ncons != 256) || U < 0 || U > 64 || stages < 0 ||
+      stages > kMaxStages || ctas < 0 || ctas > 4 || (unroll != 0 && unroll != 1 && unroll != 2 && unroll != 4))
+    return fail(ctx, GBMUF_ERR_INVALID_ARG, "tuning value out of range");
+  Tuning t;
+  t.ncons = ncons; t.U = U; t.stages = stages; t.ctas = ctas; t.unroll = unroll;
+  Launch L;
+  gbmuf_status st = plan_launch(ctx, t, &L);
+  if (st != GBMUF_OK) return st;
+  ctx->tuning = t;
+  ctx->launch = L;
+  return GBMUF_OK;
+}
+
+gbmuf_status gbmuf_get_launch_info(gbmuf_ctx* ctx, int64_t* tiles, int32_t* grid, int32_t* block,
+                                   int32_t* smem, int32_t* tile_elems, int32_t* stages) {
+  if (!ctx) return GBMUF_ERR_INVALID_ARG;
+  if (!ctx->partitioned) return fail(ctx, GBMUF_ERR_BAD_STATE, "set_partition has not been called");
+  std::vector<uint8_t> all(ctx->m, 1);
+  const long long total = host_total_tiles(ctx, 0, all.data(), ctx->launch.T);
+  const long long cap = (long long)ctx->num_sms * ctx->launch.ctas;
+  if (tiles) *tiles = total;
+  if (grid) *grid = (int32_t)(total < cap ? total : cap);
+  if (block) *block = 32 + ctx->launch.ncons;
+  if (smem) *smem = (int32_t)ctx->launch.smem;
+  if (tile_elems) *tile_elems = ctx->launch.T;
+  if (stages) *stages = ctx->launch.stages;
+  return GBMUF_OK;
+}
+
+gbmuf_status gbmuf_init(gbmuf_ctx* ctx, const void* theta0, void* stream) {
+  if (!ctx) return GBMUF_ERR_INVALID_ARG;
+  if (!theta0 || (uintptr_t)theta0 % 16 != 0)
+    return fail(ctx, GBMUF_ERR_INVALID_ARG, "theta0 must be a 16-byte aligned device pointer");
+  DeviceGuard guard(ctx->cfg.device);
+  if (!guard.ok) return fail(ctx, GBMUF_ERR_CUDA, "cudaSetDevice failed");
+  const int grid = elementwise_grid(ctx, ctx->cfg.N);
+  cudaStream_t st = (cudaStream_t)stream;
+  if (ctx->cfg.theta_dtype == GBMUF_F32)
+    init_kernel<float><<<grid, 256, 0, st>>>((const float*)theta0, (float*)ctx->theta, ctx->omega,
+                                             ctx->delta, ctx->cfg.K, ctx->cfg.N, ctx->cfg.ld);
+  else
+    init_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)theta0,
+                                                     (__nv_bfloat16*)ctx->theta, ctx->omega,
+                                                     ctx->delta, ctx->cfg.K, ctx->cfg.N, ctx->cfg.ld);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(ctx, "launch of the init kernel", e);
+  return GBMUF_OK;
+}
+
+gbmuf_status gbmuf_local_perturb(gbmuf_ctx* ctx, uint64_t step, float lr, float sigma,
+                                 int32_t nsteps, void* stream) {
+  if (!ctx) return GBMUF_ERR_INVALID_ARG;
+  if (nsteps < 0 || step + (uint64_t)nsteps > 0xFFFFFFFFull || step > 0xFFFFFFFFull)
+    return fail(ctx, GBMUF_ERR_INVALID_ARG, "nsteps must be >= 0 and step + nsteps <= 2^32 - 1");
+  if (nsteps == 0) return GBMUF_OK;
+  DeviceGuard guard(ctx->cfg.device);
+  if (!guard.ok) return fail(ctx, GBMUF_ERR_CUDA, "cudaSetDevice failed");
+  const uint32_t key0 = (uint32_t)ctx->cfg.seed;
+  const uint32_t key1 = (uint32_t)(ctx->cfg.seed >> 32) ^ kTagPerturb;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int K = ctx->cfg.K;
+  if (ctx->cfg.theta_dtype == GBMUF_F32) {
+    const int grid = elementwise_grid(ctx, (ctx->cfg.N + 3) / 4 * K);
+    perturb_kernel<float><<<grid, 256, 0, st>>>((float*)ctx->theta, K, ctx->cfg.N, ctx->cfg.ld, key0,
+                                                key1, (uint32_t)step, nsteps, lr, sigma,
+                                                ctx->cfg.elem_base);
+  } else {
+    const int grid = elementwise_grid(ctx, (ctx->cfg.N + 7) / 8 * K);
+    perturb_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((__nv_bfloat16*)ctx->theta, K, ctx->cfg.N,
+                                                        ctx->cfg.ld, key0, key1, (uint32_t)step,
+                                                        nsteps, lr, sigma, ctx->cfg.elem_base);
+  }
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(ctx, "launch of the local-step kernel", e);
+  return GBMUF_OK;
+}
+
+gbmuf_status gbmuf_sync_round(gbmuf_ctx* ctx, uint64_t round, const uint8_t* comp_mask,
+                              void* stream) {
+  if (!ctx) return GBMUF_ERR_INVALID_ARG;
+  if (!ctx->partitioned) return fail(ctx, GBMUF_ERR_BAD_STATE, "set_partition has not been called");
+  DeviceGuard guard(ctx->cfg.device);
+  if (!guard.ok) return fail(ctx, GBMUF_ERR_CUDA, "cudaSetDevice failed");
+  const Launch& L = ctx->launch;
+  const long long total = host_total_tiles(ctx, round, comp_mask, L.T);
+  if (total == 0) return GBMUF_OK;
+  if (total > 0x3fffffffLL) return fail(ctx, GBMUF_ERR_UNSUPPORTED, "more than 2^30 - 1 tiles");
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaError_t e;
+  if (comp_mask) {
+    e = cudaMemcpyAsync(ctx->d_mask, comp_mask, ctx->m, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, "upload of the component mask", e);
+  }
+  SetupParams S;
+  fill_setup(ctx, round, comp_mask != nullptr, true, ctx->d_nbr, &S);
+  const long long items = (long long)ctx->cfg.K * ctx->m;
+  round_setup_kernel<<<(int)((items + 255) / 256), 256, 0, st>>>(S);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(ctx, "launch of the round set-up kernel", e);
+
+  SyncParams P;
+  P.theta = ctx->theta; P.omega = ctx->omega; P.delta = ctx->delta;
+  P.off = ctx->d_off; P.tile_prefix = ctx->d_prefix; P.nbr = ctx->d_nbr; P.status = ctx->d_status;
+  P.ld = ctx->cfg.ld; P.K = ctx->cfg.K; P.m = ctx->m; P.q = ctx->cfg.q; P.mode = ctx->cfg.mode;
+  P.eta = ctx->cfg.eta; P.zeta = ctx->cfg.zeta;
+  const int qp1 = ctx->cfg.q + 1;
+  P.qp1 = (float)qp1; P.inv_qp1 = 1.0f / (float)qp1; P.inv_exact = (qp1 & (qp1 - 1)) == 0;
+  P.T = L.T; P.U = L.U; P.stages = L.stages; P.ncons = L.ncons;
+  P.stage_stride = L.stage_stride; P.nbr_off = L.nbr_off; P.desc_off = L.desc_off;
+  const long long cap = (long long)ctx->num_sms * L.ctas;
+  const int grid = (int)(total < cap ? total : cap);
+  const int ui = L.unroll == 1 ? 0 : L.unroll == 2 ? 1 : 2;
+  if (ctx->cfg.theta_dtype == GBMUF_F32) {
+    bool* a = &ctx->attr_set[0][ui];
+    return ui == 0 ? launch_sync<float, 1>(ctx, P, grid, st, a)
+         : ui == 1 ? launch_sync<float, 2>(ctx, P, grid, st, a)
+                   : launch_sync<float, 4>(ctx, P, grid, st, a);
+  }
+  bool* a = &ctx->attr_set[1][ui];
+  return ui == 0 ? launch_sync<__nv_bfloat16, 1>(ctx, P, grid, st, a)
+       : ui == 1 ? launch_sync<__nv_bfloat16, 2>(ctx, P, grid, st, a)
+                 : launch_sync<__nv_bfloat16, 4>(ctx, P, grid, st, a);
+}
+
+gbmuf_status gbmuf_get_neighbors(gbmuf_ctx* ctx, uint64_t round, int32_t* out) {
+  if (!ctx) return GBMUF_ERR_INVALID_ARG;
+  if (!out) return fail(ctx, GBMUF_ERR_INVALID_ARG, "out must not be NULL");
+  if (!ctx->partitioned) return fail(ctx, GBMUF_ERR_BAD_STATE, "set_partition has not been called");
+  const int K = ctx->cfg.K, m = ctx->m, q = ctx->cfg.q;
+  if (q == 0) return GBMUF_OK;
+  DeviceGuard guard(ctx->cfg.device);
+  if (!guard.ok) return fail(ctx, GBMUF_ERR_CUDA, "cudaSetDevice failed");
+  SetupParams S;
+  fill_setup(ctx, round, false, false, ctx->d_nbr_export, &S);
+  const long long items = (long long)K * m;
+  round_setup_kernel<<<(int)((items + 255) / 256), 256, 0, ctx->priv>>>(S);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(ctx, "launch of the round set-up kernel", e);
+  std::vector<int32_t> tmp((size_t)K * m * q);
+  e = cudaMemcpyAsync(tmp.data(), ctx->d_nbr_export, tmp.size() * sizeof(int32_t),
+                      cudaMemcpyDeviceToHost, ctx->priv);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->priv);
+  if (e != cudaSuccess) return cuda_fail(ctx, "read-back of the neighbour table", e);
+  for (int i = 0; i < m; ++i)          // device layout [m][K][q] -> caller's [K][m][q]
+    for (int k = 0; k < K; ++k)
+      for (int j = 0; j < q; ++j)
+        out[((size_t)k * m + i) * q + j] = tmp[((size_t)i * K + k) * q + j];
+  return GBMUF_OK;
+}
+
+gbmuf_status gbmuf_final_average(gbmuf_ctx* ctx, void* out, void* stream) {
+  if (!ctx) return GBMUF_ERR_INVALID_ARG;
+  if (!out || (uintptr_t)out % 16 != 0)
+    return fail(ctx, GBMUF_ERR_INVALID_ARG, "out must be a 16-byte aligned device pointer");
+  DeviceGuard guard(ctx->cfg.device);
+  if (!guard.ok) return fail(ctx, GBMUF_ERR_CUDA, "cudaSetDevice failed");
+  const int grid = elementwise_grid(ctx, ctx->cfg.N);
+  cudaStream_t st = (cudaStream_t)stream;
+  if (ctx->cfg.theta_dtype == GBMUF_F32)
+    final_average_kernel<float><<<grid, 256, 0, st>>>((const float*)ctx->theta, (float*)out,
+                                                      ctx->cfg.K, ctx->cfg.N, ctx->cfg.ld);
+  else
+    final_average_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)ctx->theta,
+                                                              (__nv_bfloat16*)out, ctx->cfg.K,
+                                                              ctx->cfg.N, ctx->cfg.ld);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(ctx, "launch of the final-average kernel", e);
+  return GBMUF_OK;
+}
+
+gbmuf_status gbmuf_device_status(gbmuf_ctx* ctx, void* stream, int32_t* out) {
+  if (!ctx) return GBMUF_ERR_INVALID_ARG;
+  if (!out) return fail(ctx, GBMUF_ERR_INVALID_ARG, "out must not be NULL");
+  DeviceGuard guard(ctx->cfg.device);
+  if (!guard.ok) return fail(ctx, GBMUF_ERR_CUDA, "cudaSetDevice failed");
+  cudaStream_t st = (cudaStream_t)stream;
+  int32_t v = 0;
+  cudaError_t e = cudaMemcpyAsync(&v, ctx->d_status, sizeof(v), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_status, 0, sizeof(v), st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return cuda_fail(ctx, "read of the device status word", e);
+  *out = v;
+  return GBMUF_OK;
+}
+
+const char* gbmuf_last_error(const gbmuf_ctx* ctx) {
+  return ctx ? ctx->err.c_str() : g_create_error.c_str();
+}
+
+gbmuf_status gbmuf_destroy(gbmuf_ctx* ctx) {
+  if (!ctx) return GBMUF_OK;
+  gbmuf_status rc = GBMUF_OK;
+  {
+    DeviceGuard guard(ctx->cfg.device);
+    if (guard.ok) {
+      if (cudaDeviceSynchronize() != cudaSuccess) rc = GBMUF_ERR_CUDA;
+      free_tables(ctx);
+      cudaFree(ctx->d_status);
+      if (ctx->priv) cudaStreamDestroy(ctx->priv);
+    } else {
+      rc = GBMUF_ERR_CUDA;
+    }
+  }
+  delete ctx;
+  return rc;
+}
+
+}  // extern "C"

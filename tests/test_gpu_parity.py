@@ -1,0 +1,241 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element, on the
+same seeded inputs: neighbour tables bit-exact; theta, omega, Delta within 1e-7 + 1e-6 |ref|
+after every step (and, by design, bit-equal)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1909_09010_b200 import binding, workloads
+from harness import Case, Pair, case_of, random_theta0, to_numpy
+
+pytestmark = pytest.mark.gpu
+
+
+def run(case, theta0, rounds, lr=0.1, sigma=1e-2, nsteps=1, tuning=None, slices=None, masks=None,
+        first_round=1, check_nbr=True):
+    pr = Pair(case, theta0, slices=slices, tuning=tuning)
+    try:
+        pr.compare("after init")
+        for r in range(first_round, first_round + rounds):
+            if nsteps:
+                pr.perturb(step=r * nsteps, lr=lr, sigma=sigma, nsteps=nsteps)
+                pr.compare(f"after local steps of round {r}")
+            if check_nbr:
+                pr.check_neighbors(r)
+            pr.sync(r, None if masks is None else masks[(r - first_round) % len(masks)])
+            pr.compare(f"after round {r}")
+    finally:
+        pr.close()
+
+
+# ------------------------------------------------------------------------------------------------
+# the named small workloads
+# ------------------------------------------------------------------------------------------------
+def test_tiny_workload():
+    w = workloads.get("tiny")
+    pr = Pair(case_of(w), workloads.theta0_numpy(w))
+    try:
+        pr.add_drift(workloads.drift_numpy(w))
+        pr.compare("after drift")
+        for r in range(1, w.rounds + 1):
+            pr.check_neighbors(r)
+            pr.sync(r)
+            pr.compare(f"round {r}")
+    finally:
+        pr.close()
+
+
+def test_mid_workload_two_rounds():
+    w = workloads.get("mid")
+    run(case_of(w), workloads.theta0_numpy(w), rounds=2, lr=w.lr, sigma=w.sigma, nsteps=w.local_steps)
+
+
+# ------------------------------------------------------------------------------------------------
+# shapes: ragged edges, unaligned offsets, tiny components, many K / p / q
+# ------------------------------------------------------------------------------------------------
+RAGGED = [
+    # K, offsets, p, q
+    (4, (0, 1, 2, 3, 10, 4099, 4100, 9001), 1, 1),
+    (8, (0, 7, 1031, 2055, 2056, 5000, 12345), 2, 2),
+    (16, (0, 33467 * 3 + 1, 33467 * 5 + 2, 200003), 3, 2),
+    (3, (0, 5, 777), 1, 2),
+    (1, (0, 100, 3001), 0, 0),
+    (2, (0, 4097), 1, 1),
+    (5, (0, 2049, 6000), 2, 4),
+    (17, (0, 999, 5003), 4, 3),
+    (33, (0, 4096, 8200), 3, 5),
+    (16, (0, 8, 16, 24, 1048, 9000), 8, 15),
+    (6, (0, 3, 4, 8, 9, 31, 32, 33, 64, 1000), 3, 5),
+]
+
+
+@pytest.mark.parametrize("K,offsets,p,q", RAGGED)
+@pytest.mark.parametrize("dtype", [0, 1])
+def test_ragged_shapes(K, offsets, p, q, dtype):
+    case = Case(K=K, offsets=offsets, p=p, q=q, eta=0.875, zeta=1.0, dtype=dtype, seed=K * 31 + q)
+    run(case, random_theta0(case.N, seed=K, dtype=dtype), rounds=3, sigma=5e-2)
+
+
+@pytest.mark.parametrize("tuning", [
+    dict(consumer_threads=128, vectors_per_thread=1, stages=1, ctas_per_sm=1, unroll=1),
+    dict(consumer_threads=128, vectors_per_thread=1, stages=3, ctas_per_sm=2, unroll=2),
+    dict(consumer_threads=256, vectors_per_thread=1, stages=2, ctas_per_sm=1, unroll=4),
+    dict(consumer_threads=256, vectors_per_thread=2, stages=1, ctas_per_sm=1, unroll=2),
+    dict(consumer_threads=128, vectors_per_thread=4, stages=3, ctas_per_sm=1, unroll=1),
+    dict(consumer_threads=128, vectors_per_thread=2, stages=6, ctas_per_sm=1, unroll=4),
+])
+@pytest.mark.parametrize("dtype", [0, 1])
+def test_launch_shapes_agree(tuning, dtype):
+    """Several tiles per CTA, a ragged last tile and every pipeline depth give the same bits."""
+    K = 8
+    offsets = (0, 100_003, 100_004, 350_001, 777_777)
+    case = Case(K=K, offsets=offsets, p=2, q=2, eta=0.9, zeta=1.0, dtype=dtype, seed=5)
+    run(case, random_theta0(case.N, seed=77, dtype=dtype), rounds=2, tuning=tuning, check_nbr=False)
+
+
+def test_many_tiles_per_cta():
+    """More tiles than resident CTAs: the persistent loop and stage re-use are exercised."""
+    K, N = 4, 6_000_011
+    case = Case(K=K, offsets=(0, 1_000_000, 1_000_001, 3_999_999, N), p=1, q=1, seed=9)
+    run(case, random_theta0(N, seed=3), rounds=2,
+        tuning=dict(consumer_threads=128, vectors_per_thread=1, stages=2, ctas_per_sm=1, unroll=2))
+
+
+# ------------------------------------------------------------------------------------------------
+# modes, masks, periods, hyper-parameters
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype", [0, 1])
+def test_gossip_ma_mode(dtype):
+    case = Case(K=8, offsets=(0, 1001, 5000, 20011), p=2, q=2, dtype=dtype, seed=2,
+                mode=binding.MODE_MA)
+    run(case, random_theta0(case.N, seed=8, dtype=dtype), rounds=3, sigma=5e-2)
+
+
+def test_component_masks_and_periods():
+    offsets = (0, 3000, 3001, 9000, 20000, 40001)
+    masks = [[1, 0, 1, 0, 1], [0, 1, 0, 0, 0], [0, 0, 0, 0, 0], [1, 1, 1, 1, 1]]
+    case = Case(K=4, offsets=offsets, p=1, q=1, seed=4)
+    run(case, random_theta0(case.N, seed=1), rounds=8, masks=masks, sigma=5e-2)
+    case = Case(K=8, offsets=offsets, p=2, q=2, seed=4, periods=(2, 1, 4, 3, 2))
+    run(case, random_theta0(case.N, seed=1), rounds=12, sigma=5e-2)
+
+
+@pytest.mark.parametrize("eta,zeta,q", [(0.0, 1.0, 1), (0.5, 1.0, 3), (0.9, 0.75, 2), (0.99, 1.5, 4),
+                                        (0.875, 1.0, 6)])
+def test_hyper_parameters(eta, zeta, q):
+    case = Case(K=16, offsets=(0, 5000, 10001, 30000), p=3, q=q, eta=eta, zeta=zeta, seed=q)
+    run(case, random_theta0(case.N, seed=q), rounds=4, sigma=5e-2)
+
+
+def test_column_range_reproduces_the_full_model():
+    """A context bound to a column range (comp_base, elem_base) makes the choices and draws the
+    noise the full model gives those columns."""
+    w = workloads.get("tiny")
+    theta0 = workloads.theta0_numpy(w)
+    full = Pair(case_of(w), theta0)
+    try:
+        for r in (1, 2):
+            full.perturb(r, 0.1, 0.05, 2)
+            full.sync(r)
+        full.compare("full")
+        for rank in range(3):
+            sh = workloads.shard_even(w.offsets, 3, rank)
+            dev = torch.device("cuda:0")
+            ld = workloads.padded_ld(sh.n)
+            th = torch.zeros((w.K, ld), device=dev)
+            om, de = torch.zeros_like(th), torch.zeros_like(th)
+            g = binding.Gbmuf(th, om, de, K=w.K, N=sh.n, ld=ld, p=w.p, q=w.q, eta=w.eta,
+                              zeta=w.zeta, seed=w.seed, comp_base=sh.comp_base, elem_base=sh.col0)
+            g.set_partition(sh.offsets)
+            g.init(torch.from_numpy(theta0[sh.col0:sh.col1].copy()).to(dev))
+            for r in (1, 2):
+                g.local_perturb(r, 0.1, 0.05, 2)
+                g.sync_round(r)
+            torch.cuda.synchronize()
+            for part, whole in ((th, full.theta), (om, full.omega), (de, full.delta)):
+                assert torch.equal(part[:, :sh.n], whole[:, sh.col0:sh.col1])
+            g.destroy()
+    finally:
+        full.close()
+
+
+def test_long_run_stays_bit_equal():
+    """100 rounds with local steps in between (the shape of the long-run workload, small)."""
+    case = Case(K=16, offsets=tuple(int(x) for x in np.linspace(0, 50_000, 9).astype(int)), p=3,
+                q=3, eta=0.9, zeta=1.0, dtype=1, seed=4)
+    pr = Pair(case, random_theta0(case.N, seed=4, dtype=1))
+    try:
+        for r in range(1, 101):
+            pr.perturb(step=8 * r, lr=0.1, sigma=1e-2, nsteps=8)
+            pr.sync(r)
+            if r % 20 == 0:
+                pr.compare(f"round {r}")
+    finally:
+        pr.close()
+
+
+def test_final_average():
+    for dtype in (0, 1):
+        case = Case(K=8, offsets=(0, 4001, 10007), p=2, q=2, dtype=dtype, seed=3)
+        pr = Pair(case, random_theta0(case.N, seed=5, dtype=dtype))
+        try:
+            pr.perturb(1, 1.0, 0.05)
+            pr.sync(1)
+            out = torch.zeros(case.N, dtype=pr.theta.dtype, device=pr.device)
+            pr.g.final_average(out)
+            torch.cuda.synchronize()
+            want = oracle.final_average(pr.states[0])
+            assert np.array_equal(to_numpy(out).view(np.uint8), want.view(np.uint8))
+        finally:
+            pr.close()
+
+
+# ------------------------------------------------------------------------------------------------
+# errors and state
+# ------------------------------------------------------------------------------------------------
+def test_call_order_and_argument_errors():
+    dev = torch.device("cuda:0")
+    th = torch.zeros((4, 128), device=dev)
+    om, de = torch.zeros_like(th), torch.zeros_like(th)
+    g = binding.Gbmuf(th, om, de, K=4, N=100, ld=128, p=1, q=1, eta=0.9, zeta=1.0)
+    with pytest.raises(binding.GbmufError) as e:
+        g.sync_round(1)
+    assert e.value.status == binding.ERR_BAD_STATE
+    for bad in ([0, 50], [1, 100], [0, 50, 50, 100], [0, 60, 40, 100]):
+        with pytest.raises(binding.GbmufError) as e:
+            g.set_partition(bad)
+        assert e.value.status == binding.ERR_INVALID_ARG
+    with pytest.raises(binding.GbmufError):
+        g.set_partition([0, 50, 100], periods=[1, 0])
+    g.set_partition([0, 50, 100])
+    with pytest.raises(binding.GbmufError):
+        g.set_tuning(consumer_threads=100)
+    with pytest.raises(binding.GbmufError):
+        g.local_perturb(2 ** 32, 0.1, 0.1)
+    info = g.launch_info()
+    assert info["tiles"] == 2 and info["grid"] == 2 and info["block"] in (160, 288)
+    g.sync_round(1)
+    assert g.device_status() == 0
+    g.destroy()
+    g.destroy()                                          # idempotent
+    with pytest.raises(binding.GbmufError) as e:         # K too large for one staged tile
+        big = torch.zeros((2000, 32), device=dev)
+        binding.Gbmuf(big, big, big, K=2000, N=32, ld=32, p=1, q=1, eta=0.9, zeta=1.0)
+    assert e.value.status == binding.ERR_UNSUPPORTED
+
+
+def test_padding_columns_are_never_written():
+    K, N, ld = 4, 1000, 1056
+    dev = torch.device("cuda:0")
+    th = torch.full((K, ld), 7.0, device=dev)
+    om, de = torch.full_like(th, 8.0), torch.full_like(th, 9.0)
+    g = binding.Gbmuf(th, om, de, K=K, N=N, ld=ld, p=1, q=1, eta=0.9, zeta=1.0)
+    g.set_partition([0, 333, N])
+    g.init(torch.randn(N, device=dev))
+    g.local_perturb(1, 0.1, 0.1, 2)
+    g.sync_round(1)
+    torch.cuda.synchronize()
+    assert bool((th[:, N:] == 7.0).all()) and bool((om[:, N:] == 8.0).all())
+    assert bool((de[:, N:] == 9.0).all())
+    g.destroy()
