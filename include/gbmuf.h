@@ -132,12 +132,13 @@ gbmuf_status gbmuf_final_average(gbmuf_ctx* ctx, void* out_device, void* stream)
 gbmuf_status gbmuf_device_status(gbmuf_ctx* ctx, void* stream, int32_t* out);
 
 /* Launch shape of the fused kernel.  Any argument may be 0 to keep the built-in choice.
- * consumer_threads in {128, 256}; vectors_per_thread >= 1 (a tile is consumer_threads *
- * vectors_per_thread vectors of 16 bytes of theta); stages 1..8; ctas_per_sm 1..4;
- * unroll in {1, 2, 4} workers whose omega/Delta loads are issued together.
+ * consumer_threads: multiple of 32 in 32..992 (one more warp issues the copies); tile_elems:
+ * elements of one component staged per work item, a multiple of 8; stages: 1..8 tiles in flight
+ * per CTA; ctas_per_sm: 1..8 resident CTAs the grid is sized for; flags: bit 0 = give the staged
+ * loads an evict-first L2 policy.
  * Errors: INVALID_ARG, UNSUPPORTED (does not fit shared memory). */
-gbmuf_status gbmuf_set_tuning(gbmuf_ctx* ctx, int32_t consumer_threads, int32_t vectors_per_thread,
-                              int32_t stages, int32_t ctas_per_sm, int32_t unroll);
+gbmuf_status gbmuf_set_tuning(gbmuf_ctx* ctx, int32_t consumer_threads, int32_t tile_elems,
+                              int32_t stages, int32_t ctas_per_sm, int32_t flags);
 
 /* What the next full round would launch: tiles (work items), grid and block size, dynamic shared
  * memory in bytes, elements per tile, stages.  Any out pointer may be NULL.  Requires

@@ -14,6 +14,7 @@
 // Floating point: every operation is an explicit round-to-nearest intrinsic (__fadd_rn,
 // __fmul_rn, __fdiv_rn) so that nothing is contracted into a fused multiply-add.
 
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -190,14 +191,16 @@ __device__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, int32_t* status
   atomicExch(status, (int32_t)GBMUF_ERR_TIMEOUT);
   return false;
 }
-// One-dimensional bulk copy global -> shared through the copy engine (no multicast); completion
-// is counted in bytes on the mbarrier.  Addresses and size are multiples of 16 bytes.
-__device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src, uint32_t bytes,
-                                          uint32_t bar) {
+// Two-dimensional tiled TMA load: the box [rows 0..K) x [columns x, x + box width) of a row-major
+// [K][ld] array lands in shared memory as K consecutive rows of box-width elements.  One request
+// per box (no multicast); completion is counted in bytes on the mbarrier, out-of-range columns
+// are zero-filled and still counted.  x * element size must be a multiple of 16 bytes.
+__device__ __forceinline__ void tma_load_box(uint32_t dst_smem, const CUtensorMap* map, int x, int y,
+                                             uint32_t bar) {
   asm volatile(
-      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-          dst_smem),
-      "l"(src), "r"(bytes), "r"(bar)
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], "
+      "[%1, {%2, %3}], [%4];" ::"r"(dst_smem),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
       : "memory");
 }
 
@@ -249,16 +252,19 @@ template <> struct ThetaTraits<__nv_bfloat16> {
 //
 // Work item = one tile: up to T consecutive elements of ONE component, for all K workers.  A
 // persistent CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...  Warp 0 is the producer: it
-// looks the tile up in the work-list, and has the copy engine bring the K replicas' slices of
-// that tile into a shared-memory stage (K bulk copies counted on the stage's `full` barrier),
-// running up to `stages` tiles ahead.  The other warps are consumers: each thread owns 16-byte
-// vectors of the tile; for every worker k it sums the worker's own slice and its q neighbours'
-// slices out of shared memory (own first, then draw order), divides by q+1, streams omega and
-// Delta of that worker through registers, applies the filter and writes Delta, omega and the
-// restart point theta back in place.  Because the CTA is the only reader and writer of its tile
-// in all K replicas and has staged the pre-round values before writing any, every neighbour read
-// sees the replica as it was before the round.  Unique traffic per replica-parameter: theta read
-// once, omega and Delta read once, all three written once.
+// looks the tile up in the work-list and has the copy engine bring the K replicas' slices of
+// theta, omega and Delta for that tile into a shared-memory stage (one tiled TMA request per
+// [K rows x box-width columns] box, counted on the stage's `full` barrier), running up to
+// `stages` tiles ahead.  The other warps are consumers:
+// each thread takes (16-byte vector, worker) pairs of the tile; it sums the worker's own slice
+// and its q neighbours' slices out of shared memory (own first, then draw order), divides by
+// q+1, applies the filter to the staged omega and Delta and writes Delta, omega and the restart
+// point theta straight to global memory.  All global reads are issued by the copy engine, so
+// the bytes in flight do not depend on how many threads are resident.  Because the CTA is the
+// only reader and writer of its tile in all K replicas and has staged the pre-round values
+// before writing any, every neighbour read sees the replica as it was before the round.  Unique
+// traffic per replica-parameter: theta read once, omega and Delta read once, all three written
+// once.
 // =================================================================================================
 struct TileDesc {
   long long e0;   // first element of the staged range (multiple of kAlign)
@@ -280,18 +286,10 @@ struct SyncParams {
   int K, m, q, mode;
   float eta, zeta, qp1, inv_qp1;
   int inv_exact;        // q+1 is a power of two: multiplying by 1/(q+1) equals dividing
-  int T, U, stages, ncons;
-  uint32_t stage_stride, nbr_off, desc_off;
+  int T, BW, bw_shift, bw_mask, stages, ncons;   // BW: columns per TMA box; column c of a tile is
+                                                 // in box c >> bw_shift at c & bw_mask
+  uint32_t stage_stride, omega_off, delta_off, nbr_off, desc_off;
 };
-
-template <typename TH>
-__device__ __forceinline__ float gossip_average_1(const SyncParams& P, const TH* sth,
-                                                  const int* snb, int k, int col) {
-  float s = ThetaTraits<TH>::widen(sth[(size_t)k * P.T + col]);
-  for (int j = 0; j < P.q; ++j)
-    s = __fadd_rn(s, ThetaTraits<TH>::widen(sth[(size_t)snb[k * P.q + j] * P.T + col]));
-  return P.inv_exact ? __fmul_rn(s, P.inv_qp1) : __fdiv_rn(s, P.qp1);
-}
 
 // Block-momentum filter for one element (Algorithm 1: G, Delta, omega, theta lines).  The
 // block-start value is recomputed from the pre-round omega and Delta.
@@ -306,111 +304,26 @@ __device__ __forceinline__ void bmuf_filter(float avg, float& w, float& d, float
   t = __fadd_rn(w, __fmul_rn(eta, d));
 }
 
-template <typename TH, int UNR>
-__device__ __forceinline__ void tile_vector(const SyncParams& P, const TH* sth, const int* snb,
-                                            int col, long long e) {
+template <typename TH>
+__global__ void __launch_bounds__(1024, 1)
+sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_theta,
+                  const __grid_constant__ CUtensorMap map_omega,
+                  const __grid_constant__ CUtensorMap map_delta) {
   constexpr int VEC = ThetaTraits<TH>::VEC;
   constexpr int NF4 = VEC / 4;
-  const int K = P.K, q = P.q, T = P.T;
-  TH* theta = static_cast<TH*>(P.theta);
-  if (P.mode == GBMUF_MODE_MA) {
-    for (int k = 0; k < K; ++k) {
-      float s[VEC], t[VEC];
-      ThetaTraits<TH>::lds(sth + (size_t)k * T + col, s);
-      for (int j = 0; j < q; ++j) {
-        ThetaTraits<TH>::lds(sth + (size_t)snb[k * q + j] * T + col, t);
-#pragma unroll
-        for (int x = 0; x < VEC; ++x) s[x] = __fadd_rn(s[x], t[x]);
-      }
-#pragma unroll
-      for (int x = 0; x < VEC; ++x)
-        s[x] = P.inv_exact ? __fmul_rn(s[x], P.inv_qp1) : __fdiv_rn(s[x], P.qp1);
-      ThetaTraits<TH>::stg(theta + (long long)k * P.ld + e, s);
-    }
-    return;
-  }
-  for (int k0 = 0; k0 < K; k0 += UNR) {
-    float4 W[UNR][NF4], D[UNR][NF4];
-#pragma unroll
-    for (int u = 0; u < UNR; ++u) {
-      if (k0 + u < K) {
-        const long long at = (long long)(k0 + u) * P.ld + e;
-#pragma unroll
-        for (int f = 0; f < NF4; ++f) {
-          W[u][f] = __ldcs(reinterpret_cast<const float4*>(P.omega + at) + f);
-          D[u][f] = __ldcs(reinterpret_cast<const float4*>(P.delta + at) + f);
-        }
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < UNR; ++u) {
-      const int k = k0 + u;
-      if (k < K) {
-        float s[VEC], t[VEC];
-        ThetaTraits<TH>::lds(sth + (size_t)k * T + col, s);
-        for (int j = 0; j < q; ++j) {
-          ThetaTraits<TH>::lds(sth + (size_t)snb[k * q + j] * T + col, t);
-#pragma unroll
-          for (int x = 0; x < VEC; ++x) s[x] = __fadd_rn(s[x], t[x]);
-        }
-        float* w = reinterpret_cast<float*>(&W[u][0]);
-        float* d = reinterpret_cast<float*>(&D[u][0]);
-#pragma unroll
-        for (int x = 0; x < VEC; ++x) {
-          const float avg = P.inv_exact ? __fmul_rn(s[x], P.inv_qp1) : __fdiv_rn(s[x], P.qp1);
-          bmuf_filter<TH>(avg, w[x], d[x], t[x], P.eta, P.zeta);
-        }
-        const long long at = (long long)k * P.ld + e;
-#pragma unroll
-        for (int f = 0; f < NF4; ++f) {
-          __stcs(reinterpret_cast<float4*>(P.delta + at) + f, D[u][f]);
-          __stcs(reinterpret_cast<float4*>(P.omega + at) + f, W[u][f]);
-        }
-        ThetaTraits<TH>::stg(theta + at, t);
-      }
-    }
-  }
-}
-
-// A vector that straddles the edge of the component: element by element, only what the tile owns.
-template <typename TH>
-__device__ void tile_vector_ragged(const SyncParams& P, const TH* sth, const int* snb, int col,
-                                   long long e, long long lo, long long hi) {
-  constexpr int VEC = ThetaTraits<TH>::VEC;
-  TH* theta = static_cast<TH*>(P.theta);
-  for (int x = 0; x < VEC; ++x) {
-    const long long ee = e + x;
-    if (ee < lo || ee >= hi) continue;
-    for (int k = 0; k < P.K; ++k) {
-      const float avg = gossip_average_1<TH>(P, sth, snb, k, col + x);
-      const long long at = (long long)k * P.ld + ee;
-      if (P.mode == GBMUF_MODE_MA) {
-        theta[at] = ThetaTraits<TH>::narrow(avg);
-      } else {
-        float w = P.omega[at], d = P.delta[at], t;
-        bmuf_filter<TH>(avg, w, d, t, P.eta, P.zeta);
-        P.delta[at] = d;
-        P.omega[at] = w;
-        theta[at] = ThetaTraits<TH>::narrow(t);
-      }
-    }
-  }
-}
-
-template <typename TH, int UNR>
-__global__ void sync_fused_kernel(const SyncParams P) {
-  constexpr int VEC = ThetaTraits<TH>::VEC;
   extern __shared__ __align__(128) unsigned char smem[];
   // [0,64): full barriers, [64,128): empty barriers, then the stages
   const uint32_t bars = smem_u32(smem);
   unsigned char* stage0 = smem + 128;
   const int total = P.tile_prefix[P.m];
   const int stages = P.stages;
+  const bool bmuf = P.mode == GBMUF_MODE_BMUF;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) {
       mbar_init(bars + 8 * s, 1);                  // full: one arrival (the producer) + bytes
       mbar_init(bars + 64 + 8 * s, P.ncons);       // empty: every consumer thread arrives
+      reinterpret_cast<TileDesc*>(stage0 + (size_t)s * P.stage_stride + P.desc_off)->comp = -1;
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -422,6 +335,23 @@ __global__ void sync_fused_kernel(const SyncParams P) {
     const int lane = threadIdx.x;
     int issued = 0;
     bool ok = true;
+    // The tiles of this CTA come in increasing order, so the component only ever moves forward:
+    // find the first one by bisection, then advance.  In the steady state the loop below touches
+    // no global memory except through the bulk copies.
+    int comp = 0, pfx_lo = 0, pfx_hi = 0;
+    long long cb = 0, ce = 0;
+    if (blockIdx.x < total) {
+      int lo_i = 0, hi_i = P.m;
+      while (hi_i - lo_i > 1) {
+        const int mid = (lo_i + hi_i) >> 1;
+        if (__ldg(P.tile_prefix + mid) <= (int)blockIdx.x) lo_i = mid; else hi_i = mid;
+      }
+      comp = lo_i;
+      pfx_lo = __ldg(P.tile_prefix + comp);
+      pfx_hi = __ldg(P.tile_prefix + comp + 1);
+      cb = __ldg(P.off + comp);
+      ce = __ldg(P.off + comp + 1);
+    }
     for (int it = 0, w = blockIdx.x; w < total; w += gridDim.x, ++it) {
       const int s = it % stages;
       if (it >= stages) {
@@ -429,25 +359,25 @@ __global__ void sync_fused_kernel(const SyncParams P) {
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
       }
-      // component of tile w: the last i with tile_prefix[i] <= w
-      int lo_i = 0, hi_i = P.m;
-      while (hi_i - lo_i > 1) {
-        const int mid = (lo_i + hi_i) >> 1;
-        if (__ldg(P.tile_prefix + mid) <= w) lo_i = mid; else hi_i = mid;
+      if (w >= pfx_hi) {
+        while (w >= pfx_hi) {      // w < total = tile_prefix[m], so comp stays below m
+          ++comp;
+          pfx_lo = pfx_hi;
+          pfx_hi = __ldg(P.tile_prefix + comp + 1);
+        }
+        cb = __ldg(P.off + comp);
+        ce = __ldg(P.off + comp + 1);
       }
-      const int comp = lo_i;
-      const long long cb = __ldg(P.off + comp), ce = __ldg(P.off + comp + 1);
-      const long long e0 = (cb & ~(long long)(kAlign - 1)) +
-                           (long long)(w - __ldg(P.tile_prefix + comp)) * P.T;
-      long long load_end = (ce + kAlign - 1) & ~(long long)(kAlign - 1);
-      if (load_end > e0 + P.T) load_end = e0 + P.T;
-      const uint32_t bytes = (uint32_t)(load_end - e0) * (uint32_t)sizeof(TH);
+      const long long e0 = (cb & ~(long long)(kAlign - 1)) + (long long)(w - pfx_lo) * P.T;
       unsigned char* st = stage0 + (size_t)s * P.stage_stride;
-      int* snb = reinterpret_cast<int*>(st + P.nbr_off);
-      const int32_t* gnb = P.nbr + (size_t)comp * P.K * P.q;
-      for (int x = lane; x < P.K * P.q; x += 32) snb[x] = __ldg(gnb + x);
+      TileDesc* d = reinterpret_cast<TileDesc*>(st + P.desc_off);
+      if (d->comp != comp) {       // the stage still holds the table of the component it last served
+        int* snb = reinterpret_cast<int*>(st + P.nbr_off);
+        const int32_t* gnb = P.nbr + (size_t)comp * P.K * P.q;
+        for (int x = lane; x < P.K * P.q; x += 32) snb[x] = __ldg(gnb + x);
+      }
+      __syncwarp();
       if (lane == 0) {
-        TileDesc* d = reinterpret_cast<TileDesc*>(st + P.desc_off);
         d->e0 = e0;
         d->lo = cb > e0 ? cb : e0;
         d->hi = ce < e0 + P.T ? ce : e0 + P.T;
@@ -455,12 +385,23 @@ __global__ void sync_fused_kernel(const SyncParams P) {
       }
       __syncwarp();
       const uint32_t full = bars + 8 * s;
-      if (lane == 0) mbar_arrive_expect_tx(full, bytes * (uint32_t)P.K);
+      const uint32_t row_bytes = (uint32_t)sizeof(TH) + (bmuf ? 8u : 0u);
+      if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)P.K * (uint32_t)P.T * row_bytes);
       __syncwarp();
-      const TH* src = static_cast<const TH*>(P.theta) + e0;
-      for (int k = lane; k < P.K; k += 32)
-        bulk_load(smem_u32(st) + (uint32_t)k * (uint32_t)P.T * (uint32_t)sizeof(TH),
-                  src + (long long)k * P.ld, bytes, full);
+      const uint32_t sbase = smem_u32(st);
+      const int nbox = P.T / P.BW;
+      const int ncopies = (bmuf ? 3 : 1) * nbox;
+      for (int x = lane; x < ncopies; x += 32) {
+        const int arr = x / nbox, b = x - arr * nbox;
+        const int col = (int)e0 + b * P.BW;
+        const uint32_t box_elems = (uint32_t)P.K * (uint32_t)P.BW;
+        if (arr == 0)
+          tma_load_box(sbase + (uint32_t)b * box_elems * (uint32_t)sizeof(TH), &map_theta, col, 0, full);
+        else if (arr == 1)
+          tma_load_box(sbase + P.omega_off + (uint32_t)b * box_elems * 4u, &map_omega, col, 0, full);
+        else
+          tma_load_box(sbase + P.delta_off + (uint32_t)b * box_elems * 4u, &map_delta, col, 0, full);
+      }
       issued = it + 1;
     }
     if (!ok) {
@@ -473,20 +414,84 @@ __global__ void sync_fused_kernel(const SyncParams P) {
 
   // -------------------------------------------------------------------- consumer warps
   const int c = threadIdx.x - 32;
+  const int nv = P.T / VEC;            // vectors per staged row
+  const int items = nv * P.K;          // (vector, worker) pairs per tile
+  const int q = P.q, BW = P.BW, box_elems = P.K * P.BW;
+  // pair p = c, c + ncons, ... is (worker p / nv, vector p % nv); stepped without dividing
+  const int dk = P.ncons / nv, dv = P.ncons - dk * nv;
+  const int k_first = c / nv, v_first = c - k_first * nv;
+  TH* theta = static_cast<TH*>(P.theta);
   for (int it = 0, w = blockIdx.x; w < total; w += gridDim.x, ++it) {
     const int s = it % stages;
     if (!mbar_wait_bounded(bars + 8 * s, (it / stages) & 1, P.status)) return;
     unsigned char* st = stage0 + (size_t)s * P.stage_stride;
     const TH* sth = reinterpret_cast<const TH*>(st);
+    const float* som = reinterpret_cast<const float*>(st + P.omega_off);
+    const float* sde = reinterpret_cast<const float*>(st + P.delta_off);
     const int* snb = reinterpret_cast<const int*>(st + P.nbr_off);
     const TileDesc* d = reinterpret_cast<const TileDesc*>(st + P.desc_off);
     const long long e0 = d->e0, lo = d->lo, hi = d->hi;
-    for (int u = 0; u < P.U; ++u) {
-      const int col = (u * P.ncons + c) * VEC;
+    int k_walk = k_first, v_walk = v_first;
+#pragma unroll 2
+    for (int p = c; p < items; p += P.ncons) {
+      const int k = k_walk, col = v_walk * VEC;
+      k_walk += dk;
+      v_walk += dv;
+      if (v_walk >= nv) { v_walk -= nv; ++k_walk; }
       const long long e = e0 + col;
       if (e >= hi || e + VEC <= lo) continue;
-      if (e >= lo && e + VEC <= hi) tile_vector<TH, UNR>(P, sth, snb, col, e);
-      else tile_vector_ragged<TH>(P, sth, snb, col, e, lo, hi);
+      // gossip average: own slice first, then the neighbours in draw order
+      // staged layout: box b = col / BW holds K rows of BW columns
+      const int b = col >> P.bw_shift, cin = col & P.bw_mask;
+      const int boxbase = b * box_elems + cin;
+      float a[VEC], t[VEC];
+      ThetaTraits<TH>::lds(sth + boxbase + k * BW, a);
+      for (int j = 0; j < q; ++j) {
+        ThetaTraits<TH>::lds(sth + boxbase + snb[k * q + j] * BW, t);
+#pragma unroll
+        for (int x = 0; x < VEC; ++x) a[x] = __fadd_rn(a[x], t[x]);
+      }
+#pragma unroll
+      for (int x = 0; x < VEC; ++x)
+        a[x] = P.inv_exact ? __fmul_rn(a[x], P.inv_qp1) : __fdiv_rn(a[x], P.qp1);
+      const long long at = (long long)k * P.ld + e;
+      const bool whole = e >= lo && e + VEC <= hi;
+      if (!bmuf) {                                       // gossip-MA: theta <- average
+        if (whole) {
+          ThetaTraits<TH>::stg(theta + at, a);
+        } else {
+          for (int x = 0; x < VEC; ++x)
+            if (e + x >= lo && e + x < hi) theta[at + x] = ThetaTraits<TH>::narrow(a[x]);
+        }
+        continue;
+      }
+      float4 W[NF4], D[NF4];
+#pragma unroll
+      for (int f = 0; f < NF4; ++f) {
+        W[f] = *reinterpret_cast<const float4*>(som + boxbase + k * BW + 4 * f);
+        D[f] = *reinterpret_cast<const float4*>(sde + boxbase + k * BW + 4 * f);
+      }
+      float* wv = reinterpret_cast<float*>(&W[0]);
+      float* dv = reinterpret_cast<float*>(&D[0]);
+#pragma unroll
+      for (int x = 0; x < VEC; ++x) bmuf_filter<TH>(a[x], wv[x], dv[x], t[x], P.eta, P.zeta);
+      if (whole) {
+#pragma unroll
+        for (int f = 0; f < NF4; ++f) {
+          __stcs(reinterpret_cast<float4*>(P.delta + at) + f, D[f]);
+          __stcs(reinterpret_cast<float4*>(P.omega + at) + f, W[f]);
+        }
+        ThetaTraits<TH>::stg(theta + at, t);
+      } else {
+        // a vector that straddles the edge of the component: only the elements this tile owns
+        for (int x = 0; x < VEC; ++x) {
+          if (e + x >= lo && e + x < hi) {
+            P.delta[at + x] = dv[x];
+            P.omega[at + x] = wv[x];
+            theta[at + x] = ThetaTraits<TH>::narrow(t[x]);
+          }
+        }
+      }
     }
     mbar_arrive(bars + 64 + 8 * s);   // this thread has finished reading the stage
   }
@@ -585,12 +590,12 @@ __global__ void __launch_bounds__(256) final_average_kernel(const TH* theta, TH*
 thread_local std::string g_create_error;
 
 struct Tuning {
-  int ncons = 0, U = 0, stages = 0, ctas = 0, unroll = 0;   // 0 = built-in choice
+  int ncons = 0, T = 0, stages = 0, ctas = 0, flags = 0;   // 0 = built-in choice
 };
 
 struct Launch {
-  int ncons, U, stages, ctas, unroll, T;
-  uint32_t stage_stride, nbr_off, desc_off, smem;
+  int ncons, stages, ctas, T, BW, flags;
+  uint32_t stage_stride, omega_off, delta_off, nbr_off, desc_off, smem;
 };
 
 int host_candidates(int K, int p) {
@@ -624,7 +629,8 @@ struct gbmuf_ctx {
   int smem_per_sm = 0;
   Tuning tuning;
   Launch launch;
-  bool attr_set[2][3] = {{false, false, false}, {false, false, false}};
+  CUtensorMap map_theta, map_omega, map_delta;   // boxes [K][launch.BW] over the [K][ld] arrays
+  bool attr_set[2] = {false, false};
   std::string err;
 };
 
@@ -654,44 +660,88 @@ gbmuf_status cuda_fail(gbmuf_ctx* ctx, const char* what, cudaError_t e) {
 
 size_t theta_size(const gbmuf_ctx* c) { return c->cfg.theta_dtype == GBMUF_F32 ? 4 : 2; }
 
-// Choose (or check) the launch shape of the fused kernel for this K, q and dtype.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// Tensor maps for boxes of K rows x BW columns over the three [K][ld] arrays.
+gbmuf_status build_tensor_maps(gbmuf_ctx* ctx, const Launch& L) {
+  static EncodeTiledFn encode = nullptr;
+  if (!encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn)
+      return fail(ctx, GBMUF_ERR_CUDA, "the driver does not provide cuTensorMapEncodeTiled");
+    encode = reinterpret_cast<EncodeTiledFn>(fn);
+  }
+  const cuuint64_t ld = (cuuint64_t)ctx->cfg.ld;
+  const cuuint64_t gdim[2] = {ld, (cuuint64_t)ctx->cfg.K};
+  const cuuint32_t box[2] = {(cuuint32_t)L.BW, (cuuint32_t)ctx->cfg.K};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUtensorMapL2promotion prom =
+      (L.flags & 1) ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B;
+  struct { CUtensorMap* map; void* base; CUtensorMapDataType dt; cuuint64_t esz; } arr[3] = {
+      {&ctx->map_theta, ctx->theta,
+       ctx->cfg.theta_dtype == GBMUF_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+       (cuuint64_t)theta_size(ctx)},
+      {&ctx->map_omega, ctx->omega, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4},
+      {&ctx->map_delta, ctx->delta, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4}};
+  for (auto& a : arr) {
+    const cuuint64_t gstride[1] = {ld * a.esz};
+    CUresult r = encode(a.map, a.dt, 2, a.base, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_NONE, prom, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS)
+      return fail(ctx, GBMUF_ERR_CUDA, "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r));
+  }
+  return GBMUF_OK;
+}
+
+// Choose (or check) the launch shape of the fused kernel for this K, q, mode and dtype.
 gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
   const int K = ctx->cfg.K, q = ctx->cfg.q;
   const int esz = (int)theta_size(ctx);
-  const int VEC = 16 / esz;
+  const bool bmuf = ctx->cfg.mode == GBMUF_MODE_BMUF;
   Launch L;
-  L.ncons = t.ncons ? t.ncons : 256;
-  L.unroll = t.unroll ? t.unroll : (esz == 4 ? 4 : 2);
-  L.ctas = t.ctas ? t.ctas : 2;
+  L.ctas = t.ctas ? t.ctas : 1;
+  L.flags = t.flags;
   const long long budget = (long long)ctx->smem_per_sm / L.ctas - 1024;   // per CTA, bytes
   const long long cap = budget < ctx->max_smem ? budget : ctx->max_smem;
-  auto stage_bytes = [&](int ncons, int U, uint32_t* nbr_off, uint32_t* desc_off) {
-    const long long th = (long long)K * ncons * U * 16;
-    long long nb = (th + 15) / 16 * 16;
-    long long ds = (nb + (long long)K * q * 4 + 15) / 16 * 16;
-    long long end = (ds + (long long)sizeof(TileDesc) + 127) / 128 * 128;
-    if (nbr_off) *nbr_off = (uint32_t)nb;
-    if (desc_off) *desc_off = (uint32_t)ds;
-    return end;
+  auto layout = [&](int T, Launch* l) {
+    long long at = (long long)K * T * esz;                 // theta rows
+    at = (at + 127) / 128 * 128;
+    if (l) l->omega_off = (uint32_t)at;
+    if (bmuf) at += (long long)K * T * 4;
+    at = (at + 127) / 128 * 128;
+    if (l) l->delta_off = (uint32_t)at;
+    if (bmuf) at += (long long)K * T * 4;
+    at = (at + 15) / 16 * 16;
+    if (l) l->nbr_off = (uint32_t)at;
+    at += (long long)K * q * 4;
+    at = (at + 15) / 16 * 16;
+    if (l) l->desc_off = (uint32_t)at;
+    at += (long long)sizeof(TileDesc);
+    return (at + 127) / 128 * 128;
   };
-  if (t.U) {
-    L.U = t.U;
+  if (t.T) {
+    L.T = t.T;
   } else {
-    // a stage of about 32 KB: large enough for long bursts per row, small enough for depth
-    L.U = 1;
-    while (L.U < 8 && stage_bytes(L.ncons, L.U * 2, nullptr, nullptr) <= 32 * 1024) L.U *= 2;
+    // the widest tile (longest contiguous run per row) of which one stage still fits
+    long long T = 1024;
+    while (T > 8 && layout((int)T, nullptr) + 128 > cap) T >>= 1;
+    L.T = (int)T;
   }
-  if (!t.ncons) {
-    // prefer a shape that leaves room for at least two stages per CTA
-    const long long need = t.stages ? t.stages : 2;
-    while (L.ncons > 128 && need * stage_bytes(L.ncons, L.U, nullptr, nullptr) + 128 > cap)
-      L.ncons /= 2;
-  }
-  const long long sb = stage_bytes(L.ncons, L.U, &L.nbr_off, &L.desc_off);
+  if (L.T < kAlign || L.T % kAlign != 0)
+    return fail(ctx, GBMUF_ERR_INVALID_ARG, "tile_elems must be a positive multiple of 8");
+  if (L.T > 256 && L.T % 256 != 0)
+    return fail(ctx, GBMUF_ERR_INVALID_ARG, "tile_elems above 256 must be a multiple of 256");
+  L.BW = L.T < 256 ? L.T : 256;                // a tensor-map box is at most 256 elements wide
+  const long long sb = layout(L.T, &L);
   if (sb + 128 > cap || sb >= (1 << 20))
     return fail(ctx, GBMUF_ERR_UNSUPPORTED,
-                "one staged tile (K * 16 bytes * consumer threads * vectors per thread) does not "
-                "fit the shared memory available per CTA");
+                "one staged tile (K rows of theta, omega and Delta) does not fit the shared "
+                "memory available per CTA");
   if (t.stages) {
     L.stages = t.stages;
   } else {
@@ -700,9 +750,9 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
   }
   if (L.stages < 1 || L.stages > kMaxStages || 128 + (long long)L.stages * sb > cap)
     return fail(ctx, GBMUF_ERR_UNSUPPORTED, "stages * tile does not fit shared memory");
+  L.ncons = t.ncons ? t.ncons : (L.stages >= 2 ? 256 : 512);
   L.stage_stride = (uint32_t)sb;
   L.smem = (uint32_t)(128 + (long long)L.stages * sb);
-  L.T = L.ncons * L.U * VEC;
   *out = L;
   return GBMUF_OK;
 }
@@ -720,16 +770,16 @@ long long host_total_tiles(const gbmuf_ctx* ctx, uint64_t round, const uint8_t* 
   return total;
 }
 
-template <typename TH, int UNR>
+template <typename TH>
 gbmuf_status launch_sync(gbmuf_ctx* ctx, const SyncParams& P, int grid, cudaStream_t st, bool* attr) {
-  auto kern = sync_fused_kernel<TH, UNR>;
+  auto kern = sync_fused_kernel<TH>;
   if (!*attr) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          ctx->max_smem);
     if (e != cudaSuccess) return cuda_fail(ctx, "cudaFuncSetAttribute", e);
     *attr = true;
   }
-  kern<<<grid, 32 + P.ncons, ctx->launch.smem, st>>>(P);
+  kern<<<grid, 32 + P.ncons, ctx->launch.smem, st>>>(P, ctx->map_theta, ctx->map_omega, ctx->map_delta);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, "launch of the fused round kernel", e);
   return GBMUF_OK;
@@ -789,6 +839,10 @@ gbmuf_status gbmuf_create(const gbmuf_config* cfg, void* theta, float* omega, fl
                 "q exceeds the number of ring neighbours min(2p, K-1) (Algorithm 1: q <= 2p)");
   if (cand > kMaxCand)
     return fail(nullptr, GBMUF_ERR_UNSUPPORTED, "more than 64 ring neighbours per worker");
+  if (cfg->K > 256)
+    return fail(nullptr, GBMUF_ERR_UNSUPPORTED, "more than 256 workers (one staged box holds all K rows)");
+  if (cfg->ld > 0x7fffffffLL)
+    return fail(nullptr, GBMUF_ERR_UNSUPPORTED, "ld above 2^31 - 1 elements");
   if (!theta || !omega || !delta)
     return fail(nullptr, GBMUF_ERR_INVALID_ARG, "theta, omega and delta must not be NULL");
   if (((uintptr_t)theta | (uintptr_t)omega | (uintptr_t)delta) % 128 != 0)
@@ -811,6 +865,7 @@ gbmuf_status gbmuf_create(const gbmuf_config* cfg, void* theta, float* omega, fl
   cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerMultiprocessor, cfg->device);
   ctx->smem_per_sm = v;
   gbmuf_status st = plan_launch(ctx, ctx->tuning, &ctx->launch);
+  if (st == GBMUF_OK) st = build_tensor_maps(ctx, ctx->launch);
   if (st != GBMUF_OK) { g_create_error = ctx->err; delete ctx; return st; }
   e = cudaMalloc(&ctx->d_status, sizeof(int32_t));
   if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(int32_t));
@@ -866,17 +921,21 @@ gbmuf_status gbmuf_set_partition(gbmuf_ctx* ctx, int32_t m, const int64_t* offse
   return GBMUF_OK;
 }
 
-gbmuf_status gbmuf_set_tuning(gbmuf_ctx* ctx, int32_t ncons, int32_t U, int32_t stages,
-                              int32_t ctas, int32_t unroll) {
+gbmuf_status gbmuf_set_tuning(gbmuf_ctx* ctx, int32_t ncons, int32_t tile_elems, int32_t stages,
+                              int32_t ctas, int32_t flags) {
   if (!ctx) return GBMUF_ERR_INVALID_ARG;
-  if ((ncons != 0 && ncons != 128 && ncons != 256) || U < 0 || U > 64 || stages < 0 ||
-      stages > kMaxStages || ctas < 0 || ctas > 4 || (unroll != 0 && unroll != 1 && unroll != 2 && unroll != 4))
+  if (ncons < 0 || ncons > 992 || ncons % 32 != 0 || tile_elems < 0 || tile_elems > (1 << 16) ||
+      stages < 0 || stages > kMaxStages || ctas < 0 || ctas > 8 || flags < 0 || flags > 1)
     return fail(ctx, GBMUF_ERR_INVALID_ARG, "tuning value out of range");
   Tuning t;
-  t.ncons = ncons; t.U = U; t.stages = stages; t.ctas = ctas; t.unroll = unroll;
+  t.ncons = ncons; t.T = tile_elems; t.stages = stages; t.ctas = ctas; t.flags = flags;
   Launch L;
   gbmuf_status st = plan_launch(ctx, t, &L);
   if (st != GBMUF_OK) return st;
+  DeviceGuard guard(ctx->cfg.device);
+  if (!guard.ok) return fail(ctx, GBMUF_ERR_CUDA, "cudaSetDevice failed");
+  st = build_tensor_maps(ctx, L);
+  if (st != GBMUF_OK) { build_tensor_maps(ctx, ctx->launch); return st; }
   ctx->tuning = t;
   ctx->launch = L;
   return GBMUF_OK;
@@ -976,21 +1035,15 @@ gbmuf_status gbmuf_sync_round(gbmuf_ctx* ctx, uint64_t round, const uint8_t* com
   P.eta = ctx->cfg.eta; P.zeta = ctx->cfg.zeta;
   const int qp1 = ctx->cfg.q + 1;
   P.qp1 = (float)qp1; P.inv_qp1 = 1.0f / (float)qp1; P.inv_exact = (qp1 & (qp1 - 1)) == 0;
-  P.T = L.T; P.U = L.U; P.stages = L.stages; P.ncons = L.ncons;
-  P.stage_stride = L.stage_stride; P.nbr_off = L.nbr_off; P.desc_off = L.desc_off;
+  P.T = L.T; P.BW = L.BW; P.stages = L.stages; P.ncons = L.ncons;
+  if (L.T > L.BW) { P.bw_shift = 8; P.bw_mask = 255; }      // several boxes of 256 columns
+  else { P.bw_shift = 30; P.bw_mask = (1 << 30) - 1; }       // one box
+  P.stage_stride = L.stage_stride; P.omega_off = L.omega_off; P.delta_off = L.delta_off;
+  P.nbr_off = L.nbr_off; P.desc_off = L.desc_off;
   const long long cap = (long long)ctx->num_sms * L.ctas;
   const int grid = (int)(total < cap ? total : cap);
-  const int ui = L.unroll == 1 ? 0 : L.unroll == 2 ? 1 : 2;
-  if (ctx->cfg.theta_dtype == GBMUF_F32) {
-    bool* a = &ctx->attr_set[0][ui];
-    return ui == 0 ? launch_sync<float, 1>(ctx, P, grid, st, a)
-         : ui == 1 ? launch_sync<float, 2>(ctx, P, grid, st, a)
-                   : launch_sync<float, 4>(ctx, P, grid, st, a);
-  }
-  bool* a = &ctx->attr_set[1][ui];
-  return ui == 0 ? launch_sync<__nv_bfloat16, 1>(ctx, P, grid, st, a)
-       : ui == 1 ? launch_sync<__nv_bfloat16, 2>(ctx, P, grid, st, a)
-                 : launch_sync<__nv_bfloat16, 4>(ctx, P, grid, st, a);
+  if (ctx->cfg.theta_dtype == GBMUF_F32) return launch_sync<float>(ctx, P, grid, st, &ctx->attr_set[0]);
+  return launch_sync<__nv_bfloat16>(ctx, P, grid, st, &ctx->attr_set[1]);
 }
 
 gbmuf_status gbmuf_get_neighbors(gbmuf_ctx* ctx, uint64_t round, int32_t* out) {

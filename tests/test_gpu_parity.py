@@ -78,12 +78,14 @@ def test_ragged_shapes(K, offsets, p, q, dtype):
 
 
 @pytest.mark.parametrize("tuning", [
-    dict(consumer_threads=128, vectors_per_thread=1, stages=1, ctas_per_sm=1, unroll=1),
-    dict(consumer_threads=128, vectors_per_thread=1, stages=3, ctas_per_sm=2, unroll=2),
-    dict(consumer_threads=256, vectors_per_thread=1, stages=2, ctas_per_sm=1, unroll=4),
-    dict(consumer_threads=256, vectors_per_thread=2, stages=1, ctas_per_sm=1, unroll=2),
-    dict(consumer_threads=128, vectors_per_thread=4, stages=3, ctas_per_sm=1, unroll=1),
-    dict(consumer_threads=128, vectors_per_thread=2, stages=6, ctas_per_sm=1, unroll=4),
+    dict(consumer_threads=32, tile_elems=64, stages=1, ctas_per_sm=1),
+    dict(consumer_threads=128, tile_elems=256, stages=3, ctas_per_sm=2),
+    dict(consumer_threads=256, tile_elems=512, stages=2, ctas_per_sm=1),
+    dict(consumer_threads=512, tile_elems=1024, stages=1, ctas_per_sm=1),
+    dict(consumer_threads=96, tile_elems=200, stages=8, ctas_per_sm=1),
+    dict(consumer_threads=992, tile_elems=768, stages=2, ctas_per_sm=1),
+    dict(consumer_threads=256, tile_elems=2048, stages=1, ctas_per_sm=1),
+    dict(consumer_threads=512, tile_elems=512, stages=2, ctas_per_sm=1, flags=1),
 ])
 @pytest.mark.parametrize("dtype", [0, 1])
 def test_launch_shapes_agree(tuning, dtype):
@@ -99,7 +101,7 @@ def test_many_tiles_per_cta():
     K, N = 4, 6_000_011
     case = Case(K=K, offsets=(0, 1_000_000, 1_000_001, 3_999_999, N), p=1, q=1, seed=9)
     run(case, random_theta0(N, seed=3), rounds=2,
-        tuning=dict(consumer_threads=128, vectors_per_thread=1, stages=2, ctas_per_sm=1, unroll=2))
+        tuning=dict(consumer_threads=128, tile_elems=512, stages=2, ctas_per_sm=1))
 
 
 # ------------------------------------------------------------------------------------------------
@@ -212,16 +214,20 @@ def test_call_order_and_argument_errors():
     with pytest.raises(binding.GbmufError):
         g.set_tuning(consumer_threads=100)
     with pytest.raises(binding.GbmufError):
+        g.set_tuning(tile_elems=100)
+    with pytest.raises(binding.GbmufError):
+        g.set_tuning(tile_elems=1000)
+    with pytest.raises(binding.GbmufError):
         g.local_perturb(2 ** 32, 0.1, 0.1)
     info = g.launch_info()
-    assert info["tiles"] == 2 and info["grid"] == 2 and info["block"] in (160, 288)
+    assert info["tiles"] == 2 and info["grid"] == 2 and info["block"] in (288, 544)
     g.sync_round(1)
     assert g.device_status() == 0
     g.destroy()
     g.destroy()                                          # idempotent
     with pytest.raises(binding.GbmufError) as e:         # K too large for one staged tile
-        big = torch.zeros((2000, 32), device=dev)
-        binding.Gbmuf(big, big, big, K=2000, N=32, ld=32, p=1, q=1, eta=0.9, zeta=1.0)
+        big = torch.zeros((300, 32), device=dev)
+        binding.Gbmuf(big, big, big, K=300, N=32, ld=32, p=1, q=1, eta=0.9, zeta=1.0)
     assert e.value.status == binding.ERR_UNSUPPORTED
 
 
