@@ -291,7 +291,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="gbmuf", choices=["gbmuf", "reference"])
     ap.add_argument("--workload", default="wikitext103")
-    ap.add_argument("--tuning", default="", help="consumer_threads,tile_elems,stages,ctas_per_sm,flags")
+    ap.add_argument("--tuning", default="", help="consumer_threads,tile_elems,theta_stages,ring_slots,flags")
     ap.add_argument("--ref-cols", type=int, default=1 << 23,
                     help="columns of the workload the CPU oracle is timed on")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -131,17 +131,18 @@ gbmuf_status gbmuf_final_average(gbmuf_ctx* ctx, void* out_device, void* stream)
  * early and the buffers' contents are unspecified. */
 gbmuf_status gbmuf_device_status(gbmuf_ctx* ctx, void* stream, int32_t* out);
 
-/* Launch shape of the fused kernel.  Any argument may be 0 to keep the built-in choice.
- * consumer_threads: multiple of 32 in 32..992 (one more warp issues the copies); tile_elems:
- * elements of one component staged per work item, a multiple of 8; stages: 1..8 tiles in flight
- * per CTA; ctas_per_sm: 1..8 resident CTAs the grid is sized for; flags: bit 0 = give the staged
- * loads an evict-first L2 policy.
+/* Launch shape of the fused kernel (one persistent CTA per SM).  Any argument may be 0 to keep
+ * the built-in choice.  consumer_threads: multiple of 32 in 32..992 (one more warp issues the
+ * copies); tile_elems: elements of one component staged per work item for all K workers, a
+ * multiple of 8 and, above 256, of 256; theta_stages: 1 or 2 tiles of theta resident per CTA;
+ * ring_slots: 2..8 rows of omega/Delta in flight; flags: bit 0 = 256-byte L2 promotion for the
+ * theta loads (default 128).
  * Errors: INVALID_ARG, UNSUPPORTED (does not fit shared memory). */
 gbmuf_status gbmuf_set_tuning(gbmuf_ctx* ctx, int32_t consumer_threads, int32_t tile_elems,
-                              int32_t stages, int32_t ctas_per_sm, int32_t flags);
+                              int32_t theta_stages, int32_t ring_slots, int32_t flags);
 
 /* What the next full round would launch: tiles (work items), grid and block size, dynamic shared
- * memory in bytes, elements per tile, stages.  Any out pointer may be NULL.  Requires
+ * memory in bytes, elements per tile, theta stages.  Any out pointer may be NULL.  Requires
  * set_partition. */
 gbmuf_status gbmuf_get_launch_info(gbmuf_ctx* ctx, int64_t* tiles, int32_t* grid, int32_t* block,
                                    int32_t* smem_bytes, int32_t* tile_elems, int32_t* stages);

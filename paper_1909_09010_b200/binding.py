@@ -149,9 +149,9 @@ class Gbmuf:
         self._check(lib().gbmuf_device_status(self._h, _stream(stream), ctypes.byref(v)))
         return v.value
 
-    def set_tuning(self, consumer_threads=0, tile_elems=0, stages=0, ctas_per_sm=0, flags=0):
-        self._check(lib().gbmuf_set_tuning(self._h, consumer_threads, tile_elems, stages,
-                                           ctas_per_sm, flags))
+    def set_tuning(self, consumer_threads=0, tile_elems=0, theta_stages=0, ring_slots=0, flags=0):
+        self._check(lib().gbmuf_set_tuning(self._h, consumer_threads, tile_elems, theta_stages,
+                                           ring_slots, flags))
 
     def launch_info(self) -> dict:
         tiles = ctypes.c_int64()

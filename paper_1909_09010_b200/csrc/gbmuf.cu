@@ -55,7 +55,6 @@ constexpr uint32_t kTagSampler = 0x53414D50u;  // second key word of the neighbo
 constexpr uint32_t kTagPerturb = 0x50455254u;  // second key word of the local-step noise stream
 constexpr int kMaxCand = 64;                   // largest candidate set min(2p, K-1)
 constexpr int kAlign = 8;                      // tiles start on multiples of 8 elements (>= 16 B)
-constexpr int kMaxStages = 8;
 
 // =================================================================================================
 // Round set-up: neighbour draws (Algorithm 1: "randomly choose q neighbors k_1..k_q") and the
@@ -204,6 +203,17 @@ __device__ __forceinline__ void tma_load_box(uint32_t dst_smem, const CUtensorMa
       : "memory");
 }
 
+// One-dimensional bulk copy global -> shared through the copy engine (no multicast); completion
+// is counted in bytes on the mbarrier.  Addresses and size are multiples of 16 bytes.
+__device__ __forceinline__ void bulk_load_row(uint32_t dst_smem, const void* src, uint32_t bytes,
+                                              uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+          dst_smem),
+      "l"(src), "r"(bytes), "r"(bar)
+      : "memory");
+}
+
 // =================================================================================================
 // theta storage types
 // =================================================================================================
@@ -251,20 +261,29 @@ template <> struct ThetaTraits<__nv_bfloat16> {
 // The fused round: gather + average + block-momentum filter, in place, one pass.
 //
 // Work item = one tile: up to T consecutive elements of ONE component, for all K workers.  A
-// persistent CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...  Warp 0 is the producer: it
-// looks the tile up in the work-list and has the copy engine bring the K replicas' slices of
-// theta, omega and Delta for that tile into a shared-memory stage (one tiled TMA request per
-// [K rows x box-width columns] box, counted on the stage's `full` barrier), running up to
-// `stages` tiles ahead.  The other warps are consumers:
-// each thread takes (16-byte vector, worker) pairs of the tile; it sums the worker's own slice
-// and its q neighbours' slices out of shared memory (own first, then draw order), divides by
-// q+1, applies the filter to the staged omega and Delta and writes Delta, omega and the restart
-// point theta straight to global memory.  All global reads are issued by the copy engine, so
-// the bytes in flight do not depend on how many threads are resident.  Because the CTA is the
-// only reader and writer of its tile in all K replicas and has staged the pre-round values
-// before writing any, every neighbour read sees the replica as it was before the round.  Unique
-// traffic per replica-parameter: theta read once, omega and Delta read once, all three written
-// once.
+// persistent CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...
+//
+// Shared memory holds (a) one or two theta stages, each the K replicas' slices of a tile -- every
+// worker's average may need any other worker's slice, so the whole K-row tile must be resident --
+// and (b) a small ring of row slots for omega and Delta, which are needed exactly once per
+// (worker, element) and therefore only pass through.  Keeping omega and Delta out of the tile
+// stage is what lets T, the contiguous run per row, be as long as 8 KB: measured DRAM efficiency
+// grows with that run length far more than with pipeline depth.
+//
+// Warp 0 is the producer.  Per tile it looks the tile up in the work-list, has the copy engine
+// fetch the theta stage (tiled TMA, one request per [K rows x 256 columns] box) and then, worker by
+// worker, one row of omega and one of Delta into the next free ring slot (bulk copies).  The other
+// warps are consumers: they wait for the theta stage, then for each worker k wait for its ring
+// slot; each thread takes 16-byte vectors of the row, sums worker k's own slice and its q
+// neighbours' slices out of shared memory (own first, then draw order), divides by q+1, applies the
+// filter and writes Delta, omega and the restart point theta straight to global memory, then
+// releases the slot.  All global reads are issued by the copy engine, so the bytes in flight do
+// not depend on how many threads are resident.  Because the CTA is the only reader and writer of
+// its tile in all K replicas and has staged the pre-round theta before writing any, every
+// neighbour read sees the replica as it was before the round.  Unique traffic per
+// replica-parameter: theta read once, omega and Delta read once, all three written once.
+//
+// Every wait is bounded; a wait that expires records GBMUF_ERR_TIMEOUT and the thread leaves.
 // =================================================================================================
 struct TileDesc {
   long long e0;   // first element of the staged range (multiple of kAlign)
@@ -273,6 +292,11 @@ struct TileDesc {
   int comp;
   int pad;
 };
+
+constexpr int kMaxRing = 8;
+// barrier block at the start of shared memory (8 bytes each)
+constexpr uint32_t kBarThetaFull = 0, kBarThetaEmpty = 16, kBarRingFull = 32, kBarRingEmpty = 96;
+constexpr uint32_t kBarBytes = 256;
 
 struct SyncParams {
   void* theta;
@@ -286,9 +310,11 @@ struct SyncParams {
   int K, m, q, mode;
   float eta, zeta, qp1, inv_qp1;
   int inv_exact;        // q+1 is a power of two: multiplying by 1/(q+1) equals dividing
-  int T, BW, bw_shift, bw_mask, stages, ncons;   // BW: columns per TMA box; column c of a tile is
-                                                 // in box c >> bw_shift at c & bw_mask
-  uint32_t stage_stride, omega_off, delta_off, nbr_off, desc_off;
+  int T, BW, bw_shift, bw_mask;   // BW: columns per TMA box; column c of a tile is in box
+                                  // c >> bw_shift at c & bw_mask
+  int stages, ring, ncons;        // theta stages (1 or 2), ring slots, consumer threads
+  uint32_t stage_stride, nbr_off, desc_off;   // theta stage: [theta boxes | nbr | desc]
+  uint32_t ring_off, slot_stride;             // ring slot: [omega row T floats | Delta row T floats]
 };
 
 // Block-momentum filter for one element (Algorithm 1: G, Delta, omega, theta lines).  The
@@ -306,24 +332,27 @@ __device__ __forceinline__ void bmuf_filter(float avg, float& w, float& d, float
 
 template <typename TH>
 __global__ void __launch_bounds__(1024, 1)
-sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_theta,
-                  const __grid_constant__ CUtensorMap map_omega,
-                  const __grid_constant__ CUtensorMap map_delta) {
+sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_theta) {
   constexpr int VEC = ThetaTraits<TH>::VEC;
   constexpr int NF4 = VEC / 4;
   extern __shared__ __align__(128) unsigned char smem[];
-  // [0,64): full barriers, [64,128): empty barriers, then the stages
   const uint32_t bars = smem_u32(smem);
-  unsigned char* stage0 = smem + 128;
+  unsigned char* stage0 = smem + kBarBytes;
+  unsigned char* ring0 = smem + P.ring_off;
   const int total = P.tile_prefix[P.m];
-  const int stages = P.stages;
+  const int S = P.stages, R = P.ring;
   const bool bmuf = P.mode == GBMUF_MODE_BMUF;
+  const int my_tiles = (int)blockIdx.x < total ? (total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < stages; ++s) {
-      mbar_init(bars + 8 * s, 1);                  // full: one arrival (the producer) + bytes
-      mbar_init(bars + 64 + 8 * s, P.ncons);       // empty: every consumer thread arrives
+    for (int s = 0; s < S; ++s) {
+      mbar_init(bars + kBarThetaFull + 8 * s, 1);          // the producer's arrival + bytes
+      mbar_init(bars + kBarThetaEmpty + 8 * s, P.ncons);   // every consumer thread arrives
       reinterpret_cast<TileDesc*>(stage0 + (size_t)s * P.stage_stride + P.desc_off)->comp = -1;
+    }
+    for (int r = 0; r < R; ++r) {
+      mbar_init(bars + kBarRingFull + 8 * r, 1);
+      mbar_init(bars + kBarRingEmpty + 8 * r, P.ncons);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -333,14 +362,13 @@ sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_th
   if (threadIdx.x < 32) {
     // ------------------------------------------------------------------ producer warp
     const int lane = threadIdx.x;
-    int issued = 0;
     bool ok = true;
     // The tiles of this CTA come in increasing order, so the component only ever moves forward:
     // find the first one by bisection, then advance.  In the steady state the loop below touches
-    // no global memory except through the bulk copies.
+    // no global memory except through the copies it issues.
     int comp = 0, pfx_lo = 0, pfx_hi = 0;
     long long cb = 0, ce = 0;
-    if (blockIdx.x < total) {
+    if (my_tiles > 0) {
       int lo_i = 0, hi_i = P.m;
       while (hi_i - lo_i > 1) {
         const int mid = (lo_i + hi_i) >> 1;
@@ -352,12 +380,18 @@ sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_th
       cb = __ldg(P.off + comp);
       ce = __ldg(P.off + comp + 1);
     }
-    for (int it = 0, w = blockIdx.x; w < total; w += gridDim.x, ++it) {
-      const int s = it % stages;
-      if (it >= stages) {
-        ok = mbar_wait_bounded(bars + 64 + 8 * s, ((it / stages) - 1) & 1, P.status);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
+    int theta_issued = 0;    // tiles whose theta stage has been requested
+    int ring_issued = 0;     // ring slots requested so far (over all tiles)
+    int ring_tile_done = 0;  // tiles whose omega/Delta rows have all been requested
+
+    // request the theta stage of this CTA's j-th tile (j = theta_issued)
+    auto issue_theta = [&]() -> bool {
+      const int j = theta_issued;
+      const int w = (int)blockIdx.x + j * (int)gridDim.x;
+      const int s = j % S;
+      if (j >= S) {
+        bool fine = mbar_wait_bounded(bars + kBarThetaEmpty + 8 * s, ((j / S) - 1) & 1, P.status);
+        if (!__all_sync(0xffffffffu, fine)) return false;
       }
       if (w >= pfx_hi) {
         while (w >= pfx_hi) {      // w < total = tile_prefix[m], so comp stays below m
@@ -384,116 +418,145 @@ sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_th
         d->comp = comp;
       }
       __syncwarp();
-      const uint32_t full = bars + 8 * s;
-      const uint32_t row_bytes = (uint32_t)sizeof(TH) + (bmuf ? 8u : 0u);
-      if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)P.K * (uint32_t)P.T * row_bytes);
+      const uint32_t full = bars + kBarThetaFull + 8 * s;
+      if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)P.K * (uint32_t)P.T * (uint32_t)sizeof(TH));
       __syncwarp();
       const uint32_t sbase = smem_u32(st);
-      const int nbox = P.T / P.BW;
-      const int ncopies = (bmuf ? 3 : 1) * nbox;
-      for (int x = lane; x < ncopies; x += 32) {
-        const int arr = x / nbox, b = x - arr * nbox;
-        const int col = (int)e0 + b * P.BW;
-        const uint32_t box_elems = (uint32_t)P.K * (uint32_t)P.BW;
-        if (arr == 0)
-          tma_load_box(sbase + (uint32_t)b * box_elems * (uint32_t)sizeof(TH), &map_theta, col, 0, full);
-        else if (arr == 1)
-          tma_load_box(sbase + P.omega_off + (uint32_t)b * box_elems * 4u, &map_omega, col, 0, full);
-        else
-          tma_load_box(sbase + P.delta_off + (uint32_t)b * box_elems * 4u, &map_delta, col, 0, full);
+      const uint32_t box_bytes = (uint32_t)P.K * (uint32_t)P.BW * (uint32_t)sizeof(TH);
+      for (int b = lane; b < P.T / P.BW; b += 32)
+        tma_load_box(sbase + (uint32_t)b * box_bytes, &map_theta, (int)e0 + b * P.BW, 0, full);
+      ++theta_issued;
+      return true;
+    };
+
+    for (int j = 0; j < S - 1 && j < my_tiles && ok; ++j) ok = issue_theta();
+    for (int it = 0; it < my_tiles && ok; ++it) {
+      if (it + S - 1 < my_tiles) ok = issue_theta();   // keeps S-1 tiles of theta ahead (S=1: this tile)
+      if (!ok) break;
+      if (bmuf) {
+        const TileDesc* d = reinterpret_cast<const TileDesc*>(stage0 + (size_t)(it % S) * P.stage_stride + P.desc_off);
+        const long long e0 = d->e0;
+        long long run = P.ld - e0;                       // a row ends at ld: never read past it
+        if (run > P.T) run = P.T;
+        const uint32_t bytes = (uint32_t)run * 4u;
+        for (int k = 0; k < P.K; ++k) {
+          const int slot = ring_issued % R;
+          if (ring_issued >= R) {
+            bool fine = mbar_wait_bounded(bars + kBarRingEmpty + 8 * slot, ((ring_issued / R) - 1) & 1, P.status);
+            ok = __all_sync(0xffffffffu, fine);
+            if (!ok) break;
+          }
+          if (lane == 0) {
+            const uint32_t full = bars + kBarRingFull + 8 * slot;
+            const uint32_t dst = smem_u32(ring0 + (size_t)slot * P.slot_stride);
+            const long long at = (long long)k * P.ld + e0;
+            mbar_arrive_expect_tx(full, 2u * bytes);
+            bulk_load_row(dst, P.omega + at, bytes, full);
+            bulk_load_row(dst + (uint32_t)P.T * 4u, P.delta + at, bytes, full);
+          }
+          ++ring_issued;
+        }
+        if (ok) ++ring_tile_done;
       }
-      issued = it + 1;
     }
     if (!ok) {
-      // leave only after the copies already issued into this CTA's shared memory have landed
-      for (int it = issued > stages ? issued - stages : 0; it < issued; ++it)
-        mbar_wait_bounded(bars + 8 * (it % stages), (it / stages) & 1, P.status);
+      // leave only after the copies already requested into this CTA's shared memory have landed
+      for (int j = theta_issued > S ? theta_issued - S : 0; j < theta_issued; ++j)
+        mbar_wait_bounded(bars + kBarThetaFull + 8 * (j % S), (j / S) & 1, P.status);
+      for (int j = ring_issued > R ? ring_issued - R : 0; j < ring_issued; ++j)
+        mbar_wait_bounded(bars + kBarRingFull + 8 * (j % R), (j / R) & 1, P.status);
     }
+    (void)ring_tile_done;
     return;
   }
 
   // -------------------------------------------------------------------- consumer warps
   const int c = threadIdx.x - 32;
-  const int nv = P.T / VEC;            // vectors per staged row
-  const int items = nv * P.K;          // (vector, worker) pairs per tile
+  const int nv = P.T / VEC;            // vectors per row of a tile
   const int q = P.q, BW = P.BW, box_elems = P.K * P.BW;
-  // pair p = c, c + ncons, ... is (worker p / nv, vector p % nv); stepped without dividing
-  const int dk = P.ncons / nv, dv = P.ncons - dk * nv;
-  const int k_first = c / nv, v_first = c - k_first * nv;
   TH* theta = static_cast<TH*>(P.theta);
-  for (int it = 0, w = blockIdx.x; w < total; w += gridDim.x, ++it) {
-    const int s = it % stages;
-    if (!mbar_wait_bounded(bars + 8 * s, (it / stages) & 1, P.status)) return;
+  int ring_taken = 0;
+  for (int it = 0; it < my_tiles; ++it) {
+    const int s = it % S;
+    if (!mbar_wait_bounded(bars + kBarThetaFull + 8 * s, (it / S) & 1, P.status)) return;
     unsigned char* st = stage0 + (size_t)s * P.stage_stride;
     const TH* sth = reinterpret_cast<const TH*>(st);
-    const float* som = reinterpret_cast<const float*>(st + P.omega_off);
-    const float* sde = reinterpret_cast<const float*>(st + P.delta_off);
     const int* snb = reinterpret_cast<const int*>(st + P.nbr_off);
     const TileDesc* d = reinterpret_cast<const TileDesc*>(st + P.desc_off);
     const long long e0 = d->e0, lo = d->lo, hi = d->hi;
-    int k_walk = k_first, v_walk = v_first;
-#pragma unroll 2
-    for (int p = c; p < items; p += P.ncons) {
-      const int k = k_walk, col = v_walk * VEC;
-      k_walk += dk;
-      v_walk += dv;
-      if (v_walk >= nv) { v_walk -= nv; ++k_walk; }
-      const long long e = e0 + col;
-      if (e >= hi || e + VEC <= lo) continue;
-      // gossip average: own slice first, then the neighbours in draw order
-      // staged layout: box b = col / BW holds K rows of BW columns
-      const int b = col >> P.bw_shift, cin = col & P.bw_mask;
-      const int boxbase = b * box_elems + cin;
-      float a[VEC], t[VEC];
-      ThetaTraits<TH>::lds(sth + boxbase + k * BW, a);
-      for (int j = 0; j < q; ++j) {
-        ThetaTraits<TH>::lds(sth + boxbase + snb[k * q + j] * BW, t);
-#pragma unroll
-        for (int x = 0; x < VEC; ++x) a[x] = __fadd_rn(a[x], t[x]);
+    for (int k = 0; k < P.K; ++k) {
+      const float* som = nullptr;
+      const float* sde = nullptr;
+      int slot = 0;
+      if (bmuf) {
+        slot = ring_taken % R;
+        if (!mbar_wait_bounded(bars + kBarRingFull + 8 * slot, (ring_taken / R) & 1, P.status)) return;
+        som = reinterpret_cast<const float*>(ring0 + (size_t)slot * P.slot_stride);
+        sde = som + P.T;
       }
+      for (int v = c; v < nv; v += P.ncons) {
+        const int col = v * VEC;
+        const long long e = e0 + col;
+        if (e >= hi || e + VEC <= lo) continue;
+        // staged layout of theta: box b = col / BW holds K rows of BW columns
+        const int b = col >> P.bw_shift, cin = col & P.bw_mask;
+        const int boxbase = b * box_elems + cin;
+        // gossip average: own slice first, then the neighbours in draw order
+        float a[VEC], t[VEC];
+        ThetaTraits<TH>::lds(sth + boxbase + k * BW, a);
+        for (int j = 0; j < q; ++j) {
+          ThetaTraits<TH>::lds(sth + boxbase + snb[k * q + j] * BW, t);
 #pragma unroll
-      for (int x = 0; x < VEC; ++x)
-        a[x] = P.inv_exact ? __fmul_rn(a[x], P.inv_qp1) : __fdiv_rn(a[x], P.qp1);
-      const long long at = (long long)k * P.ld + e;
-      const bool whole = e >= lo && e + VEC <= hi;
-      if (!bmuf) {                                       // gossip-MA: theta <- average
-        if (whole) {
-          ThetaTraits<TH>::stg(theta + at, a);
-        } else {
-          for (int x = 0; x < VEC; ++x)
-            if (e + x >= lo && e + x < hi) theta[at + x] = ThetaTraits<TH>::narrow(a[x]);
+          for (int x = 0; x < VEC; ++x) a[x] = __fadd_rn(a[x], t[x]);
         }
-        continue;
-      }
-      float4 W[NF4], D[NF4];
 #pragma unroll
-      for (int f = 0; f < NF4; ++f) {
-        W[f] = *reinterpret_cast<const float4*>(som + boxbase + k * BW + 4 * f);
-        D[f] = *reinterpret_cast<const float4*>(sde + boxbase + k * BW + 4 * f);
-      }
-      float* wv = reinterpret_cast<float*>(&W[0]);
-      float* dv = reinterpret_cast<float*>(&D[0]);
-#pragma unroll
-      for (int x = 0; x < VEC; ++x) bmuf_filter<TH>(a[x], wv[x], dv[x], t[x], P.eta, P.zeta);
-      if (whole) {
+        for (int x = 0; x < VEC; ++x)
+          a[x] = P.inv_exact ? __fmul_rn(a[x], P.inv_qp1) : __fdiv_rn(a[x], P.qp1);
+        const long long at = (long long)k * P.ld + e;
+        const bool whole = e >= lo && e + VEC <= hi;
+        if (!bmuf) {                                       // gossip-MA: theta <- average
+          if (whole) {
+            ThetaTraits<TH>::stg(theta + at, a);
+          } else {
+            for (int x = 0; x < VEC; ++x)
+              if (e + x >= lo && e + x < hi) theta[at + x] = ThetaTraits<TH>::narrow(a[x]);
+          }
+          continue;
+        }
+        float4 W[NF4], D[NF4];
 #pragma unroll
         for (int f = 0; f < NF4; ++f) {
-          __stcs(reinterpret_cast<float4*>(P.delta + at) + f, D[f]);
-          __stcs(reinterpret_cast<float4*>(P.omega + at) + f, W[f]);
+          W[f] = *reinterpret_cast<const float4*>(som + col + 4 * f);
+          D[f] = *reinterpret_cast<const float4*>(sde + col + 4 * f);
         }
-        ThetaTraits<TH>::stg(theta + at, t);
-      } else {
-        // a vector that straddles the edge of the component: only the elements this tile owns
-        for (int x = 0; x < VEC; ++x) {
-          if (e + x >= lo && e + x < hi) {
-            P.delta[at + x] = dv[x];
-            P.omega[at + x] = wv[x];
-            theta[at + x] = ThetaTraits<TH>::narrow(t[x]);
+        float* wv = reinterpret_cast<float*>(&W[0]);
+        float* dv = reinterpret_cast<float*>(&D[0]);
+#pragma unroll
+        for (int x = 0; x < VEC; ++x) bmuf_filter<TH>(a[x], wv[x], dv[x], t[x], P.eta, P.zeta);
+        if (whole) {
+#pragma unroll
+          for (int f = 0; f < NF4; ++f) {
+            __stcs(reinterpret_cast<float4*>(P.delta + at) + f, D[f]);
+            __stcs(reinterpret_cast<float4*>(P.omega + at) + f, W[f]);
+          }
+          ThetaTraits<TH>::stg(theta + at, t);
+        } else {
+          // a vector that straddles the edge of the component: only the elements this tile owns
+          for (int x = 0; x < VEC; ++x) {
+            if (e + x >= lo && e + x < hi) {
+              P.delta[at + x] = dv[x];
+              P.omega[at + x] = wv[x];
+              theta[at + x] = ThetaTraits<TH>::narrow(t[x]);
+            }
           }
         }
       }
+      if (bmuf) {
+        mbar_arrive(bars + kBarRingEmpty + 8 * slot);    // this thread is done with the slot
+        ++ring_taken;
+      }
     }
-    mbar_arrive(bars + 64 + 8 * s);   // this thread has finished reading the stage
+    mbar_arrive(bars + kBarThetaEmpty + 8 * s);          // this thread is done with the theta stage
   }
 }
 
@@ -590,12 +653,12 @@ __global__ void __launch_bounds__(256) final_average_kernel(const TH* theta, TH*
 thread_local std::string g_create_error;
 
 struct Tuning {
-  int ncons = 0, T = 0, stages = 0, ctas = 0, flags = 0;   // 0 = built-in choice
+  int ncons = 0, T = 0, stages = 0, ring = 0, flags = 0;   // 0 = built-in choice
 };
 
 struct Launch {
-  int ncons, stages, ctas, T, BW, flags;
-  uint32_t stage_stride, omega_off, delta_off, nbr_off, desc_off, smem;
+  int ncons, stages, ring, T, BW, flags;
+  uint32_t stage_stride, nbr_off, desc_off, ring_off, slot_stride, smem;
 };
 
 int host_candidates(int K, int p) {
@@ -629,7 +692,7 @@ struct gbmuf_ctx {
   int smem_per_sm = 0;
   Tuning tuning;
   Launch launch;
-  CUtensorMap map_theta, map_omega, map_delta;   // boxes [K][launch.BW] over the [K][ld] arrays
+  CUtensorMap map_theta;   // boxes [K rows][launch.BW columns] over theta
   bool attr_set[2] = {false, false};
   std::string err;
 };
@@ -665,7 +728,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// Tensor maps for boxes of K rows x BW columns over the three [K][ld] arrays.
+// Tensor map for boxes of K rows x BW columns over the [K][ld] theta array.
 gbmuf_status build_tensor_maps(gbmuf_ctx* ctx, const Launch& L) {
   static EncodeTiledFn encode = nullptr;
   if (!encode) {
@@ -682,77 +745,80 @@ gbmuf_status build_tensor_maps(gbmuf_ctx* ctx, const Launch& L) {
   const cuuint32_t estr[2] = {1, 1};
   const CUtensorMapL2promotion prom =
       (L.flags & 1) ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B;
-  struct { CUtensorMap* map; void* base; CUtensorMapDataType dt; cuuint64_t esz; } arr[3] = {
-      {&ctx->map_theta, ctx->theta,
-       ctx->cfg.theta_dtype == GBMUF_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
-       (cuuint64_t)theta_size(ctx)},
-      {&ctx->map_omega, ctx->omega, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4},
-      {&ctx->map_delta, ctx->delta, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4}};
-  for (auto& a : arr) {
-    const cuuint64_t gstride[1] = {ld * a.esz};
-    CUresult r = encode(a.map, a.dt, 2, a.base, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                        CU_TENSOR_MAP_SWIZZLE_NONE, prom, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS)
-      return fail(ctx, GBMUF_ERR_CUDA, "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r));
-  }
+  const cuuint64_t esz = (cuuint64_t)theta_size(ctx);
+  const cuuint64_t gstride[1] = {ld * esz};
+  CUresult r = encode(&ctx->map_theta,
+                      ctx->cfg.theta_dtype == GBMUF_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                                        : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+                      2, ctx->theta, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                      CU_TENSOR_MAP_SWIZZLE_NONE, prom, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS)
+    return fail(ctx, GBMUF_ERR_CUDA, "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r));
   return GBMUF_OK;
 }
 
 // Choose (or check) the launch shape of the fused kernel for this K, q, mode and dtype.
+// Shared memory: 256 bytes of barriers, `stages` theta stages of K*T elements (+ neighbour table
+// and descriptor), and in BMUF mode `ring` slots of 2*T floats.
 gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
   const int K = ctx->cfg.K, q = ctx->cfg.q;
   const int esz = (int)theta_size(ctx);
+  const int VEC = 16 / esz;
   const bool bmuf = ctx->cfg.mode == GBMUF_MODE_BMUF;
   Launch L;
-  L.ctas = t.ctas ? t.ctas : 1;
   L.flags = t.flags;
-  const long long budget = (long long)ctx->smem_per_sm / L.ctas - 1024;   // per CTA, bytes
-  const long long cap = budget < ctx->max_smem ? budget : ctx->max_smem;
-  auto layout = [&](int T, Launch* l) {
-    long long at = (long long)K * T * esz;                 // theta rows
-    at = (at + 127) / 128 * 128;
-    if (l) l->omega_off = (uint32_t)at;
-    if (bmuf) at += (long long)K * T * 4;
-    at = (at + 127) / 128 * 128;
-    if (l) l->delta_off = (uint32_t)at;
-    if (bmuf) at += (long long)K * T * 4;
-    at = (at + 15) / 16 * 16;
+  const long long cap = ctx->max_smem < ctx->smem_per_sm - 1024 ? ctx->max_smem : ctx->smem_per_sm - 1024;
+  auto stage_bytes = [&](int T, Launch* l) {
+    long long at = ((long long)K * T * esz + 15) / 16 * 16;
     if (l) l->nbr_off = (uint32_t)at;
-    at += (long long)K * q * 4;
-    at = (at + 15) / 16 * 16;
+    at = (at + (long long)K * q * 4 + 15) / 16 * 16;
     if (l) l->desc_off = (uint32_t)at;
     at += (long long)sizeof(TileDesc);
     return (at + 127) / 128 * 128;
   };
+  auto total_bytes = [&](int T, int S, int R) {
+    return (long long)kBarBytes + S * stage_bytes(T, nullptr) + (bmuf ? (long long)R * 2 * T * 4 : 0);
+  };
+  const int want_stages = t.stages ? t.stages : 1;
+  auto ring_for = [&](int T) {   // slots used with tile T: the caller's, else as many as fit up to 4
+    if (!bmuf) return 0;
+    if (t.ring) return t.ring;
+    int r = 4;
+    while (r > 2 && total_bytes(T, want_stages, r) > cap) --r;
+    return r;
+  };
   if (t.T) {
     L.T = t.T;
   } else {
-    // the widest tile (longest contiguous run per row) of which one stage still fits
-    long long T = 1024;
-    while (T > 8 && layout((int)T, nullptr) + 128 > cap) T >>= 1;
-    L.T = (int)T;
+    // The widest power-of-two tile (longest contiguous run per row) that fits: measured DRAM
+    // efficiency keeps growing with the run length up to 16 KB, and a tile that is a whole
+    // number of consumer passes keeps every thread busy.
+    int T = 4096;
+    while (T > 8 && total_bytes(T, want_stages, ring_for(T)) > cap) T >>= 1;
+    L.T = T;
   }
+  L.ring = ring_for(L.T);
   if (L.T < kAlign || L.T % kAlign != 0)
     return fail(ctx, GBMUF_ERR_INVALID_ARG, "tile_elems must be a positive multiple of 8");
   if (L.T > 256 && L.T % 256 != 0)
     return fail(ctx, GBMUF_ERR_INVALID_ARG, "tile_elems above 256 must be a multiple of 256");
   L.BW = L.T < 256 ? L.T : 256;                // a tensor-map box is at most 256 elements wide
-  const long long sb = layout(L.T, &L);
-  if (sb + 128 > cap || sb >= (1 << 20))
+  L.stages = t.stages ? t.stages : 1;
+  if ((long long)K * L.T * esz >= (1 << 20) || total_bytes(L.T, L.stages, L.ring) > cap)
     return fail(ctx, GBMUF_ERR_UNSUPPORTED,
-                "one staged tile (K rows of theta, omega and Delta) does not fit the shared "
-                "memory available per CTA");
-  if (t.stages) {
-    L.stages = t.stages;
-  } else {
-    L.stages = (int)((cap - 128) / sb);
-    if (L.stages > 4) L.stages = 4;
-  }
-  if (L.stages < 1 || L.stages > kMaxStages || 128 + (long long)L.stages * sb > cap)
-    return fail(ctx, GBMUF_ERR_UNSUPPORTED, "stages * tile does not fit shared memory");
-  L.ncons = t.ncons ? t.ncons : (L.stages >= 2 ? 256 : 512);
+                "the theta stage(s) (K rows of the tile) and the omega/Delta ring do not fit the "
+                "shared memory of one SM");
+  const long long sb = stage_bytes(L.T, &L);
   L.stage_stride = (uint32_t)sb;
-  L.smem = (uint32_t)(128 + (long long)L.stages * sb);
+  L.ring_off = (uint32_t)(kBarBytes + L.stages * sb);
+  L.slot_stride = (uint32_t)(2 * L.T * 4);
+  L.smem = (uint32_t)total_bytes(L.T, L.stages, L.ring);
+  if (t.ncons) {
+    L.ncons = t.ncons;
+  } else {
+    int n = (L.T / VEC + 31) / 32 * 32;        // one vector per thread and row, within 128..512
+    L.ncons = n < 128 ? 128 : n > 512 ? 512 : n;
+  }
   *out = L;
   return GBMUF_OK;
 }
@@ -779,7 +845,7 @@ gbmuf_status launch_sync(gbmuf_ctx* ctx, const SyncParams& P, int grid, cudaStre
     if (e != cudaSuccess) return cuda_fail(ctx, "cudaFuncSetAttribute", e);
     *attr = true;
   }
-  kern<<<grid, 32 + P.ncons, ctx->launch.smem, st>>>(P, ctx->map_theta, ctx->map_omega, ctx->map_delta);
+  kern<<<grid, 32 + P.ncons, ctx->launch.smem, st>>>(P, ctx->map_theta);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, "launch of the fused round kernel", e);
   return GBMUF_OK;
@@ -922,13 +988,13 @@ gbmuf_status gbmuf_set_partition(gbmuf_ctx* ctx, int32_t m, const int64_t* offse
 }
 
 gbmuf_status gbmuf_set_tuning(gbmuf_ctx* ctx, int32_t ncons, int32_t tile_elems, int32_t stages,
-                              int32_t ctas, int32_t flags) {
+                              int32_t ring, int32_t flags) {
   if (!ctx) return GBMUF_ERR_INVALID_ARG;
   if (ncons < 0 || ncons > 992 || ncons % 32 != 0 || tile_elems < 0 || tile_elems > (1 << 16) ||
-      stages < 0 || stages > kMaxStages || ctas < 0 || ctas > 8 || flags < 0 || flags > 1)
+      stages < 0 || stages > 2 || ring < 0 || ring > kMaxRing || ring == 1 || flags < 0 || flags > 1)
     return fail(ctx, GBMUF_ERR_INVALID_ARG, "tuning value out of range");
   Tuning t;
-  t.ncons = ncons; t.T = tile_elems; t.stages = stages; t.ctas = ctas; t.flags = flags;
+  t.ncons = ncons; t.T = tile_elems; t.stages = stages; t.ring = ring; t.flags = flags;
   Launch L;
   gbmuf_status st = plan_launch(ctx, t, &L);
   if (st != GBMUF_OK) return st;
@@ -947,7 +1013,7 @@ gbmuf_status gbmuf_get_launch_info(gbmuf_ctx* ctx, int64_t* tiles, int32_t* grid
   if (!ctx->partitioned) return fail(ctx, GBMUF_ERR_BAD_STATE, "set_partition has not been called");
   std::vector<uint8_t> all(ctx->m, 1);
   const long long total = host_total_tiles(ctx, 0, all.data(), ctx->launch.T);
-  const long long cap = (long long)ctx->num_sms * ctx->launch.ctas;
+  const long long cap = (long long)ctx->num_sms;
   if (tiles) *tiles = total;
   if (grid) *grid = (int32_t)(total < cap ? total : cap);
   if (block) *block = 32 + ctx->launch.ncons;
@@ -1035,12 +1101,12 @@ gbmuf_status gbmuf_sync_round(gbmuf_ctx* ctx, uint64_t round, const uint8_t* com
   P.eta = ctx->cfg.eta; P.zeta = ctx->cfg.zeta;
   const int qp1 = ctx->cfg.q + 1;
   P.qp1 = (float)qp1; P.inv_qp1 = 1.0f / (float)qp1; P.inv_exact = (qp1 & (qp1 - 1)) == 0;
-  P.T = L.T; P.BW = L.BW; P.stages = L.stages; P.ncons = L.ncons;
+  P.T = L.T; P.BW = L.BW; P.stages = L.stages; P.ring = L.ring; P.ncons = L.ncons;
   if (L.T > L.BW) { P.bw_shift = 8; P.bw_mask = 255; }      // several boxes of 256 columns
   else { P.bw_shift = 30; P.bw_mask = (1 << 30) - 1; }       // one box
-  P.stage_stride = L.stage_stride; P.omega_off = L.omega_off; P.delta_off = L.delta_off;
-  P.nbr_off = L.nbr_off; P.desc_off = L.desc_off;
-  const long long cap = (long long)ctx->num_sms * L.ctas;
+  P.stage_stride = L.stage_stride; P.nbr_off = L.nbr_off; P.desc_off = L.desc_off;
+  P.ring_off = L.ring_off; P.slot_stride = L.slot_stride;
+  const long long cap = (long long)ctx->num_sms;              // one persistent CTA per SM
   const int grid = (int)(total < cap ? total : cap);
   if (ctx->cfg.theta_dtype == GBMUF_F32) return launch_sync<float>(ctx, P, grid, st, &ctx->attr_set[0]);
   return launch_sync<__nv_bfloat16>(ctx, P, grid, st, &ctx->attr_set[1]);
