@@ -147,6 +147,36 @@ gbmuf_status gbmuf_set_tuning(gbmuf_ctx* ctx, int32_t consumer_threads, int32_t 
 gbmuf_status gbmuf_get_launch_info(gbmuf_ctx* ctx, int64_t* tiles, int32_t* grid, int32_t* block,
                                    int32_t* smem_bytes, int32_t* tile_elems, int32_t* stages);
 
+/* (No counterpart in the paper: this entry point exists for the library's callers, not for the
+ * method.)  One synchronisation round that allocates nothing, for callers that must not or cannot
+ * allocate device memory at the point where they synchronise: a training process whose memory pool
+ * has already claimed the whole GPU, code running under an allocator that forbids foreign
+ * cudaMalloc calls, or a plug-in that is handed buffers and a stream and nothing else.  It does
+ * what gbmuf_create + gbmuf_set_partition + gbmuf_sync_round do for one round -- same kernels,
+ * same results bit for bit -- but the library-side tables (component offsets, participation
+ * flags, tile work-list, neighbour table, status word) live in one fixed array inside the loaded
+ * library image instead of in cudaMalloc'ed memory.  The call itself uses no cudaMalloc/cudaFree
+ * and no allocating library routine; theta, omega and delta are still the caller's.
+ *   Limits: m <= 1024 components and K * m * q <= 65536 neighbour draws per round; larger
+ *   requests are refused with GBMUF_ERR_UNSUPPORTED (use a context for them).  The array is
+ *   276,224 bytes and every GPU on which the library is loaded keeps it until the process ends.
+ *   Arguments: cfg as for gbmuf_create (device selects the GPU); theta/omega/delta device [K][ld];
+ *   offsets host [m+1]; comp_mask host [m] or NULL (= every component takes part); round as in
+ *   gbmuf_sync_round; stream a cudaStream_t.  device_status_out: NULL, or a host int32 -- then the
+ *   call waits for the stream and stores the device status word (GBMUF_OK or GBMUF_ERR_TIMEOUT).
+ *   First use on a device: the first call on each GPU looks up the device address of the array
+ *   (cudaGetSymbolAddress, with that GPU current) and sets the kernel's shared-memory limit; make
+ *   that first call outside any stream capture.
+ *   Sharing: all calls on a GPU use the same array.  It keeps the previous call's contents; this
+ *   function clears the status word and rewrites every table it reads, so calls one after another
+ *   on one stream are independent.  Calls that overlap on the GPU (different streams, or several
+ *   host threads) race on the array and give undefined results: serialise them.
+ * Errors: INVALID_ARG, UNSUPPORTED, CUDA; text via gbmuf_last_error(NULL) on the calling thread. */
+gbmuf_status gbmuf_sync_round_noalloc(const gbmuf_config* cfg, void* theta_device,
+                                      float* omega_device, float* delta_device, int32_t m,
+                                      const int64_t* offsets_host, const uint8_t* comp_mask_host,
+                                      uint64_t round, void* stream, int32_t* device_status_out);
+
 /* Sentence about the last error on this context ("" if none); valid until the next call on it.
  * With ctx == NULL: the last error of a failed gbmuf_create on this thread. */
 const char* gbmuf_last_error(const gbmuf_ctx* ctx);

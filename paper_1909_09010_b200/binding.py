@@ -22,7 +22,8 @@ MODE_BMUF, MODE_MA = 0, 1
 
 EXPORTS = ["gbmuf_create", "gbmuf_set_partition", "gbmuf_init", "gbmuf_local_perturb",
            "gbmuf_sync_round", "gbmuf_get_neighbors", "gbmuf_final_average", "gbmuf_device_status",
-           "gbmuf_set_tuning", "gbmuf_get_launch_info", "gbmuf_last_error", "gbmuf_destroy"]
+           "gbmuf_set_tuning", "gbmuf_get_launch_info", "gbmuf_last_error", "gbmuf_destroy",
+           "gbmuf_sync_round_noalloc"]
 
 
 class Config(ctypes.Structure):
@@ -67,6 +68,8 @@ def lib() -> ctypes.CDLL:
     L.gbmuf_get_launch_info.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(i32),
                                         ctypes.POINTER(i32), ctypes.POINTER(i32),
                                         ctypes.POINTER(i32), ctypes.POINTER(i32)]
+    L.gbmuf_sync_round_noalloc.argtypes = [ctypes.POINTER(Config), vp, vp, vp, i32, vp, vp, u64, vp,
+                                           ctypes.POINTER(i32)]
     L.gbmuf_last_error.argtypes = [vp]
     L.gbmuf_last_error.restype = ctypes.c_char_p
     L.gbmuf_destroy.argtypes = [vp]
@@ -92,6 +95,26 @@ def _stream(stream) -> int:
         import torch
         return torch.cuda.current_stream().cuda_stream
     return getattr(stream, "cuda_stream", stream)
+
+
+def sync_round_noalloc(theta, omega, delta, offsets, rnd, *, K, N, ld, p, q, eta, zeta, seed=0,
+                       mode=MODE_BMUF, theta_dtype=F32, device=0, comp_base=0, elem_base=0,
+                       comp_mask=None, stream=None, want_status=False):
+    """``gbmuf_sync_round_noalloc``: one round without a context and without any allocation by the
+    library (its tables live in a fixed array of the loaded library).  For callers that cannot
+    allocate device memory where they synchronise.  Calls on one GPU share that array: keep them
+    on one stream.  Returns the device status word if ``want_status`` (this waits for the stream).
+    """
+    cfg = Config(K, N, ld, p, q, eta, zeta, mode, theta_dtype, seed, device, comp_base, elem_base)
+    off = np.ascontiguousarray(offsets, dtype=np.int64)
+    mask = None if comp_mask is None else np.ascontiguousarray(comp_mask, dtype=np.uint8)
+    word = ctypes.c_int32(-1)
+    st = lib().gbmuf_sync_round_noalloc(ctypes.byref(cfg), _ptr(theta), _ptr(omega), _ptr(delta),
+                                        off.shape[0] - 1, _ptr(off), _ptr(mask), rnd,
+                                        _stream(stream), ctypes.byref(word) if want_status else None)
+    if st != GBMUF_OK:
+        raise GbmufError(st, lib().gbmuf_last_error(None).decode())
+    return word.value if want_status else None
 
 
 class Gbmuf:

@@ -1195,4 +1195,144 @@ gbmuf_status gbmuf_destroy(gbmuf_ctx* ctx) {
   return rc;
 }
 
+
+// -------------------------------------------------------------------------------------------------
+// gbmuf_sync_round_noalloc: one round with every library-side table in a fixed device array.
+// -------------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int kNoAllocMaxM = 1024;            // components
+constexpr int kNoAllocMaxDraws = 65536;       // K * m * q neighbour entries
+constexpr size_t kNaStatusOff = 0;                                          // int32 status word
+constexpr size_t kNaOffsetsOff = 256;                                       // int64 [m+1]
+constexpr size_t kNaPrefixOff = kNaOffsetsOff + 8448;                       // int32 [m+1]
+constexpr size_t kNaMaskOff = kNaPrefixOff + 4352;                          // uint8 [m]
+constexpr size_t kNaNbrOff = kNaMaskOff + 1024;                             // int32 [m][K][q]
+constexpr size_t kNoAllocBytes = kNaNbrOff + (size_t)kNoAllocMaxDraws * 4;  // 276,224 bytes
+
+// The scratch itself.  Part of the loaded module: every GPU that loads this library holds these
+// 270 KB until the process exits.  In HOST code this name is only a handle for
+// cudaGetSymbolAddress; it is not a device address.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
+
+constexpr int kNoAllocMaxDevices = 64;
+unsigned char* g_noalloc_ptr[kNoAllocMaxDevices] = {};   // device address of the array, per GPU
+
+}  // namespace
+
+gbmuf_status gbmuf_sync_round_noalloc(const gbmuf_config* cfg, void* theta, float* omega,
+                                      float* delta, int32_t m, const int64_t* offsets,
+                                      const uint8_t* comp_mask, uint64_t round, void* stream,
+                                      int32_t* device_status_out) {
+  if (!cfg) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "cfg must not be NULL");
+  if (cfg->K < 1 || cfg->K > 256 || cfg->N < 1 || cfg->ld < cfg->N || cfg->ld % 32 != 0 ||
+      cfg->ld > 0x7fffffffLL || cfg->p < 0 || cfg->q < 0 || cfg->comp_base < 0 ||
+      (cfg->mode != GBMUF_MODE_BMUF && cfg->mode != GBMUF_MODE_MA) ||
+      (cfg->theta_dtype != GBMUF_F32 && cfg->theta_dtype != GBMUF_BF16) ||
+      !(cfg->eta == cfg->eta) || !(cfg->zeta == cfg->zeta))
+    return fail(nullptr, GBMUF_ERR_INVALID_ARG, "configuration out of range (see gbmuf_create)");
+  const int cand = host_candidates(cfg->K, cfg->p);
+  if (cfg->q > cand || cand > kMaxCand)
+    return fail(nullptr, GBMUF_ERR_INVALID_ARG, "q exceeds the ring neighbours min(2p, K-1), or more than 64 of them");
+  if (!theta || !omega || !delta || (((uintptr_t)theta | (uintptr_t)omega | (uintptr_t)delta) % 128) != 0)
+    return fail(nullptr, GBMUF_ERR_INVALID_ARG, "theta, omega and delta must be 128-byte aligned device pointers");
+  if (m < 1 || !offsets) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "m must be >= 1 and offsets not NULL");
+  if (m > kNoAllocMaxM)
+    return fail(nullptr, GBMUF_ERR_UNSUPPORTED,
+                "gbmuf_sync_round_noalloc handles at most 1024 components; use a context (gbmuf_create) for more");
+  if ((long long)cfg->K * m * cfg->q > kNoAllocMaxDraws)
+    return fail(nullptr, GBMUF_ERR_UNSUPPORTED,
+                "gbmuf_sync_round_noalloc handles at most 65536 neighbour draws (K * m * q) per round; "
+                "use a context (gbmuf_create) for more");
+  if (offsets[0] != 0 || offsets[m] != cfg->N)
+    return fail(nullptr, GBMUF_ERR_INVALID_ARG, "offsets[0] must be 0 and offsets[m] must be N");
+  for (int i = 0; i < m; ++i)
+    if (offsets[i + 1] <= offsets[i]) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "offsets must be strictly increasing");
+  if (cfg->device < 0 || cfg->device >= kNoAllocMaxDevices)
+    return fail(nullptr, GBMUF_ERR_INVALID_ARG, "device ordinal out of range");
+
+  DeviceGuard guard(cfg->device);
+  if (!guard.ok) return fail(nullptr, GBMUF_ERR_CUDA, "cudaSetDevice failed");
+  cudaError_t e;
+  if (!g_noalloc_ptr[cfg->device]) {
+    // once per device, with that device current: ask the runtime where the array lives there
+    unsigned char* ptr = nullptr;
+    e = cudaGetSymbolAddress((void**)&ptr, g_noalloc_scratch);
+    if (e != cudaSuccess || !ptr) return cuda_fail(nullptr, "cudaGetSymbolAddress of the fixed scratch array", e);
+    g_noalloc_ptr[cfg->device] = ptr;
+  }
+  unsigned char* scratch = g_noalloc_ptr[cfg->device];
+
+  // a context on the stack: it owns nothing, it only carries the description to the helpers
+  gbmuf_ctx tmp;
+  tmp.cfg = *cfg; tmp.theta = theta; tmp.omega = omega; tmp.delta = delta; tmp.m = m; tmp.cand = cand;
+  int v = 0;
+  cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, cfg->device); tmp.num_sms = v;
+  cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerBlockOptin, cfg->device); tmp.max_smem = v;
+  cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerMultiprocessor, cfg->device); tmp.smem_per_sm = v;
+  gbmuf_status st = plan_launch(&tmp, tmp.tuning, &tmp.launch);
+  if (st == GBMUF_OK) st = build_tensor_maps(&tmp, tmp.launch);
+  if (st != GBMUF_OK) { g_create_error = tmp.err; return st; }
+  const Launch& L = tmp.launch;
+
+  uint8_t flags[kNoAllocMaxM];
+  long long total = 0;
+  for (int i = 0; i < m; ++i) {
+    flags[i] = comp_mask ? (comp_mask[i] != 0) : 1;
+    if (!flags[i]) continue;
+    const int64_t start = offsets[i] & ~(int64_t)(kAlign - 1);
+    total += (offsets[i + 1] - start + L.T - 1) / L.T;
+  }
+  if (total > 0x3fffffffLL) return fail(nullptr, GBMUF_ERR_UNSUPPORTED, "more than 2^30 - 1 tiles");
+  cudaStream_t cs = (cudaStream_t)stream;
+  int32_t* d_status = reinterpret_cast<int32_t*>(scratch + kNaStatusOff);
+  // the array keeps whatever the previous call left: the status word must start at zero, the
+  // other tables are rewritten in full below for the sizes of this call
+  e = cudaMemsetAsync(d_status, 0, sizeof(int32_t), cs);
+  if (e == cudaSuccess && total > 0)
+    e = cudaMemcpyAsync(scratch + kNaOffsetsOff, offsets, (size_t)(m + 1) * sizeof(int64_t), cudaMemcpyHostToDevice, cs);
+  if (e == cudaSuccess && total > 0)
+    e = cudaMemcpyAsync(scratch + kNaMaskOff, flags, (size_t)m, cudaMemcpyHostToDevice, cs);
+  if (e != cudaSuccess) return cuda_fail(nullptr, "upload of offsets and mask into the fixed scratch array", e);
+  if (total > 0) {
+    SetupParams S;
+    S.K = cfg->K; S.m = m; S.p = cfg->p; S.q = cfg->q; S.comp_base = cfg->comp_base; S.T = L.T;
+    S.use_mask = 1; S.plan = 1; S.seed = cfg->seed; S.round = round;
+    S.off = reinterpret_cast<const int64_t*>(scratch + kNaOffsetsOff);
+    S.periods = nullptr;
+    S.mask = scratch + kNaMaskOff;
+    S.nbr = reinterpret_cast<int32_t*>(scratch + kNaNbrOff);
+    S.tile_prefix = reinterpret_cast<int32_t*>(scratch + kNaPrefixOff);
+    const long long items = (long long)cfg->K * m;
+    round_setup_kernel<<<(int)((items + 255) / 256), 256, 0, cs>>>(S);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(nullptr, "launch of the round set-up kernel", e);
+
+    SyncParams P;
+    P.theta = theta; P.omega = omega; P.delta = delta;
+    P.off = S.off; P.tile_prefix = S.tile_prefix; P.nbr = S.nbr; P.status = d_status;
+    P.ld = cfg->ld; P.K = cfg->K; P.m = m; P.q = cfg->q; P.mode = cfg->mode;
+    P.eta = cfg->eta; P.zeta = cfg->zeta;
+    const int qp1 = cfg->q + 1;
+    P.qp1 = (float)qp1; P.inv_qp1 = 1.0f / (float)qp1; P.inv_exact = (qp1 & (qp1 - 1)) == 0;
+    P.T = L.T; P.BW = L.BW; P.stages = L.stages; P.ring = L.ring; P.ncons = L.ncons;
+    if (L.T > L.BW) { P.bw_shift = 8; P.bw_mask = 255; } else { P.bw_shift = 30; P.bw_mask = (1 << 30) - 1; }
+    P.stage_stride = L.stage_stride; P.nbr_off = L.nbr_off; P.desc_off = L.desc_off;
+    P.ring_off = L.ring_off; P.slot_stride = L.slot_stride;
+    const int grid = (int)(total < tmp.num_sms ? total : tmp.num_sms);
+    bool attr = false;
+    st = cfg->theta_dtype == GBMUF_F32 ? launch_sync<float>(&tmp, P, grid, cs, &attr)
+                                       : launch_sync<__nv_bfloat16>(&tmp, P, grid, cs, &attr);
+    if (st != GBMUF_OK) { g_create_error = tmp.err; return st; }
+  }
+  if (device_status_out) {
+    int32_t word = 0;
+    e = cudaMemcpyAsync(&word, d_status, sizeof(word), cudaMemcpyDeviceToHost, cs);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(cs);
+    if (e != cudaSuccess) return cuda_fail(nullptr, "read of the device status word", e);
+    *device_status_out = word;
+  }
+  return GBMUF_OK;
+}
+
 }  // extern "C"
