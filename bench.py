@@ -35,7 +35,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of the fused kernel per replica-parameter from an ncu capture (dram__bytes_read.sum
 # + dram__bytes_write.sum divided by the replica-parameters of the captured launch), valid only
 # for the kernel source it was taken from (sha256 of csrc/gbmuf.cu, first 12 hex digits).
-NCU_TRAFFIC = {"source_sha": None, "bytes_per_replica_param": None}
+NCU_TRAFFIC = {"source_sha": "471dcd42ea5c", "bytes_per_replica_param": 6.382952e9 / 268435536}
 
 
 def algorithmic_bytes_per_replica_param(dtype: int, mode: int = 0) -> int:
@@ -238,6 +238,41 @@ def run_gpu(args, w):
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
     total_sync_s = float(tt.item())
 
+    # ---- end to end: the same round through the host-buffer entry point (replicas in page-locked
+    # host memory; host->device and device->host copies of theta, omega and Delta inside the timed
+    # call), on a bounded column sample so that all ranks together pin at most ~26 GB of host RAM
+    e2e = None
+    if not args.no_e2e:
+        C = min(N, args.e2e_cols // world // 32 * 32)
+        sh = workloads.shard_columns(w.offsets, 0, C)
+        cld = workloads.padded_ld(C)
+        hth = torch.empty((K, cld), dtype=tdt, pin_memory=True)
+        hom = torch.empty((K, cld), dtype=torch.float32, pin_memory=True)
+        hde = torch.empty((K, cld), dtype=torch.float32, pin_memory=True)
+        hth[:, :C].copy_(theta[:, :C])
+        hom[:, :C].copy_(omega[:, :C])
+        hde[:, :C].copy_(delta[:, :C])
+        torch.cuda.synchronize()
+        kw = dict(K=K, N=C, ld=cld, p=w.p, q=w.q, eta=w.eta, zeta=w.zeta, seed=w.seed,
+                  theta_dtype=w.dtype, device=local, comp_base=rank * w.m, elem_base=rank * N)
+        binding.sync_round_host(hth, hom, hde, sh.offsets, rnd, **kw)          # warm-up
+        barrier()
+        t0 = time.perf_counter()
+        for i in range(args.e2e_steps):
+            binding.sync_round_host(hth, hom, hde, sh.offsets, rnd + 1 + i, **kw)
+        barrier()
+        t_e2e = time.perf_counter() - t0
+        tt = torch.tensor([t_e2e], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        esz = 4 if w.dtype == 0 else 2
+        e2e = {"value": world * K * C * args.e2e_steps / float(tt.item()), "unit": UNIT,
+               "h2d_bytes_per_step": K * C * (esz + 8), "d2h_bytes_per_step": K * C * (esz + 8),
+               "steps": args.e2e_steps, "ms_per_step": float(tt.item()) / args.e2e_steps * 1e3,
+               "sample": f"columns [0,{C}) of {w.name} per GPU, all K={K} replicas, "
+                         "page-locked host arrays, gbmuf_sync_round_host"}
+        del hth, hom, hde
+
     line = None
     if rank == 0:
         units = world * K * N * args.steps
@@ -268,7 +303,7 @@ def run_gpu(args, w):
                              "frac_of_nominal_8TBs": achieved / 8000.0,
                              "algorithmic_bytes_per_replica_param": bpe, "traffic": traffic,
                              "kernel": "sync_fused_kernel"},
-                "clocks": clocks, "gpu_launches": 3 * args.steps, "e2e": None}
+                "clocks": clocks, "gpu_launches": 3 * args.steps, "e2e": e2e}
         if not args.no_cpu_baseline and world == 1:
             times, units_cpu = time_oracle_rounds(w, args.ref_cols, 3)
             t = sum(times) / len(times)
@@ -295,6 +330,10 @@ def main():
     ap.add_argument("--ref-cols", type=int, default=1 << 23,
                     help="columns of the workload the CPU oracle is timed on")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--e2e-cols", type=int, default=1 << 27,
+                    help="columns (summed over ranks) of the end-to-end host-buffer sample")
+    ap.add_argument("--e2e-steps", type=int, default=3)
     args = ap.parse_args()
     from paper_1909_09010_b200 import workloads
     w = workloads.get(args.workload)

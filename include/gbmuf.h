@@ -147,6 +147,20 @@ gbmuf_status gbmuf_set_tuning(gbmuf_ctx* ctx, int32_t consumer_threads, int32_t 
 gbmuf_status gbmuf_get_launch_info(gbmuf_ctx* ctx, int64_t* tiles, int32_t* grid, int32_t* block,
                                    int32_t* smem_bytes, int32_t* tile_elems, int32_t* stages);
 
+/* One synchronisation round (as gbmuf_sync_round, same arithmetic and the same neighbour draws)
+ * over replicas that live in HOST memory: theta, omega, delta are host arrays [K][ld] (ld >= N, no
+ * alignment rule; page-locked memory lets the copies overlap, pageable memory works but
+ * serialises them).  Given the neighbour table every element of the round is independent, so the
+ * columns are cut into chunks of chunk_cols (a multiple of 32; 0 = 4,194,304) that rotate through
+ * three sets of device buffers: copy in, set-up + fused kernel, copy out, each set on its own
+ * stream.  Chunks in which no component takes part are not copied at all.  The call allocates
+ * its device buffers (3 * K * chunk_cols * (element size + 8) bytes), returns when the host
+ * arrays hold the result, and frees them.  comp_mask: host [m] or NULL (= all take part).
+ * Errors: INVALID_ARG, ALLOC, CUDA, TIMEOUT, UNSUPPORTED; text via gbmuf_last_error(NULL). */
+gbmuf_status gbmuf_sync_round_host(const gbmuf_config* cfg, void* theta_host, float* omega_host,
+                                   float* delta_host, int32_t m, const int64_t* offsets_host,
+                                   const uint8_t* comp_mask_host, uint64_t round, int64_t chunk_cols);
+
 /* (No counterpart in the paper: this entry point exists for the library's callers, not for the
  * method.)  One synchronisation round that allocates nothing, for callers that must not or cannot
  * allocate device memory at the point where they synchronise: a training process whose memory pool

@@ -23,7 +23,7 @@ MODE_BMUF, MODE_MA = 0, 1
 EXPORTS = ["gbmuf_create", "gbmuf_set_partition", "gbmuf_init", "gbmuf_local_perturb",
            "gbmuf_sync_round", "gbmuf_get_neighbors", "gbmuf_final_average", "gbmuf_device_status",
            "gbmuf_set_tuning", "gbmuf_get_launch_info", "gbmuf_last_error", "gbmuf_destroy",
-           "gbmuf_sync_round_noalloc"]
+           "gbmuf_sync_round_noalloc", "gbmuf_sync_round_host"]
 
 
 class Config(ctypes.Structure):
@@ -70,6 +70,7 @@ def lib() -> ctypes.CDLL:
                                         ctypes.POINTER(i32), ctypes.POINTER(i32)]
     L.gbmuf_sync_round_noalloc.argtypes = [ctypes.POINTER(Config), vp, vp, vp, i32, vp, vp, u64, vp,
                                            ctypes.POINTER(i32)]
+    L.gbmuf_sync_round_host.argtypes = [ctypes.POINTER(Config), vp, vp, vp, i32, vp, vp, u64, i64]
     L.gbmuf_last_error.argtypes = [vp]
     L.gbmuf_last_error.restype = ctypes.c_char_p
     L.gbmuf_destroy.argtypes = [vp]
@@ -115,6 +116,20 @@ def sync_round_noalloc(theta, omega, delta, offsets, rnd, *, K, N, ld, p, q, eta
     if st != GBMUF_OK:
         raise GbmufError(st, lib().gbmuf_last_error(None).decode())
     return word.value if want_status else None
+
+
+def sync_round_host(theta, omega, delta, offsets, rnd, *, K, N, ld, p, q, eta, zeta, seed=0,
+                    mode=MODE_BMUF, theta_dtype=F32, device=0, comp_base=0, elem_base=0,
+                    comp_mask=None, chunk_cols=0):
+    """``gbmuf_sync_round_host``: one round over HOST arrays [K][ld] (numpy arrays or CPU torch
+    tensors, ideally page-locked), streamed through the GPU in column chunks.  Synchronous."""
+    cfg = Config(K, N, ld, p, q, eta, zeta, mode, theta_dtype, seed, device, comp_base, elem_base)
+    off = np.ascontiguousarray(offsets, dtype=np.int64)
+    mask = None if comp_mask is None else np.ascontiguousarray(comp_mask, dtype=np.uint8)
+    st = lib().gbmuf_sync_round_host(ctypes.byref(cfg), _ptr(theta), _ptr(omega), _ptr(delta),
+                                     off.shape[0] - 1, _ptr(off), _ptr(mask), rnd, chunk_cols)
+    if st != GBMUF_OK:
+        raise GbmufError(st, lib().gbmuf_last_error(None).decode())
 
 
 class Gbmuf:

@@ -1335,4 +1335,188 @@ gbmuf_status gbmuf_sync_round_noalloc(const gbmuf_config* cfg, void* theta, floa
   return GBMUF_OK;
 }
 
+
+// -------------------------------------------------------------------------------------------------
+// gbmuf_sync_round_host: one round over replicas that live in HOST memory.
+// -------------------------------------------------------------------------------------------------
+namespace {
+
+struct HostSet {               // one of the buffer sets column chunks rotate through
+  gbmuf_ctx ctx;               // describes the device chunk buffers to the launch helpers
+  unsigned char* tables = nullptr;
+  cudaStream_t stream = nullptr;
+};
+
+void free_host_sets(HostSet* sets, int n) {
+  for (int i = 0; i < n; ++i) {
+    cudaFree(sets[i].ctx.theta); cudaFree(sets[i].ctx.omega); cudaFree(sets[i].ctx.delta);
+    cudaFree(sets[i].tables);
+    if (sets[i].stream) cudaStreamDestroy(sets[i].stream);
+  }
+}
+
+}  // namespace
+
+gbmuf_status gbmuf_sync_round_host(const gbmuf_config* cfg, void* theta, float* omega, float* delta,
+                                   int32_t m, const int64_t* offsets, const uint8_t* comp_mask,
+                                   uint64_t round, int64_t chunk_cols) {
+  if (!cfg) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "cfg must not be NULL");
+  if (cfg->K < 1 || cfg->K > 256 || cfg->N < 1 || cfg->ld < cfg->N || cfg->p < 0 || cfg->q < 0 ||
+      cfg->comp_base < 0 || (cfg->mode != GBMUF_MODE_BMUF && cfg->mode != GBMUF_MODE_MA) ||
+      (cfg->theta_dtype != GBMUF_F32 && cfg->theta_dtype != GBMUF_BF16) ||
+      !(cfg->eta == cfg->eta) || !(cfg->zeta == cfg->zeta) || cfg->device < 0)
+    return fail(nullptr, GBMUF_ERR_INVALID_ARG, "configuration out of range (see gbmuf_create)");
+  const int cand = host_candidates(cfg->K, cfg->p);
+  if (cfg->q > cand || cand > kMaxCand)
+    return fail(nullptr, GBMUF_ERR_INVALID_ARG, "q exceeds the ring neighbours min(2p, K-1), or more than 64 of them");
+  if (!theta || !omega || !delta) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "theta, omega and delta must not be NULL");
+  if (m < 1 || m > 65536 || !offsets) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "m must be in 1..65536 and offsets not NULL");
+  if (offsets[0] != 0 || offsets[m] != cfg->N)
+    return fail(nullptr, GBMUF_ERR_INVALID_ARG, "offsets[0] must be 0 and offsets[m] must be N");
+  for (int i = 0; i < m; ++i)
+    if (offsets[i + 1] <= offsets[i]) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "offsets must be strictly increasing");
+  if (chunk_cols < 0 || (chunk_cols > 0 && chunk_cols % 32 != 0) || chunk_cols > (1LL << 30))
+    return fail(nullptr, GBMUF_ERR_INVALID_ARG, "chunk_cols must be 0 or a multiple of 32 up to 2^30");
+  if (chunk_cols == 0) chunk_cols = 1 << 22;
+  const long long N = cfg->N;
+  if (chunk_cols > (N + 31) / 32 * 32) chunk_cols = (N + 31) / 32 * 32;
+  const long long nchunks = (N + chunk_cols - 1) / chunk_cols;
+  const int esz = cfg->theta_dtype == GBMUF_F32 ? 4 : 2;
+  const int K = cfg->K, q = cfg->q;
+
+  DeviceGuard guard(cfg->device);
+  if (!guard.ok) return fail(nullptr, GBMUF_ERR_CUDA, "cudaSetDevice failed");
+
+  constexpr int kSets = 3;
+  const int nsets = nchunks < kSets ? (int)nchunks : kSets;
+  HostSet sets[kSets];
+  for (int i = 0; i < kSets; ++i) { sets[i].ctx.theta = nullptr; sets[i].ctx.omega = nullptr; sets[i].ctx.delta = nullptr; }
+  // table block of one set: offsets int64 [m+2] | prefix int32 [m+2] | nbr int32 [K*(m+1)*q] | mask
+  const size_t t_off = 0, t_prefix = ((size_t)(m + 2) * 8 + 255) / 256 * 256;
+  const size_t t_nbr = t_prefix + ((size_t)(m + 2) * 4 + 255) / 256 * 256;
+  const size_t t_mask = t_nbr + ((size_t)K * (m + 1) * (q > 0 ? q : 1) * 4 + 255) / 256 * 256;
+  const size_t t_status = t_mask + ((size_t)(m + 1) + 255) / 256 * 256;
+  const size_t t_bytes = t_status + 256;
+  gbmuf_status st = GBMUF_OK;
+  cudaError_t e = cudaSuccess;
+  for (int i = 0; i < nsets && st == GBMUF_OK; ++i) {
+    gbmuf_ctx& c = sets[i].ctx;
+    c.cfg = *cfg; c.cfg.N = chunk_cols; c.cfg.ld = chunk_cols; c.m = m; c.cand = cand;
+    c.theta = nullptr; c.omega = nullptr; c.delta = nullptr;
+    int v = 0;
+    cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, cfg->device); c.num_sms = v;
+    cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerBlockOptin, cfg->device); c.max_smem = v;
+    cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerMultiprocessor, cfg->device); c.smem_per_sm = v;
+    e = cudaMalloc(&c.theta, (size_t)K * chunk_cols * esz);
+    if (e == cudaSuccess) e = cudaMalloc(&c.omega, (size_t)K * chunk_cols * 4);
+    if (e == cudaSuccess) e = cudaMalloc(&c.delta, (size_t)K * chunk_cols * 4);
+    if (e == cudaSuccess) e = cudaMalloc(&sets[i].tables, t_bytes);
+    if (e == cudaSuccess) e = cudaMemset(sets[i].tables + t_status, 0, 256);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&sets[i].stream, cudaStreamNonBlocking);
+    if (e != cudaSuccess) {
+      st = e == cudaErrorMemoryAllocation ? fail(nullptr, GBMUF_ERR_ALLOC, "device chunk buffers")
+                                          : cuda_fail(nullptr, "set-up of the chunk buffers", e);
+      break;
+    }
+    st = plan_launch(&c, c.tuning, &c.launch);
+    if (st == GBMUF_OK) st = build_tensor_maps(&c, c.launch);
+    if (st != GBMUF_OK) g_create_error = c.err;
+  }
+  if (st != GBMUF_OK) { free_host_sets(sets, nsets); return st; }
+
+  // per-chunk host tables must outlive the asynchronous uploads
+  std::vector<std::vector<int64_t>> chunk_off((size_t)nchunks);
+  std::vector<std::vector<uint8_t>> chunk_mask((size_t)nchunks);
+  int first = 0;   // first component that reaches into the current chunk
+  for (long long ci = 0; ci < nchunks && st == GBMUF_OK; ++ci) {
+    const long long c0 = ci * chunk_cols, c1 = c0 + chunk_cols < N ? c0 + chunk_cols : N;
+    while (offsets[first + 1] <= c0) ++first;
+    std::vector<int64_t>& lo = chunk_off[(size_t)ci];
+    std::vector<uint8_t>& mk = chunk_mask[(size_t)ci];
+    lo.push_back(0);
+    int i = first;
+    long long total = 0;
+    HostSet& hs = sets[ci % nsets];
+    const int T = hs.ctx.launch.T;
+    while (true) {
+      const long long b = offsets[i] > c0 ? offsets[i] - c0 : 0;
+      const long long en = offsets[i + 1] < c1 ? offsets[i + 1] - c0 : c1 - c0;
+      const uint8_t due = comp_mask ? (comp_mask[i] != 0) : 1;
+      mk.push_back(due);
+      lo.push_back(en);
+      if (due) total += (en - (b & ~(long long)(kAlign - 1)) + T - 1) / T;
+      if (offsets[i + 1] >= c1) break;
+      ++i;
+    }
+    if (total == 0) continue;                    // nothing in this chunk takes part: leave it alone
+    const int mc = (int)mk.size();
+    cudaStream_t cs = hs.stream;
+    const size_t w_th = (size_t)(c1 - c0) * esz, w_f = (size_t)(c1 - c0) * 4;
+    e = cudaMemcpy2DAsync(hs.ctx.theta, (size_t)chunk_cols * esz, (const char*)theta + (size_t)c0 * esz,
+                          (size_t)cfg->ld * esz, w_th, K, cudaMemcpyHostToDevice, cs);
+    if (e == cudaSuccess && cfg->mode == GBMUF_MODE_BMUF) {
+      e = cudaMemcpy2DAsync(hs.ctx.omega, (size_t)chunk_cols * 4, omega + c0, (size_t)cfg->ld * 4, w_f, K,
+                            cudaMemcpyHostToDevice, cs);
+      if (e == cudaSuccess)
+        e = cudaMemcpy2DAsync(hs.ctx.delta, (size_t)chunk_cols * 4, delta + c0, (size_t)cfg->ld * 4, w_f, K,
+                              cudaMemcpyHostToDevice, cs);
+    }
+    if (e == cudaSuccess)
+      e = cudaMemcpyAsync(hs.tables + t_off, lo.data(), (size_t)(mc + 1) * 8, cudaMemcpyHostToDevice, cs);
+    if (e == cudaSuccess)
+      e = cudaMemcpyAsync(hs.tables + t_mask, mk.data(), (size_t)mc, cudaMemcpyHostToDevice, cs);
+    if (e != cudaSuccess) { st = cuda_fail(nullptr, "host-to-device copy of a column chunk", e); break; }
+
+    SetupParams S;
+    S.K = K; S.m = mc; S.p = cfg->p; S.q = q; S.comp_base = cfg->comp_base + first; S.T = T;
+    S.use_mask = 1; S.plan = 1; S.seed = cfg->seed; S.round = round;
+    S.off = reinterpret_cast<const int64_t*>(hs.tables + t_off);
+    S.periods = nullptr;
+    S.mask = hs.tables + t_mask;
+    S.nbr = reinterpret_cast<int32_t*>(hs.tables + t_nbr);
+    S.tile_prefix = reinterpret_cast<int32_t*>(hs.tables + t_prefix);
+    round_setup_kernel<<<(int)(((long long)K * mc + 255) / 256), 256, 0, cs>>>(S);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) { st = cuda_fail(nullptr, "launch of the round set-up kernel", e); break; }
+    const Launch& L = hs.ctx.launch;
+    SyncParams P;
+    P.theta = hs.ctx.theta; P.omega = hs.ctx.omega; P.delta = hs.ctx.delta;
+    P.off = S.off; P.tile_prefix = S.tile_prefix; P.nbr = S.nbr;
+    P.status = reinterpret_cast<int32_t*>(hs.tables + t_status);
+    P.ld = chunk_cols; P.K = K; P.m = mc; P.q = q; P.mode = cfg->mode; P.eta = cfg->eta; P.zeta = cfg->zeta;
+    const int qp1 = q + 1;
+    P.qp1 = (float)qp1; P.inv_qp1 = 1.0f / (float)qp1; P.inv_exact = (qp1 & (qp1 - 1)) == 0;
+    P.T = L.T; P.BW = L.BW; P.stages = L.stages; P.ring = L.ring; P.ncons = L.ncons;
+    if (L.T > L.BW) { P.bw_shift = 8; P.bw_mask = 255; } else { P.bw_shift = 30; P.bw_mask = (1 << 30) - 1; }
+    P.stage_stride = L.stage_stride; P.nbr_off = L.nbr_off; P.desc_off = L.desc_off;
+    P.ring_off = L.ring_off; P.slot_stride = L.slot_stride;
+    const int grid = (int)(total < hs.ctx.num_sms ? total : hs.ctx.num_sms);
+    st = esz == 4 ? launch_sync<float>(&hs.ctx, P, grid, cs, &hs.ctx.attr_set[0])
+                  : launch_sync<__nv_bfloat16>(&hs.ctx, P, grid, cs, &hs.ctx.attr_set[1]);
+    if (st != GBMUF_OK) { g_create_error = hs.ctx.err; break; }
+    e = cudaMemcpy2DAsync((char*)theta + (size_t)c0 * esz, (size_t)cfg->ld * esz, hs.ctx.theta,
+                          (size_t)chunk_cols * esz, w_th, K, cudaMemcpyDeviceToHost, cs);
+    if (e == cudaSuccess && cfg->mode == GBMUF_MODE_BMUF) {
+      e = cudaMemcpy2DAsync(omega + c0, (size_t)cfg->ld * 4, hs.ctx.omega, (size_t)chunk_cols * 4, w_f, K,
+                            cudaMemcpyDeviceToHost, cs);
+      if (e == cudaSuccess)
+        e = cudaMemcpy2DAsync(delta + c0, (size_t)cfg->ld * 4, hs.ctx.delta, (size_t)chunk_cols * 4, w_f, K,
+                              cudaMemcpyDeviceToHost, cs);
+    }
+    if (e != cudaSuccess) { st = cuda_fail(nullptr, "device-to-host copy of a column chunk", e); break; }
+  }
+  int32_t worst = 0;
+  for (int i = 0; i < nsets; ++i) {
+    e = cudaStreamSynchronize(sets[i].stream);
+    int32_t word = 0;
+    if (e == cudaSuccess) e = cudaMemcpy(&word, sets[i].tables + t_status, 4, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess && st == GBMUF_OK) st = cuda_fail(nullptr, "waiting for the column chunks", e);
+    if (word != 0) worst = word;
+  }
+  free_host_sets(sets, nsets);
+  if (st == GBMUF_OK && worst != 0)
+    st = fail(nullptr, GBMUF_ERR_TIMEOUT, "a bounded device-side wait expired; the host arrays are unspecified");
+  return st;
+}
+
 }  // extern "C"
