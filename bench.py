@@ -336,7 +336,12 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     args = ap.parse_args()
     from paper_1909_09010_b200 import workloads
-    w = workloads.get(args.workload)
+    name, _, opts = args.workload.partition(":")           # e.g. sweep:C=64,q=4,eta=0.5
+    over = {}
+    for kv in filter(None, opts.split(",")):
+        k, v = kv.split("=")
+        over[k] = float(v) if k == "eta" else int(v)
+    w = workloads.get(name, **over)
     if args.impl == "reference":
         run_reference(args, w)
     else:

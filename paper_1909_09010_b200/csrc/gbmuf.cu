@@ -419,9 +419,9 @@ sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_th
       }
       __syncwarp();
       const uint32_t full = bars + kBarThetaFull + 8 * s;
+      const uint32_t sbase = smem_u32(st);
       if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)P.K * (uint32_t)P.T * (uint32_t)sizeof(TH));
       __syncwarp();
-      const uint32_t sbase = smem_u32(st);
       const uint32_t box_bytes = (uint32_t)P.K * (uint32_t)P.BW * (uint32_t)sizeof(TH);
       for (int b = lane; b < P.T / P.BW; b += 32)
         tma_load_box(sbase + (uint32_t)b * box_bytes, &map_theta, (int)e0 + b * P.BW, 0, full);
@@ -622,15 +622,36 @@ __global__ void __launch_bounds__(256) perturb_kernel(TH* theta, int K, long lon
 template <typename TH>
 __global__ void __launch_bounds__(256) init_kernel(const TH* theta0, TH* theta, float* omega,
                                                    float* delta, int K, long long N, long long ld) {
-  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < N;
-       e += (long long)gridDim.x * blockDim.x) {
-    const TH v = theta0[e];
-    const float f = ThetaTraits<TH>::widen(v);
-    for (int k = 0; k < K; ++k) {
-      const long long at = (long long)k * ld + e;
-      theta[at] = v;
-      omega[at] = f;
-      delta[at] = 0.0f;
+  constexpr int VEC = ThetaTraits<TH>::VEC;
+  const long long nvec = (N + VEC - 1) / VEC;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec;
+       i += (long long)gridDim.x * blockDim.x) {
+    const long long e = i * VEC;
+    if (e + VEC <= N) {
+      const uint4 raw = *reinterpret_cast<const uint4*>(theta0 + e);   // 16 bytes of theta_0
+      float f[VEC];
+      ThetaTraits<TH>::lds(theta0 + e, f);
+      const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int k = 0; k < K; ++k) {
+        const long long at = (long long)k * ld + e;
+        __stcs(reinterpret_cast<uint4*>(theta + at), raw);
+#pragma unroll
+        for (int h = 0; h < VEC / 4; ++h) {
+          __stcs(reinterpret_cast<float4*>(omega + at) + h,
+                 make_float4(f[4 * h], f[4 * h + 1], f[4 * h + 2], f[4 * h + 3]));
+          __stcs(reinterpret_cast<float4*>(delta + at) + h, zero);
+        }
+      }
+    } else {
+      for (long long x = e; x < N; ++x) {
+        const TH v = theta0[x];
+        for (int k = 0; k < K; ++k) {
+          const long long at = (long long)k * ld + x;
+          theta[at] = v;
+          omega[at] = ThetaTraits<TH>::widen(v);
+          delta[at] = 0.0f;
+        }
+      }
     }
   }
 }
@@ -638,12 +659,31 @@ __global__ void __launch_bounds__(256) init_kernel(const TH* theta0, TH* theta, 
 template <typename TH>
 __global__ void __launch_bounds__(256) final_average_kernel(const TH* theta, TH* out, int K,
                                                             long long N, long long ld) {
+  constexpr int VEC = ThetaTraits<TH>::VEC;
   const float fk = (float)K;
-  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < N;
-       e += (long long)gridDim.x * blockDim.x) {
-    float s = ThetaTraits<TH>::widen(theta[e]);
-    for (int k = 1; k < K; ++k) s = __fadd_rn(s, ThetaTraits<TH>::widen(theta[(long long)k * ld + e]));
-    out[e] = ThetaTraits<TH>::narrow(__fdiv_rn(s, fk));
+  const long long nvec = (N + VEC - 1) / VEC;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec;
+       i += (long long)gridDim.x * blockDim.x) {
+    const long long e = i * VEC;
+    if (e + VEC <= N) {
+      float s[VEC], t[VEC];
+      ThetaTraits<TH>::lds(theta + e, s);
+      for (int k = 1; k < K; ++k) {                  // k = 0, 1, ..., K-1 in that order
+        ThetaTraits<TH>::lds(theta + (long long)k * ld + e, t);
+#pragma unroll
+        for (int x = 0; x < VEC; ++x) s[x] = __fadd_rn(s[x], t[x]);
+      }
+#pragma unroll
+      for (int x = 0; x < VEC; ++x) s[x] = __fdiv_rn(s[x], fk);
+      ThetaTraits<TH>::stg(out + e, s);
+    } else {
+      for (long long x = e; x < N; ++x) {
+        float s = ThetaTraits<TH>::widen(theta[x]);
+        for (int k = 1; k < K; ++k)
+          s = __fadd_rn(s, ThetaTraits<TH>::widen(theta[(long long)k * ld + x]));
+        out[x] = ThetaTraits<TH>::narrow(__fdiv_rn(s, fk));
+      }
+    }
   }
 }
 
@@ -851,6 +891,23 @@ gbmuf_status launch_sync(gbmuf_ctx* ctx, const SyncParams& P, int grid, cudaStre
   return GBMUF_OK;
 }
 
+// Everything the fused kernel needs to know about one launch.
+void fill_sync_params(const gbmuf_config& cfg, const Launch& L, void* theta, float* omega,
+                      float* delta, long long ld, int m, const int64_t* off, const int32_t* prefix,
+                      const int32_t* nbr, int32_t* status, SyncParams* P) {
+  P->theta = theta; P->omega = omega; P->delta = delta;
+  P->off = off; P->tile_prefix = prefix; P->nbr = nbr; P->status = status;
+  P->ld = ld; P->K = cfg.K; P->m = m; P->q = cfg.q; P->mode = cfg.mode;
+  P->eta = cfg.eta; P->zeta = cfg.zeta;
+  const int qp1 = cfg.q + 1;
+  P->qp1 = (float)qp1; P->inv_qp1 = 1.0f / (float)qp1; P->inv_exact = (qp1 & (qp1 - 1)) == 0;
+  P->T = L.T; P->BW = L.BW; P->stages = L.stages; P->ring = L.ring; P->ncons = L.ncons;
+  if (L.T > L.BW) { P->bw_shift = 8; P->bw_mask = 255; }          // several boxes of 256 columns
+  else { P->bw_shift = 30; P->bw_mask = (1 << 30) - 1; }          // one box
+  P->stage_stride = L.stage_stride; P->nbr_off = L.nbr_off; P->desc_off = L.desc_off;
+  P->ring_off = L.ring_off; P->slot_stride = L.slot_stride;
+}
+
 void fill_setup(const gbmuf_ctx* ctx, uint64_t round, bool use_mask, bool plan, int32_t* nbr,
                 SetupParams* S) {
   S->K = ctx->cfg.K; S->m = ctx->m; S->p = ctx->cfg.p; S->q = ctx->cfg.q;
@@ -1029,7 +1086,7 @@ gbmuf_status gbmuf_init(gbmuf_ctx* ctx, const void* theta0, void* stream) {
     return fail(ctx, GBMUF_ERR_INVALID_ARG, "theta0 must be a 16-byte aligned device pointer");
   DeviceGuard guard(ctx->cfg.device);
   if (!guard.ok) return fail(ctx, GBMUF_ERR_CUDA, "cudaSetDevice failed");
-  const int grid = elementwise_grid(ctx, ctx->cfg.N);
+  const int grid = elementwise_grid(ctx, (ctx->cfg.N + 3) / 4);
   cudaStream_t st = (cudaStream_t)stream;
   if (ctx->cfg.theta_dtype == GBMUF_F32)
     init_kernel<float><<<grid, 256, 0, st>>>((const float*)theta0, (float*)ctx->theta, ctx->omega,
@@ -1095,17 +1152,8 @@ gbmuf_status gbmuf_sync_round(gbmuf_ctx* ctx, uint64_t round, const uint8_t* com
   if (e != cudaSuccess) return cuda_fail(ctx, "launch of the round set-up kernel", e);
 
   SyncParams P;
-  P.theta = ctx->theta; P.omega = ctx->omega; P.delta = ctx->delta;
-  P.off = ctx->d_off; P.tile_prefix = ctx->d_prefix; P.nbr = ctx->d_nbr; P.status = ctx->d_status;
-  P.ld = ctx->cfg.ld; P.K = ctx->cfg.K; P.m = ctx->m; P.q = ctx->cfg.q; P.mode = ctx->cfg.mode;
-  P.eta = ctx->cfg.eta; P.zeta = ctx->cfg.zeta;
-  const int qp1 = ctx->cfg.q + 1;
-  P.qp1 = (float)qp1; P.inv_qp1 = 1.0f / (float)qp1; P.inv_exact = (qp1 & (qp1 - 1)) == 0;
-  P.T = L.T; P.BW = L.BW; P.stages = L.stages; P.ring = L.ring; P.ncons = L.ncons;
-  if (L.T > L.BW) { P.bw_shift = 8; P.bw_mask = 255; }      // several boxes of 256 columns
-  else { P.bw_shift = 30; P.bw_mask = (1 << 30) - 1; }       // one box
-  P.stage_stride = L.stage_stride; P.nbr_off = L.nbr_off; P.desc_off = L.desc_off;
-  P.ring_off = L.ring_off; P.slot_stride = L.slot_stride;
+  fill_sync_params(ctx->cfg, L, ctx->theta, ctx->omega, ctx->delta, ctx->cfg.ld, ctx->m, ctx->d_off,
+                   ctx->d_prefix, ctx->d_nbr, ctx->d_status, &P);
   const long long cap = (long long)ctx->num_sms;              // one persistent CTA per SM
   const int grid = (int)(total < cap ? total : cap);
   if (ctx->cfg.theta_dtype == GBMUF_F32) return launch_sync<float>(ctx, P, grid, st, &ctx->attr_set[0]);
@@ -1144,7 +1192,7 @@ gbmuf_status gbmuf_final_average(gbmuf_ctx* ctx, void* out, void* stream) {
     return fail(ctx, GBMUF_ERR_INVALID_ARG, "out must be a 16-byte aligned device pointer");
   DeviceGuard guard(ctx->cfg.device);
   if (!guard.ok) return fail(ctx, GBMUF_ERR_CUDA, "cudaSetDevice failed");
-  const int grid = elementwise_grid(ctx, ctx->cfg.N);
+  const int grid = elementwise_grid(ctx, (ctx->cfg.N + 3) / 4);
   cudaStream_t st = (cudaStream_t)stream;
   if (ctx->cfg.theta_dtype == GBMUF_F32)
     final_average_kernel<float><<<grid, 256, 0, st>>>((const float*)ctx->theta, (float*)out,
@@ -1309,16 +1357,7 @@ gbmuf_status gbmuf_sync_round_noalloc(const gbmuf_config* cfg, void* theta, floa
     if (e != cudaSuccess) return cuda_fail(nullptr, "launch of the round set-up kernel", e);
 
     SyncParams P;
-    P.theta = theta; P.omega = omega; P.delta = delta;
-    P.off = S.off; P.tile_prefix = S.tile_prefix; P.nbr = S.nbr; P.status = d_status;
-    P.ld = cfg->ld; P.K = cfg->K; P.m = m; P.q = cfg->q; P.mode = cfg->mode;
-    P.eta = cfg->eta; P.zeta = cfg->zeta;
-    const int qp1 = cfg->q + 1;
-    P.qp1 = (float)qp1; P.inv_qp1 = 1.0f / (float)qp1; P.inv_exact = (qp1 & (qp1 - 1)) == 0;
-    P.T = L.T; P.BW = L.BW; P.stages = L.stages; P.ring = L.ring; P.ncons = L.ncons;
-    if (L.T > L.BW) { P.bw_shift = 8; P.bw_mask = 255; } else { P.bw_shift = 30; P.bw_mask = (1 << 30) - 1; }
-    P.stage_stride = L.stage_stride; P.nbr_off = L.nbr_off; P.desc_off = L.desc_off;
-    P.ring_off = L.ring_off; P.slot_stride = L.slot_stride;
+    fill_sync_params(*cfg, L, theta, omega, delta, cfg->ld, m, S.off, S.tile_prefix, S.nbr, d_status, &P);
     const int grid = (int)(total < tmp.num_sms ? total : tmp.num_sms);
     bool attr = false;
     st = cfg->theta_dtype == GBMUF_F32 ? launch_sync<float>(&tmp, P, grid, cs, &attr)
@@ -1480,16 +1519,8 @@ gbmuf_status gbmuf_sync_round_host(const gbmuf_config* cfg, void* theta, float* 
     if (e != cudaSuccess) { st = cuda_fail(nullptr, "launch of the round set-up kernel", e); break; }
     const Launch& L = hs.ctx.launch;
     SyncParams P;
-    P.theta = hs.ctx.theta; P.omega = hs.ctx.omega; P.delta = hs.ctx.delta;
-    P.off = S.off; P.tile_prefix = S.tile_prefix; P.nbr = S.nbr;
-    P.status = reinterpret_cast<int32_t*>(hs.tables + t_status);
-    P.ld = chunk_cols; P.K = K; P.m = mc; P.q = q; P.mode = cfg->mode; P.eta = cfg->eta; P.zeta = cfg->zeta;
-    const int qp1 = q + 1;
-    P.qp1 = (float)qp1; P.inv_qp1 = 1.0f / (float)qp1; P.inv_exact = (qp1 & (qp1 - 1)) == 0;
-    P.T = L.T; P.BW = L.BW; P.stages = L.stages; P.ring = L.ring; P.ncons = L.ncons;
-    if (L.T > L.BW) { P.bw_shift = 8; P.bw_mask = 255; } else { P.bw_shift = 30; P.bw_mask = (1 << 30) - 1; }
-    P.stage_stride = L.stage_stride; P.nbr_off = L.nbr_off; P.desc_off = L.desc_off;
-    P.ring_off = L.ring_off; P.slot_stride = L.slot_stride;
+    fill_sync_params(*cfg, L, hs.ctx.theta, hs.ctx.omega, hs.ctx.delta, chunk_cols, mc, S.off,
+                     S.tile_prefix, S.nbr, reinterpret_cast<int32_t*>(hs.tables + t_status), &P);
     const int grid = (int)(total < hs.ctx.num_sms ? total : hs.ctx.num_sms);
     st = esz == 4 ? launch_sync<float>(&hs.ctx, P, grid, cs, &hs.ctx.attr_set[0])
                   : launch_sync<__nv_bfloat16>(&hs.ctx, P, grid, cs, &hs.ctx.attr_set[1]);

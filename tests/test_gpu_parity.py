@@ -245,3 +245,101 @@ def test_padding_columns_are_never_written():
     assert bool((th[:, N:] == 7.0).all()) and bool((om[:, N:] == 8.0).all())
     assert bool((de[:, N:] == 9.0).all())
     g.destroy()
+
+
+# ------------------------------------------------------------------------------------------------
+# resume, graph replay, random shapes
+# ------------------------------------------------------------------------------------------------
+def test_resume_from_saved_state_is_bit_identical():
+    """The state of a run is (theta, omega, Delta, round number, seed, partition): the draws and the
+    noise are counter-based, so R rounds + save / restore + R rounds equals 2R rounds."""
+    w = workloads.get("tiny")
+    dev = torch.device("cuda:0")
+    kw = dict(K=w.K, N=w.N, ld=w.ld, p=w.p, q=w.q, eta=w.eta, zeta=w.zeta, seed=w.seed)
+
+    def fresh():
+        th = torch.zeros((w.K, w.ld), device=dev)
+        return th, torch.zeros_like(th), torch.zeros_like(th)
+
+    def advance(g, first, count):
+        for r in range(first, first + count):
+            g.local_perturb(2 * r, 0.1, 0.05, 2)
+            g.sync_round(r)
+
+    a = fresh()
+    ga = binding.Gbmuf(*a, **kw)
+    ga.set_partition(w.offsets)
+    ga.init(torch.from_numpy(workloads.theta0_numpy(w)).to(dev))
+    advance(ga, 1, 3)
+    torch.cuda.synchronize()
+    saved = [t.cpu().clone() for t in a]                 # "checkpoint"
+    advance(ga, 4, 3)
+    b = tuple(t.to(dev) for t in saved)                  # "restore" into other buffers, new context
+    gb = binding.Gbmuf(*b, **kw)
+    gb.set_partition(w.offsets)
+    advance(gb, 4, 3)
+    torch.cuda.synchronize()
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)
+    ga.destroy()
+    gb.destroy()
+
+
+def test_rounds_replayed_from_a_cuda_graph():
+    """Rounds without a host mask only launch kernels, so a sequence of them can be captured once
+    and replayed (the launch-bound tiny workload is where that pays)."""
+    w = workloads.get("tiny")
+    pr = Pair(case_of(w), workloads.theta0_numpy(w))
+    try:
+        pr.add_drift(workloads.drift_numpy(w))
+        pr.sync(1)                                      # first call outside capture
+        pr.compare("before capture")
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            graph.capture_begin()
+            for r in (2, 3, 4):
+                pr.g.local_perturb(r, 0.1, 0.02, 1, stream=side)
+                pr.g.sync_round(r, stream=side)
+            graph.capture_end()
+        torch.cuda.current_stream().wait_stream(side)
+        graph.replay()
+        torch.cuda.synchronize()
+        for r in (2, 3, 4):                             # the oracle replays the same calls once
+            for sh, st in zip(pr.shards, pr.states):
+                oracle.local_perturb(st, w.seed, r, 0.1, 0.02, 1, elem_base=sh.col0)
+                nbr = oracle.sample_neighbors(w.seed, r, w.K, sh.m, w.p, w.q, comp_base=sh.comp_base)
+                oracle.sync_round(st, sh.offsets, nbr, w.eta, w.zeta)
+        pr.compare("after graph replay")
+    finally:
+        pr.close()
+
+
+def test_random_shapes_property():
+    """Random K, p, q, component edges (unaligned, tiny and large), eta, zeta, dtype, mode."""
+    from hypothesis import given, settings, strategies as st_, HealthCheck
+
+    @settings(max_examples=25, deadline=None, derandomize=True,
+              suppress_health_check=list(HealthCheck))
+    @given(st_.data())
+    def inner(data):
+        K = data.draw(st_.integers(1, 24))
+        p = data.draw(st_.integers(0, 6))
+        c = min(2 * p, K - 1)
+        q = data.draw(st_.integers(0, c))
+        m = data.draw(st_.integers(1, 6))
+        N = data.draw(st_.integers(m, 30_000))
+        cuts = sorted(data.draw(st_.sets(st_.integers(1, N - 1), min_size=m - 1, max_size=m - 1))) if m > 1 else []
+        offsets = tuple([0] + cuts + [N])
+        eta = data.draw(st_.sampled_from([0.0, 0.5, 0.875, 0.9, 0.99]))
+        zeta = data.draw(st_.sampled_from([0.5, 1.0, 1.25]))
+        dtype = data.draw(st_.integers(0, 1))
+        mode = data.draw(st_.sampled_from([0, 0, 0, 1]))
+        tile = data.draw(st_.sampled_from([0, 64, 256, 512]))
+        case = Case(K=K, offsets=offsets, p=p, q=q, eta=eta, zeta=zeta, dtype=dtype,
+                    seed=data.draw(st_.integers(0, 2 ** 63)), mode=mode)
+        tuning = dict(tile_elems=tile, consumer_threads=data.draw(st_.sampled_from([64, 256]))) if tile else None
+        run(case, random_theta0(N, seed=K + N, dtype=dtype), rounds=2, sigma=5e-2, tuning=tuning)
+
+    inner()
