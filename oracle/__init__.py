@@ -60,6 +60,8 @@ def _bind(path: str) -> ctypes.CDLL:
     L.gbo_init.restype = i32
     L.gbo_local_perturb.argtypes = [i32, i64, i64, i32, vp, u64, u64, f32, f32, i32, i64]
     L.gbo_local_perturb.restype = i32
+    L.gbo_local_adagrad.argtypes = [i32, i64, i64, i32, vp, vp, vp, f32, f32, f32, i32, vp]
+    L.gbo_local_adagrad.restype = i32
     L.gbo_final_average.argtypes = [i32, i64, i64, i32, vp, vp]
     L.gbo_final_average.restype = i32
     return L
@@ -187,6 +189,18 @@ def local_perturb(st: State, seed: int, step: int, lr: float, sigma: float, nste
                   elem_base: int = 0) -> None:
     rc = lib().gbo_local_perturb(st.K, st.N, st.ld, st.dtype, _ptr(st.theta), seed, step, lr, sigma,
                                  nsteps, elem_base)
+    if rc != 0:
+        raise ValueError("bad arguments")
+
+
+def local_adagrad(st: State, grad: np.ndarray, accum: np.ndarray, lr: float, eps: float = 0.0,
+                  clip_norm: float = 0.0, ranges=()) -> None:
+    """Adagrad local step with group gradient-norm clipping, in place on st.theta and accum."""
+    grad = np.ascontiguousarray(grad, dtype=np.float32)
+    assert grad.shape == (st.K, st.ld) and accum.shape == (st.K, st.ld) and accum.dtype == np.float32
+    rg = np.ascontiguousarray(np.asarray(ranges, dtype=np.int64).reshape(-1, 2))
+    rc = lib().gbo_local_adagrad(st.K, st.N, st.ld, st.dtype, _ptr(st.theta), _ptr(grad), _ptr(accum),
+                                 lr, eps, clip_norm, rg.shape[0], _ptr(rg) if rg.size else None)
     if rc != 0:
         raise ValueError("bad arguments")
 

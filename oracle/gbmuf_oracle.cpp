@@ -19,6 +19,7 @@
 // the geometric-series closed form of the block-momentum filter, fixed points, worker-order
 // independence, moments of the perturbation noise.  No function here is "parity unpinned".
 
+#include <cmath>
 #include <cstdint>
 #include <cstdlib>
 #include <cstring>
@@ -266,6 +267,49 @@ int gbo_local_perturb(int K, int64_t N, int64_t ld, int dtype, void* theta, uint
         v = v - upd;
         v = store_theta(theta, dtype, at, v);
       }
+    }
+  }
+  return 0;
+}
+
+// The local step with the optimiser of the paper's experiments (Section 3.2) in place of the
+// plain SGD line of Algorithm 1: Adagrad, with the gradient norm of a group of parameters (there:
+// the LSTM weights) clipped to clip_norm.  Per worker k:
+//   norm_k = sqrt(sum of g^2 over the elements inside the clip ranges)       (summed in double)
+//   g'     = g * (clip_norm / max(norm_k, clip_norm)) inside the ranges, g elsewhere
+//   a     <- a + g' * g'
+//   theta <- store(theta - (lr * g') / (sqrt(a) + eps))
+// grad and accum are fp32 [K][ld]; ranges is nranges pairs [begin, end) of element indices;
+// clip_norm <= 0 switches clipping off.
+int gbo_local_adagrad(int K, int64_t N, int64_t ld, int dtype, void* theta, const float* grad,
+                      float* accum, float lr, float eps, float clip_norm, int nranges,
+                      const int64_t* ranges) {
+  if (K < 1 || N < 0 || ld < N || nranges < 0) return -1;
+  for (int k = 0; k < K; ++k) {
+    float scale = 1.0f;
+    if (clip_norm > 0.0f && nranges > 0) {
+      double ss = 0.0;
+      for (int r = 0; r < nranges; ++r)
+        for (int64_t e = ranges[2 * r]; e < ranges[2 * r + 1]; ++e) {
+          const double g = (double)grad[(int64_t)k * ld + e];
+          ss += g * g;
+        }
+      const float norm = (float)std::sqrt(ss);
+      scale = clip_norm / (norm > clip_norm ? norm : clip_norm);
+    }
+    for (int64_t e = 0; e < N; ++e) {
+      const int64_t at = (int64_t)k * ld + e;
+      bool inside = false;
+      for (int r = 0; r < nranges; ++r) inside = inside || (e >= ranges[2 * r] && e < ranges[2 * r + 1]);
+      float g = grad[at];
+      if (inside && clip_norm > 0.0f) g = g * scale;
+      const float gg = g * g;
+      const float a = accum[at] + gg;
+      accum[at] = a;
+      const float denom = std::sqrt(a) + eps;
+      const float num = lr * g;
+      const float upd = num / denom;
+      store_theta(theta, dtype, at, load_theta(theta, dtype, at) - upd);
     }
   }
   return 0;

@@ -10,7 +10,7 @@ import pytest
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 PINS = ["tests/test_oracle_philox.py", "tests/test_oracle_sampler.py",
-        "tests/test_oracle_perturb.py", "tests/test_oracle_sync.py"]
+        "tests/test_oracle_perturb.py", "tests/test_oracle_adagrad.py", "tests/test_oracle_sync.py"]
 
 # (name, text in oracle/gbmuf_oracle.cpp, replacement)
 MUTANTS = [
@@ -59,6 +59,19 @@ MUTANTS = [
      "(uint32_t)(pair >> 32), 0u, (uint32_t)(step + s)"),
     ("perturb_local_index", "const uint64_t ge = (uint64_t)(elem_base + e);",
      "const uint64_t ge = (uint64_t)(e);"),
+    ("adagrad_accumulates_unclipped", "const float gg = g * g;", "const float gg = grad[at] * grad[at];"),
+    ("adagrad_no_sqrt", "const float denom = std::sqrt(a) + eps;", "const float denom = a + eps;"),
+    ("adagrad_sign", "load_theta(theta, dtype, at) - upd);", "load_theta(theta, dtype, at) + upd);"),
+    ("adagrad_lr_dropped", "const float num = lr * g;", "const float num = g;"),
+    ("adagrad_clip_inverted", "scale = clip_norm / (norm > clip_norm ? norm : clip_norm);",
+     "scale = (norm > clip_norm ? norm : clip_norm) / clip_norm;"),
+    ("adagrad_clips_always", "scale = clip_norm / (norm > clip_norm ? norm : clip_norm);",
+     "scale = clip_norm / norm;"),
+    ("adagrad_norm_over_everything", "for (int64_t e = ranges[2 * r]; e < ranges[2 * r + 1]; ++e) {",
+     "for (int64_t e = 0; e < N; ++e) {"),
+    ("adagrad_scales_outside_ranges", "if (inside && clip_norm > 0.0f) g = g * scale;",
+     "if (clip_norm > 0.0f) g = g * scale;"),
+    ("adagrad_accumulator_not_stored", "accum[at] = a;", ""),
     ("final_average_divides_by_k_minus_1", "s / (float)K", "s / (float)(K > 1 ? K - 1 : 1)"),
 ]
 
