@@ -103,6 +103,21 @@ gbmuf_status gbmuf_init(gbmuf_ctx* ctx, const void* theta0_device, void* stream)
 gbmuf_status gbmuf_local_perturb(gbmuf_ctx* ctx, uint64_t step, float lr, float sigma,
                                  int32_t nsteps, void* stream);
 
+/* The local step with the optimiser of the paper's experiments (Section 3.2: Adagrad; the norm of
+ * the LSTM gradients clipped to 10.0) in place of the plain SGD line of Algorithm 1, on gradients
+ * the caller supplies.  grad: device fp32 [K][ld] (read only); accum: device fp32 [K][ld], the
+ * Adagrad accumulator, caller-owned and caller-initialised (the usual start is 0.1), updated in
+ * place; both 128-byte aligned.  Per worker k: norm_k = sqrt(sum of g^2 over the components whose
+ * clip_mask byte is non-zero) (double accumulation, fixed order); inside those components
+ * g' = g * (clip_norm / max(norm_k, clip_norm)), elsewhere g' = g; a <- a + g'g';
+ * theta <- store(theta - (lr * g') / (sqrt(a) + eps)).  clip_mask: host, m bytes, or NULL (no
+ * clipping; clip_norm <= 0 also switches it off); at most 16 separate runs of adjacent masked
+ * components.  lr is the caller's alpha_t (the paper decays 0.1 by 0.9 per epoch).
+ * Errors: INVALID_ARG, BAD_STATE (mask without set_partition), UNSUPPORTED, ALLOC, CUDA. */
+gbmuf_status gbmuf_local_adagrad(gbmuf_ctx* ctx, const float* grad_device, float* accum_device,
+                                 float lr, float eps, float clip_norm,
+                                 const uint8_t* clip_mask_host, void* stream);
+
 /* One synchronisation round `round` (the t of Algorithm 1).  Components taking part:
  * comp_mask != NULL: host, m bytes, component i takes part iff comp_mask[i] != 0;
  * comp_mask == NULL: component i takes part iff round % periods[i] == 0.

@@ -23,7 +23,7 @@ MODE_BMUF, MODE_MA = 0, 1
 EXPORTS = ["gbmuf_create", "gbmuf_set_partition", "gbmuf_init", "gbmuf_local_perturb",
            "gbmuf_sync_round", "gbmuf_get_neighbors", "gbmuf_final_average", "gbmuf_device_status",
            "gbmuf_set_tuning", "gbmuf_get_launch_info", "gbmuf_last_error", "gbmuf_destroy",
-           "gbmuf_sync_round_noalloc", "gbmuf_sync_round_host"]
+           "gbmuf_sync_round_noalloc", "gbmuf_sync_round_host", "gbmuf_local_adagrad"]
 
 
 class Config(ctypes.Structure):
@@ -60,6 +60,7 @@ def lib() -> ctypes.CDLL:
     L.gbmuf_set_partition.argtypes = [vp, i32, vp, vp]
     L.gbmuf_init.argtypes = [vp, vp, vp]
     L.gbmuf_local_perturb.argtypes = [vp, u64, f32, f32, i32, vp]
+    L.gbmuf_local_adagrad.argtypes = [vp, vp, vp, f32, f32, f32, vp, vp]
     L.gbmuf_sync_round.argtypes = [vp, u64, vp, vp]
     L.gbmuf_get_neighbors.argtypes = [vp, u64, vp]
     L.gbmuf_final_average.argtypes = [vp, vp, vp]
@@ -165,6 +166,15 @@ class Gbmuf:
 
     def local_perturb(self, step, lr, sigma, nsteps=1, stream=None):
         self._check(lib().gbmuf_local_perturb(self._h, step, lr, sigma, nsteps, _stream(stream)))
+
+    def local_adagrad(self, grad, accum, lr, eps=0.0, clip_norm=0.0, clip_mask=None, stream=None):
+        mask = None
+        if clip_mask is not None:
+            mask = np.ascontiguousarray(clip_mask, dtype=np.uint8)
+            if mask.shape[0] != self.m:
+                raise ValueError("clip_mask must have one entry per component")
+        self._check(lib().gbmuf_local_adagrad(self._h, _ptr(grad), _ptr(accum), lr, eps, clip_norm,
+                                              _ptr(mask), _stream(stream)))
 
     def sync_round(self, rnd, comp_mask=None, stream=None):
         mask = None

@@ -576,11 +576,10 @@ __global__ void __launch_bounds__(256) perturb_kernel(TH* theta, int K, long lon
                                                       long long elem_base) {
   constexpr int VEC = ThetaTraits<TH>::VEC;
   const long long nvec = (N + VEC - 1) / VEC;
-  const long long total = nvec * K;
-  for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
-       idx += (long long)gridDim.x * blockDim.x) {
-    const int k = (int)(idx / nvec);
-    const long long e = (idx % nvec) * VEC;
+  const int k = blockIdx.y;                 // one grid row per worker
+  for (long long iv = (long long)blockIdx.x * blockDim.x + threadIdx.x; iv < nvec;
+       iv += (long long)gridDim.x * blockDim.x) {
+    const long long e = iv * VEC;
     TH* row = theta + (long long)k * ld + e;
     const int n = N - e < VEC ? (int)(N - e) : VEC;
     float v[VEC];
@@ -612,6 +611,128 @@ __global__ void __launch_bounds__(256) perturb_kernel(TH* theta, int K, long lon
       ThetaTraits<TH>::stg(row, v);
     } else {
       for (int x = 0; x < n; ++x) row[x] = ThetaTraits<TH>::narrow(v[x]);
+    }
+  }
+}
+
+// =================================================================================================
+// Local step with the optimiser of the paper's experiments (Section 3.2): Adagrad with the
+// gradient norm of a group of components clipped.  Three kernels: per-(worker, block) partial sums
+// of squares in double over the clip ranges, a fixed-order final sum that turns them into one
+// scale factor per worker (deterministic: no atomics), and the element-wise update.
+// =================================================================================================
+constexpr int kMaxClipRanges = 16;
+constexpr int kNormBlocks = 128;    // partial sums per worker
+
+struct ClipRanges {
+  int n;
+  long long begin[kMaxClipRanges], end[kMaxClipRanges];
+};
+
+__global__ void __launch_bounds__(256) sumsq_partial_kernel(const float* grad, long long ld,
+                                                            ClipRanges R, double* partial) {
+  const int k = blockIdx.y;
+  const float* row = grad + (long long)k * ld;
+  // four independent partial sums per thread keep four loads in flight; the order of the
+  // additions is fixed by the launch shape, so the result is reproducible
+  double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (int r = 0; r < R.n; ++r) {
+    long long e = R.begin[r] + (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    for (; e + 3 * stride < R.end[r]; e += 4 * stride) {
+      const double g0 = (double)row[e], g1 = (double)row[e + stride];
+      const double g2 = (double)row[e + 2 * stride], g3 = (double)row[e + 3 * stride];
+      a0 += g0 * g0; a1 += g1 * g1; a2 += g2 * g2; a3 += g3 * g3;
+    }
+    for (; e < R.end[r]; e += stride) {
+      const double g = (double)row[e];
+      a0 += g * g;
+    }
+  }
+  double acc = (a0 + a1) + (a2 + a3);
+  __shared__ double warp_sum[8];
+  for (int d = 16; d > 0; d >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, d);
+  if ((threadIdx.x & 31) == 0) warp_sum[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double s = 0.0;
+    for (int w = 0; w < 8; ++w) s += warp_sum[w];
+    partial[(size_t)k * gridDim.x + blockIdx.x] = s;
+  }
+}
+
+__global__ void clip_scale_kernel(const double* partial, int K, int nblk, float clip_norm,
+                                  float* scale) {
+  const int k = blockIdx.x * blockDim.x + threadIdx.x;
+  if (k >= K) return;
+  double s = 0.0;
+  for (int b = 0; b < nblk; ++b) s += partial[(size_t)k * nblk + b];
+  const float norm = (float)sqrt(s);
+  scale[k] = __fdiv_rn(clip_norm, norm > clip_norm ? norm : clip_norm);
+}
+
+template <typename TH>
+__global__ void __launch_bounds__(256) adagrad_kernel(TH* theta, const float* grad, float* accum,
+                                                      int K, long long N, long long ld, float lr,
+                                                      float eps, const float* scale, ClipRanges R) {
+  constexpr int VEC = ThetaTraits<TH>::VEC;
+  const long long nvec = (N + VEC - 1) / VEC;
+  const int k = blockIdx.y;                 // one grid row per worker
+  for (long long iv = (long long)blockIdx.x * blockDim.x + threadIdx.x; iv < nvec;
+       iv += (long long)gridDim.x * blockDim.x) {
+    const long long e = iv * VEC;
+    const long long at = (long long)k * ld + e;
+    const int n = N - e < VEC ? (int)(N - e) : VEC;
+    const float sc = scale ? scale[k] : 1.0f;
+    float th[VEC], g[VEC], a[VEC];
+    if (n == VEC) {
+      ThetaTraits<TH>::lds(theta + at, th);
+#pragma unroll
+      for (int h = 0; h < VEC / 4; ++h) {
+        const float4 gv = __ldcs(reinterpret_cast<const float4*>(grad + at) + h);
+        const float4 av = __ldcs(reinterpret_cast<const float4*>(accum + at) + h);
+        g[4 * h] = gv.x; g[4 * h + 1] = gv.y; g[4 * h + 2] = gv.z; g[4 * h + 3] = gv.w;
+        a[4 * h] = av.x; a[4 * h + 1] = av.y; a[4 * h + 2] = av.z; a[4 * h + 3] = av.w;
+      }
+    } else {
+      for (int x = 0; x < n; ++x) {
+        th[x] = ThetaTraits<TH>::widen(theta[at + x]);
+        g[x] = grad[at + x];
+        a[x] = accum[at + x];
+      }
+    }
+    // where the vector lies relative to the clip ranges: 0 outside all, 1 inside one, 2 straddling
+    int where = 0;
+    if (scale) {
+      for (int r = 0; r < R.n; ++r) {
+        if (e >= R.begin[r] && e + VEC <= R.end[r]) where = 1;
+        else if (e < R.end[r] && e + VEC > R.begin[r] && where == 0) where = 2;
+      }
+    }
+#pragma unroll
+    for (int x = 0; x < VEC; ++x) {
+      if (x < n) {
+        bool inside = where == 1;
+        if (where == 2)
+          for (int r = 0; r < R.n; ++r) inside = inside || (e + x >= R.begin[r] && e + x < R.end[r]);
+        float gx = g[x];
+        if (inside) gx = __fmul_rn(gx, sc);
+        a[x] = __fadd_rn(a[x], __fmul_rn(gx, gx));
+        const float denom = __fadd_rn(__fsqrt_rn(a[x]), eps);
+        th[x] = ThetaTraits<TH>::round_store(__fsub_rn(th[x], __fdiv_rn(__fmul_rn(lr, gx), denom)));
+      }
+    }
+    if (n == VEC) {
+#pragma unroll
+      for (int h = 0; h < VEC / 4; ++h)
+        __stcs(reinterpret_cast<float4*>(accum + at) + h,
+               make_float4(a[4 * h], a[4 * h + 1], a[4 * h + 2], a[4 * h + 3]));
+      ThetaTraits<TH>::stg(theta + at, th);
+    } else {
+      for (int x = 0; x < n; ++x) {
+        accum[at + x] = a[x];
+        theta[at + x] = ThetaTraits<TH>::narrow(th[x]);
+      }
     }
   }
 }
@@ -726,6 +847,8 @@ struct gbmuf_ctx {
   int32_t* d_nbr = nullptr;
   int32_t* d_nbr_export = nullptr;
   int32_t* d_status = nullptr;
+  double* d_norm_partial = nullptr;   // [K][kNormBlocks], local_adagrad
+  float* d_clip_scale = nullptr;      // [K]
   cudaStream_t priv = nullptr;
   int num_sms = 0;
   int max_smem = 0;        // opt-in dynamic shared memory per block
@@ -926,6 +1049,17 @@ int elementwise_grid(const gbmuf_ctx* ctx, long long work_items) {
   return (int)blocks;
 }
 
+// Blocks per worker row for the kernels that put the worker on blockIdx.y: enough to cover the
+// row, capped so that the whole grid is about 16 blocks per SM.
+int row_grid(const gbmuf_ctx* ctx, long long vectors_per_row, int K) {
+  long long blocks = (vectors_per_row + 255) / 256;
+  long long cap = ((long long)ctx->num_sms * 16 + K - 1) / K;
+  if (cap < 1) cap = 1;
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  return (int)blocks;
+}
+
 void free_tables(gbmuf_ctx* ctx) {
   cudaFree(ctx->d_off); cudaFree(ctx->d_periods); cudaFree(ctx->d_mask); cudaFree(ctx->d_prefix);
   cudaFree(ctx->d_nbr); cudaFree(ctx->d_nbr_export);
@@ -1113,18 +1247,72 @@ gbmuf_status gbmuf_local_perturb(gbmuf_ctx* ctx, uint64_t step, float lr, float 
   cudaStream_t st = (cudaStream_t)stream;
   const int K = ctx->cfg.K;
   if (ctx->cfg.theta_dtype == GBMUF_F32) {
-    const int grid = elementwise_grid(ctx, (ctx->cfg.N + 3) / 4 * K);
+    const dim3 grid(row_grid(ctx, (ctx->cfg.N + 3) / 4, K), K);
     perturb_kernel<float><<<grid, 256, 0, st>>>((float*)ctx->theta, K, ctx->cfg.N, ctx->cfg.ld, key0,
                                                 key1, (uint32_t)step, nsteps, lr, sigma,
                                                 ctx->cfg.elem_base);
   } else {
-    const int grid = elementwise_grid(ctx, (ctx->cfg.N + 7) / 8 * K);
+    const dim3 grid(row_grid(ctx, (ctx->cfg.N + 7) / 8, K), K);
     perturb_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((__nv_bfloat16*)ctx->theta, K, ctx->cfg.N,
                                                         ctx->cfg.ld, key0, key1, (uint32_t)step,
                                                         nsteps, lr, sigma, ctx->cfg.elem_base);
   }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, "launch of the local-step kernel", e);
+  return GBMUF_OK;
+}
+
+gbmuf_status gbmuf_local_adagrad(gbmuf_ctx* ctx, const float* grad, float* accum, float lr,
+                                 float eps, float clip_norm, const uint8_t* clip_mask,
+                                 void* stream) {
+  if (!ctx) return GBMUF_ERR_INVALID_ARG;
+  if (!grad || !accum || (((uintptr_t)grad | (uintptr_t)accum) % 128) != 0)
+    return fail(ctx, GBMUF_ERR_INVALID_ARG, "grad and accum must be 128-byte aligned device pointers");
+  if (!(lr == lr) || !(eps == eps) || !(clip_norm == clip_norm))
+    return fail(ctx, GBMUF_ERR_INVALID_ARG, "lr, eps and clip_norm must not be NaN");
+  ClipRanges R;
+  R.n = 0;
+  const bool clip = clip_mask != nullptr && clip_norm > 0.0f;
+  if (clip) {
+    if (!ctx->partitioned) return fail(ctx, GBMUF_ERR_BAD_STATE, "a clip mask needs set_partition first");
+    for (int i = 0; i < ctx->m; ++i) {
+      if (!clip_mask[i]) continue;
+      if (R.n > 0 && R.end[R.n - 1] == ctx->off[i]) { R.end[R.n - 1] = ctx->off[i + 1]; continue; }
+      if (R.n == kMaxClipRanges)
+        return fail(ctx, GBMUF_ERR_UNSUPPORTED, "more than 16 separate runs of clipped components");
+      R.begin[R.n] = ctx->off[i];
+      R.end[R.n] = ctx->off[i + 1];
+      ++R.n;
+    }
+  }
+  DeviceGuard guard(ctx->cfg.device);
+  if (!guard.ok) return fail(ctx, GBMUF_ERR_CUDA, "cudaSetDevice failed");
+  cudaStream_t st = (cudaStream_t)stream;
+  const int K = ctx->cfg.K;
+  cudaError_t e;
+  const float* scale = nullptr;
+  if (clip && R.n > 0) {
+    if (!ctx->d_norm_partial) {
+      e = cudaMalloc(&ctx->d_norm_partial, (size_t)K * kNormBlocks * sizeof(double));
+      if (e == cudaSuccess) e = cudaMalloc(&ctx->d_clip_scale, (size_t)K * sizeof(float));
+      if (e != cudaSuccess) return fail(ctx, GBMUF_ERR_ALLOC, "scratch of the gradient-norm reduction");
+    }
+    sumsq_partial_kernel<<<dim3(kNormBlocks, K), 256, 0, st>>>(grad, ctx->cfg.ld, R, ctx->d_norm_partial);
+    clip_scale_kernel<<<(K + 127) / 128, 128, 0, st>>>(ctx->d_norm_partial, K, kNormBlocks, clip_norm,
+                                                       ctx->d_clip_scale);
+    scale = ctx->d_clip_scale;
+  }
+  if (ctx->cfg.theta_dtype == GBMUF_F32) {
+    const dim3 grid(row_grid(ctx, (ctx->cfg.N + 3) / 4, K), K);
+    adagrad_kernel<float><<<grid, 256, 0, st>>>((float*)ctx->theta, grad, accum, K, ctx->cfg.N,
+                                                ctx->cfg.ld, lr, eps, scale, R);
+  } else {
+    const dim3 grid(row_grid(ctx, (ctx->cfg.N + 7) / 8, K), K);
+    adagrad_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((__nv_bfloat16*)ctx->theta, grad, accum, K,
+                                                        ctx->cfg.N, ctx->cfg.ld, lr, eps, scale, R);
+  }
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(ctx, "launch of the Adagrad local-step kernels", e);
   return GBMUF_OK;
 }
 
@@ -1234,6 +1422,8 @@ gbmuf_status gbmuf_destroy(gbmuf_ctx* ctx) {
       if (cudaDeviceSynchronize() != cudaSuccess) rc = GBMUF_ERR_CUDA;
       free_tables(ctx);
       cudaFree(ctx->d_status);
+      cudaFree(ctx->d_norm_partial);
+      cudaFree(ctx->d_clip_scale);
       if (ctx->priv) cudaStreamDestroy(ctx->priv);
     } else {
       rc = GBMUF_ERR_CUDA;
