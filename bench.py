@@ -34,8 +34,8 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of the fused kernel per replica-parameter from an ncu capture (dram__bytes_read.sum
 # + dram__bytes_write.sum divided by the replica-parameters of the captured launch), valid only
-# for the kernel source it was taken from (sha256 of csrc/gbmuf.cu, first 12 hex digits).
-NCU_TRAFFIC = {"source_sha": "471dcd42ea5c", "bytes_per_replica_param": 6.382952e9 / 268435536}
+# for the kernel source it was taken from (source_sha() below).
+NCU_TRAFFIC = {"source_sha": "dbe65a82866d", "bytes_per_replica_param": 6.383453e9 / 268435536}
 
 
 def algorithmic_bytes_per_replica_param(dtype: int, mode: int = 0) -> int:
@@ -100,8 +100,13 @@ class ClockSampler:
 
 
 def source_sha() -> str:
+    """Fingerprint of the fused kernel's source: the part of csrc/gbmuf.cu from the barrier /
+    bulk-copy primitives to the end of sync_fused_kernel (theta traits and filter included)."""
     with open(os.path.join(ROOT, "paper_1909_09010_b200", "csrc", "gbmuf.cu"), "rb") as f:
-        return hashlib.sha256(f.read()).hexdigest()[:12]
+        text = f.read()
+    a = text.index(b"// Shared-memory barrier and bulk-copy primitives")
+    b = text.index(b"// Synthetic local step")
+    return hashlib.sha256(text[a:b]).hexdigest()[:12]
 
 
 # ------------------------------------------------------------------------------------------------
