@@ -343,3 +343,35 @@ def test_random_shapes_property():
         run(case, random_theta0(N, seed=K + N, dtype=dtype), rounds=2, sigma=5e-2, tuning=tuning)
 
     inner()
+
+
+# ------------------------------------------------------------------------------------------------
+# extremes: many components, many workers, degenerate sizes
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("m,N,seed", [(300, 40_000, 1), (700, 9_000, 2), (3000, 100_000, 3)])
+def test_many_components(m, N, seed):
+    """More components than one pass of the work-list scan (256) handles, with many one- and
+    two-element components and a mask that leaves runs of them out."""
+    g = np.random.Generator(np.random.PCG64(seed))
+    cuts = np.sort(g.choice(np.arange(1, N), size=m - 1, replace=False))
+    offsets = tuple([0] + [int(x) for x in cuts] + [N])
+    masks = [None, [int(x) for x in (g.random(m) < 0.6)], [1 if (i // 37) % 2 else 0 for i in range(m)]]
+    case = Case(K=4, offsets=offsets, p=1, q=1, eta=0.9, zeta=1.0, seed=seed)
+    run(case, random_theta0(N, seed=seed), rounds=3, masks=masks, sigma=5e-2, check_nbr=(m <= 700))
+
+
+@pytest.mark.parametrize("K,p,q,dtype", [(64, 5, 7, 0), (128, 6, 3, 1), (256, 7, 2, 0), (200, 32, 64, 0)])
+def test_many_workers(K, p, q, dtype):
+    offsets = (0, 1001, 1002, 6007)
+    case = Case(K=K, offsets=offsets, p=p, q=q, eta=0.875, zeta=1.0, dtype=dtype, seed=K)
+    run(case, random_theta0(offsets[-1], seed=K, dtype=dtype), rounds=2, sigma=5e-2)
+
+
+@pytest.mark.parametrize("K,N,p,q", [(1, 1, 0, 0), (2, 1, 1, 1), (3, 7, 1, 2), (16, 8, 3, 2), (5, 33, 2, 4)])
+def test_degenerate_sizes(K, N, p, q):
+    for dtype in (0, 1):
+        case = Case(K=K, offsets=(0, N), p=p, q=q, dtype=dtype, seed=N)
+        run(case, random_theta0(N, seed=N, dtype=dtype), rounds=3, sigma=5e-2)
+    if N >= 7:
+        case = Case(K=K, offsets=tuple(range(N + 1)), p=p, q=q, seed=N)     # every element its own component
+        run(case, random_theta0(N, seed=N), rounds=2, sigma=5e-2)
