@@ -183,6 +183,12 @@ def get(name: str, **over) -> Workload:
         cuts = tuple(int(x) // 4 * 4 for x in np.linspace(0, n, 17)[:-1]) + (n,)
         w = Workload("profile16", K=16, vocab=0, hidden=0, layers=0, p=3, q=2, eta=0.875, zeta=1.0,
                      dtype=F32, seed=2, rounds=4, local_steps=1, lr=0.1, sigma=1e-3, offsets=cuts)
+    elif name == "profile16bf":
+        # the long-run mixed-precision replica set (bf16 theta) cut down to 2^24+5 columns
+        n = (1 << 24) + 5
+        cuts = tuple(int(x) // 8 * 8 for x in np.linspace(0, n, 65)[:-1]) + (n,)
+        w = Workload("profile16bf", K=16, vocab=0, hidden=0, layers=0, p=3, q=3, eta=0.9, zeta=1.0,
+                     dtype=BF16, seed=4, rounds=4, local_steps=1, lr=0.1, sigma=1e-3, offsets=cuts)
     else:
         raise KeyError(name)
     return replace(w, **over) if over else w
