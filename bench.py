@@ -35,7 +35,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of the fused kernel per replica-parameter from an ncu capture (dram__bytes_read.sum
 # + dram__bytes_write.sum divided by the replica-parameters of the captured launch), valid only
 # for the kernel source it was taken from (source_sha() below).
-NCU_TRAFFIC = {"source_sha": "dbe65a82866d", "bytes_per_replica_param": 6.383453e9 / 268435536}
+NCU_TRAFFIC = {"source_sha": "3448523d4e7d", "bytes_per_replica_param": 6.383120e9 / 268435536}
 
 
 def algorithmic_bytes_per_replica_param(dtype: int, mode: int = 0) -> int:

@@ -146,6 +146,15 @@ gbmuf_status gbmuf_final_average(gbmuf_ctx* ctx, void* out_device, void* stream)
  * early and the buffers' contents are unspecified. */
 gbmuf_status gbmuf_device_status(gbmuf_ctx* ctx, void* stream, int32_t* out);
 
+/* Self-test of the failure reporting.  Every device-side wait in this library is bounded (two
+ * seconds of the GPU's wall clock); when one expires the kernel records GBMUF_ERR_TIMEOUT in the
+ * status word and leaves instead of hanging.  This call launches a one-warp kernel that waits on a
+ * barrier nothing ever signals, waits for it, and returns GBMUF_OK iff the wait expired and the
+ * kernel returned; *seconds_out (host, may be NULL) receives the kernel's duration.  Afterwards
+ * gbmuf_device_status reports GBMUF_ERR_TIMEOUT once (reading clears it) and the context remains
+ * fully usable.  No fault, trap or unbounded loop is involved. */
+gbmuf_status gbmuf_selftest_wait_timeout(gbmuf_ctx* ctx, void* stream, double* seconds_out);
+
 /* Launch shape of the fused kernel (one persistent CTA per SM).  Any argument may be 0 to keep
  * the built-in choice.  consumer_threads: multiple of 32 in 32..992 (one more warp issues the
  * copies); tile_elems: elements of one component staged per work item for all K workers, a

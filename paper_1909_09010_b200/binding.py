@@ -23,7 +23,8 @@ MODE_BMUF, MODE_MA = 0, 1
 EXPORTS = ["gbmuf_create", "gbmuf_set_partition", "gbmuf_init", "gbmuf_local_perturb",
            "gbmuf_sync_round", "gbmuf_get_neighbors", "gbmuf_final_average", "gbmuf_device_status",
            "gbmuf_set_tuning", "gbmuf_get_launch_info", "gbmuf_last_error", "gbmuf_destroy",
-           "gbmuf_sync_round_noalloc", "gbmuf_sync_round_host", "gbmuf_local_adagrad"]
+           "gbmuf_sync_round_noalloc", "gbmuf_sync_round_host", "gbmuf_local_adagrad",
+           "gbmuf_selftest_wait_timeout"]
 
 
 class Config(ctypes.Structure):
@@ -72,6 +73,7 @@ def lib() -> ctypes.CDLL:
     L.gbmuf_sync_round_noalloc.argtypes = [ctypes.POINTER(Config), vp, vp, vp, i32, vp, vp, u64, vp,
                                            ctypes.POINTER(i32)]
     L.gbmuf_sync_round_host.argtypes = [ctypes.POINTER(Config), vp, vp, vp, i32, vp, vp, u64, i64]
+    L.gbmuf_selftest_wait_timeout.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_double)]
     L.gbmuf_last_error.argtypes = [vp]
     L.gbmuf_last_error.restype = ctypes.c_char_p
     L.gbmuf_destroy.argtypes = [vp]
@@ -196,6 +198,12 @@ class Gbmuf:
         v = ctypes.c_int32(-1)
         self._check(lib().gbmuf_device_status(self._h, _stream(stream), ctypes.byref(v)))
         return v.value
+
+    def selftest_wait_timeout(self, stream=None) -> float:
+        """Lets a bounded device-side wait expire on purpose; returns the kernel's duration (s)."""
+        sec = ctypes.c_double(0.0)
+        self._check(lib().gbmuf_selftest_wait_timeout(self._h, _stream(stream), ctypes.byref(sec)))
+        return sec.value
 
     def set_tuning(self, consumer_threads=0, tile_elems=0, theta_stages=0, ring_slots=0, flags=0):
         self._check(lib().gbmuf_set_tuning(self._h, consumer_threads, tile_elems, theta_stages,

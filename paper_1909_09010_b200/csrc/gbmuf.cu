@@ -180,12 +180,23 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Wait for the phase with the given parity to complete.  Gives up after about a second, records
-// GBMUF_ERR_TIMEOUT in the device status word and returns false; the caller then leaves its loop.
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // two seconds
+// Wait for the phase with the given parity to complete.  Bounded in wall-clock time: after
+// kWaitLimitNs it records GBMUF_ERR_TIMEOUT in the device status word and returns false; the
+// caller then leaves its loop.  (try_wait may itself suspend the thread for a while, so the bound
+// is on the timer, not on the number of tries.)
 __device__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, int32_t* status) {
-  for (uint32_t spin = 0; spin < (1u << 22); ++spin) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_timer_ns();
+  for (uint32_t spin = 0;; ++spin) {
     if (mbar_try_wait(bar, parity)) return true;
     if (spin > 32) __nanosleep(spin > 4096 ? 256 : 32);
+    if ((spin & 63) == 63 && global_timer_ns() - t0 > kWaitLimitNs) break;
   }
   atomicExch(status, (int32_t)GBMUF_ERR_TIMEOUT);
   return false;
@@ -558,6 +569,20 @@ sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_th
     }
     mbar_arrive(bars + kBarThetaEmpty + 8 * s);          // this thread is done with the theta stage
   }
+}
+
+// Self-test of the bounded wait: one warp waits on a barrier that nothing will ever signal.  The
+// wait must expire, set the status word and return; nothing here can hang or trap.
+__global__ void wait_timeout_selftest_kernel(int32_t* status, int32_t* returned) {
+  __shared__ __align__(8) unsigned long long bar_storage;
+  const uint32_t bar = smem_u32(&bar_storage);
+  if (threadIdx.x == 0) {
+    mbar_init(bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  const bool ok = mbar_wait_bounded(bar, 0, status);
+  if (threadIdx.x == 0) *returned = ok ? 1 : 2;
 }
 
 // =================================================================================================
@@ -1391,6 +1416,37 @@ gbmuf_status gbmuf_final_average(gbmuf_ctx* ctx, void* out, void* stream) {
                                                               ctx->cfg.N, ctx->cfg.ld);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, "launch of the final-average kernel", e);
+  return GBMUF_OK;
+}
+
+gbmuf_status gbmuf_selftest_wait_timeout(gbmuf_ctx* ctx, void* stream, double* seconds_out) {
+  if (!ctx) return GBMUF_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->cfg.device);
+  if (!guard.ok) return fail(ctx, GBMUF_ERR_CUDA, "cudaSetDevice failed");
+  cudaStream_t st = (cudaStream_t)stream;
+  int32_t* d_ret = nullptr;
+  cudaEvent_t a = nullptr, b = nullptr;
+  cudaError_t e = cudaMalloc(&d_ret, sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaMemsetAsync(d_ret, 0, sizeof(int32_t), st);
+  if (e == cudaSuccess) e = cudaEventCreate(&a);
+  if (e == cudaSuccess) e = cudaEventCreate(&b);
+  if (e == cudaSuccess) e = cudaEventRecord(a, st);
+  if (e == cudaSuccess) {
+    wait_timeout_selftest_kernel<<<1, 32, 0, st>>>(ctx->d_status, d_ret);
+    e = cudaGetLastError();
+  }
+  if (e == cudaSuccess) e = cudaEventRecord(b, st);
+  int32_t ret = 0;
+  if (e == cudaSuccess) e = cudaMemcpyAsync(&ret, d_ret, sizeof(ret), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  float ms = 0.f;
+  if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, a, b);
+  if (a) cudaEventDestroy(a);
+  if (b) cudaEventDestroy(b);
+  cudaFree(d_ret);
+  if (e != cudaSuccess) return cuda_fail(ctx, "wait-timeout self-test", e);
+  if (seconds_out) *seconds_out = ms / 1e3;
+  if (ret != 2) return fail(ctx, GBMUF_ERR_BAD_STATE, "the self-test wait did not expire as it should");
   return GBMUF_OK;
 }
 

@@ -375,3 +375,21 @@ def test_degenerate_sizes(K, N, p, q):
     if N >= 7:
         case = Case(K=K, offsets=tuple(range(N + 1)), p=p, q=q, seed=N)     # every element its own component
         run(case, random_theta0(N, seed=N), rounds=2, sigma=5e-2)
+
+
+def test_expired_wait_is_reported_not_hung():
+    """Failure reporting without a fault: a wait on a barrier that nothing signals expires after
+    its two-second limit, the kernel returns, the status word says TIMEOUT once, and the context
+    goes on working."""
+    w = workloads.get("tiny")
+    pr = Pair(case_of(w), workloads.theta0_numpy(w))
+    try:
+        pr.perturb(1, 0.1, 0.05)
+        sec = pr.g.selftest_wait_timeout()
+        assert 1.5 < sec < 10.0, sec
+        assert pr.g.device_status() == binding.ERR_TIMEOUT
+        assert pr.g.device_status() == 0                   # reading cleared it
+        pr.sync(1)
+        pr.compare("round after the expired wait")
+    finally:
+        pr.close()
