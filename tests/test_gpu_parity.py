@@ -393,3 +393,52 @@ def test_expired_wait_is_reported_not_hung():
         pr.compare("round after the expired wait")
     finally:
         pr.close()
+
+
+@pytest.mark.parametrize("dtype", [0, 1])
+def test_special_values_propagate_identically(dtype):
+    """Denormals (no flush-to-zero), signed zeros, infinities, NaN and extreme magnitudes go
+    through the round as IEEE arithmetic dictates: bit-equal with the oracle wherever the result
+    is not NaN, NaN exactly where the oracle has NaN."""
+    K, N = 8, 6000
+    offsets = (0, 1000, 1001, 4003, N)
+    g = np.random.Generator(np.random.PCG64(12))
+    theta0 = (g.standard_normal(N) * 0.1).astype(np.float32)
+    specials = np.array([0.0, -0.0, 1e-45, -1e-45, 1e-40, 3e-39, 1.1754944e-38, 3.4e38, -3.4e38,
+                         np.inf, -np.inf, np.nan, 1e30, -1e-30, 65504.0, 1.0], dtype=np.float32)
+    theta0[g.choice(N, size=400, replace=False)] = g.choice(specials, size=400)
+    theta0[1001:1200] = (g.integers(-2000, 2000, size=199) * 1e-42).astype(np.float32)   # a denormal stretch
+    if dtype == 1:
+        theta0 = oracle.f32_to_bf16(theta0)
+    case = Case(K=K, offsets=offsets, p=2, q=2, eta=0.9, zeta=1.0, dtype=dtype, seed=3)
+    pr = Pair(case, theta0)
+    try:
+        drift = (g.standard_normal((K, N)) * 0.05).astype(np.float32)
+        drift[g.random((K, N)) < 0.02] = np.float32(1e-42)           # denormal nudges
+        drift[:, 1001:1200] = (g.integers(-500, 500, size=(K, 199)) * 1e-43).astype(np.float32)
+        saw_denormal = False
+        if dtype == 0:
+            pr.add_drift(drift)
+        else:
+            pr.perturb(1, 1.0, 0.05)
+        for r in (1, 2, 3):
+            pr.sync(r)
+            torch.cuda.synchronize()
+            st = pr.states[0]
+            for name, got, ref in (("omega", to_numpy(pr.omega), st.omega), ("delta", to_numpy(pr.delta), st.delta),
+                                   ("theta", to_numpy(pr.theta), st.theta)):
+                if ref.dtype == np.uint16:
+                    gf, rf = oracle.bf16_to_f32(got), oracle.bf16_to_f32(ref)
+                else:
+                    gf, rf = got, ref
+                nan_g, nan_r = np.isnan(gf), np.isnan(rf)
+                assert np.array_equal(nan_g, nan_r), f"{name}: NaN pattern differs in round {r}"
+                assert np.array_equal(got[~nan_r], ref[~nan_r]) and \
+                    np.array_equal(np.signbit(gf[~nan_r]), np.signbit(rf[~nan_r])), f"{name} round {r}"
+            assert pr.g.device_status() == 0
+            d = st.delta[np.isfinite(st.delta)]
+            saw_denormal = saw_denormal or bool((np.abs(d[d != 0]) < 1.1754944e-38).any())
+        assert np.isnan(st.theta if dtype == 0 else oracle.bf16_to_f32(st.theta)).any()
+        assert saw_denormal or dtype == 1, "the test never produced a denormal Delta"
+    finally:
+        pr.close()
