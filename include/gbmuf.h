@@ -55,7 +55,8 @@ typedef enum { GBMUF_F32 = 0, GBMUF_BF16 = 1 } gbmuf_dtype;
 typedef enum { GBMUF_MODE_BMUF = 0, GBMUF_MODE_MA = 1 } gbmuf_mode;
 
 typedef struct {
-  int32_t K;           /* number of workers n (Definition 1), 1 <= K <= 65535                     */
+  int32_t K;           /* number of workers n (Definition 1), 1 <= K <= 256 (all K slices of a
+                          tile are staged together on one SM)                                     */
   int64_t N;           /* parameters per replica, >= 1                                            */
   int64_t ld;          /* row stride in elements: >= N, multiple of 32                            */
   int32_t p;           /* symmetric degree of the ring (Definition 1), >= 0; the candidate set of
@@ -77,7 +78,7 @@ typedef struct {
 /* Bind a context to three caller-owned device buffers (theta, omega, delta: [K][ld], see the
  * conventions above).  Allocates only small tables (a few KB plus 4*K*m*q bytes later on).
  * The buffers must stay valid until gbmuf_destroy.  Errors: INVALID_ARG (any range, alignment or
- * NULL violation; q > c), UNSUPPORTED (K*element size too large for one staged tile, c > 64),
+ * NULL violation; q > c), UNSUPPORTED (K > 256, ld >= 2^31, c > 64),
  * CUDA, ALLOC. */
 gbmuf_status gbmuf_create(const gbmuf_config* cfg, void* theta_device, float* omega_device,
                           float* delta_device, gbmuf_ctx** out);

@@ -1102,7 +1102,7 @@ extern "C" {
 gbmuf_status gbmuf_create(const gbmuf_config* cfg, void* theta, float* omega, float* delta,
                           gbmuf_ctx** out) {
   if (!cfg || !out) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "cfg and out must not be NULL");
-  if (cfg->K < 1 || cfg->K > 65535) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "K must be in 1..65535");
+  if (cfg->K < 1) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "K must be >= 1");
   if (cfg->N < 1) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "N must be >= 1");
   if (cfg->ld < cfg->N || cfg->ld % 32 != 0)
     return fail(nullptr, GBMUF_ERR_INVALID_ARG, "ld must be >= N and a multiple of 32");

@@ -49,7 +49,7 @@ def test_argument_errors_need_no_gpu():
         return L.gbmuf_create(ctypes.byref(cfg), fake, fake, fake, ctypes.byref(h))
 
     assert create(K=0) == binding.ERR_INVALID_ARG
-    assert create(K=70000) == binding.ERR_INVALID_ARG
+    assert create(K=70000, p=1, q=1) == binding.ERR_UNSUPPORTED     # more than 256 workers
     assert create(N=0) == binding.ERR_INVALID_ARG
     assert create(ld=96) == binding.ERR_INVALID_ARG            # ld < N
     assert create(ld=130) == binding.ERR_INVALID_ARG           # not a multiple of 32
