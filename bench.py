@@ -33,9 +33,11 @@ UNIT = "replica-params/s"
 FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of the fused kernel per replica-parameter from an ncu capture (dram__bytes_read.sum
-# + dram__bytes_write.sum divided by the replica-parameters of the captured launch), valid only
+# + dram__bytes_write.sum divided by the replica-parameters of the captured launch; key = theta
+# dtype: 0 fp32 from workload profile16, 1 bf16 from profile16bf), valid only
 # for the kernel source it was taken from (source_sha() below).
-NCU_TRAFFIC = {"source_sha": "3448523d4e7d", "bytes_per_replica_param": 6.383120e9 / 268435536}
+NCU_TRAFFIC = {"source_sha": "ca6a56ca1eb2", "bytes_per_replica_param": {0: 6.382624e9 / 268435536,
+                                                                   1: 5.309772e9 / 268435536}}
 
 
 def algorithmic_bytes_per_replica_param(dtype: int, mode: int = 0) -> int:
@@ -289,8 +291,8 @@ def run_gpu(args, w):
         t_launch = (sum(sync_ms) / len(sync_ms)) / 1e3
         achieved = bpe * K * N / t_launch / 1e9
         traffic = None
-        if NCU_TRAFFIC["source_sha"] == source_sha() and NCU_TRAFFIC["bytes_per_replica_param"]:
-            traffic = NCU_TRAFFIC["bytes_per_replica_param"] * K * N
+        if NCU_TRAFFIC["source_sha"] == source_sha():
+            traffic = NCU_TRAFFIC["bytes_per_replica_param"][w.dtype] * K * N
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": total_sync_s / args.steps * 1e3,
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -301,6 +303,7 @@ def run_gpu(args, w):
                            "l2": "inputs_larger_than_l2 (state %.1f GB per GPU)" %
                                  ((K * ld * (8 + (4 if w.dtype == 0 else 2))) / 1e9),
                            "launch": info, "local_step_ms": sum(pert_ms) / len(pert_ms),
+                           "round_plus_local_step_ms": (sum(pert_ms) + sum(sync_ms)) / len(sync_ms),
                            "sync_ms_min": min(sync_ms), "sync_ms_max": max(sync_ms),
                            "device_status": status},
                 "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",

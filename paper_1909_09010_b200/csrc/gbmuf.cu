@@ -240,7 +240,9 @@ template <> struct ThetaTraits<float> {
   }
   static __device__ __forceinline__ void stg(float* p, const float (&x)[4]) {
     __stcs(reinterpret_cast<float4*>(p), make_float4(x[0], x[1], x[2], x[3]));
-  }
+  }  // four consecutive elements (what one thread of the fused kernel handles per row)
+  static __device__ __forceinline__ void lds_quad(const float* p, float (&x)[4]) { lds(p, x); }
+  static __device__ __forceinline__ void stg_quad(float* p, const float (&x)[4]) { stg(p, x); }
 };
 template <> struct ThetaTraits<__nv_bfloat16> {
   static constexpr int VEC = 8;
@@ -265,6 +267,19 @@ template <> struct ThetaTraits<__nv_bfloat16> {
     h = __floats2bfloat162_rn(x[4], x[5]); t.z = *reinterpret_cast<uint32_t*>(&h);
     h = __floats2bfloat162_rn(x[6], x[7]); t.w = *reinterpret_cast<uint32_t*>(&h);
     __stcs(reinterpret_cast<uint4*>(p), t);
+  }
+  // four consecutive elements = 8 bytes
+  static __device__ __forceinline__ void lds_quad(const __nv_bfloat16* p, float (&x)[4]) {
+    const uint2 t = *reinterpret_cast<const uint2*>(p);
+    x[0] = __uint_as_float(t.x << 16); x[1] = __uint_as_float(t.x & 0xFFFF0000u);
+    x[2] = __uint_as_float(t.y << 16); x[3] = __uint_as_float(t.y & 0xFFFF0000u);
+  }
+  static __device__ __forceinline__ void stg_quad(__nv_bfloat16* p, const float (&x)[4]) {
+    uint2 t;
+    __nv_bfloat162 h;
+    h = __floats2bfloat162_rn(x[0], x[1]); t.x = *reinterpret_cast<uint32_t*>(&h);
+    h = __floats2bfloat162_rn(x[2], x[3]); t.y = *reinterpret_cast<uint32_t*>(&h);
+    __stcs(reinterpret_cast<uint2*>(p), t);
   }
 };
 
@@ -344,8 +359,7 @@ __device__ __forceinline__ void bmuf_filter(float avg, float& w, float& d, float
 template <typename TH>
 __global__ void __launch_bounds__(1024, 1)
 sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_theta) {
-  constexpr int VEC = ThetaTraits<TH>::VEC;
-  constexpr int NF4 = VEC / 4;
+  constexpr int VEC = 4;   // elements per thread and row: 16 bytes of omega / Delta, 16 or 8 of theta
   extern __shared__ __align__(128) unsigned char smem[];
   const uint32_t bars = smem_u32(smem);
   unsigned char* stage0 = smem + kBarBytes;
@@ -393,7 +407,6 @@ sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_th
     }
     int theta_issued = 0;    // tiles whose theta stage has been requested
     int ring_issued = 0;     // ring slots requested so far (over all tiles)
-    int ring_tile_done = 0;  // tiles whose omega/Delta rows have all been requested
 
     // request the theta stage of this CTA's j-th tile (j = theta_issued)
     auto issue_theta = [&]() -> bool {
@@ -467,7 +480,6 @@ sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_th
           }
           ++ring_issued;
         }
-        if (ok) ++ring_tile_done;
       }
     }
     if (!ok) {
@@ -477,7 +489,6 @@ sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_th
       for (int j = ring_issued > R ? ring_issued - R : 0; j < ring_issued; ++j)
         mbar_wait_bounded(bars + kBarRingFull + 8 * (j % R), (j / R) & 1, P.status);
     }
-    (void)ring_tile_done;
     return;
   }
 
@@ -514,9 +525,9 @@ sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_th
         const int boxbase = b * box_elems + cin;
         // gossip average: own slice first, then the neighbours in draw order
         float a[VEC], t[VEC];
-        ThetaTraits<TH>::lds(sth + boxbase + k * BW, a);
+        ThetaTraits<TH>::lds_quad(sth + boxbase + k * BW, a);
         for (int j = 0; j < q; ++j) {
-          ThetaTraits<TH>::lds(sth + boxbase + snb[k * q + j] * BW, t);
+          ThetaTraits<TH>::lds_quad(sth + boxbase + snb[k * q + j] * BW, t);
 #pragma unroll
           for (int x = 0; x < VEC; ++x) a[x] = __fadd_rn(a[x], t[x]);
         }
@@ -527,30 +538,22 @@ sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_th
         const bool whole = e >= lo && e + VEC <= hi;
         if (!bmuf) {                                       // gossip-MA: theta <- average
           if (whole) {
-            ThetaTraits<TH>::stg(theta + at, a);
+            ThetaTraits<TH>::stg_quad(theta + at, a);
           } else {
             for (int x = 0; x < VEC; ++x)
               if (e + x >= lo && e + x < hi) theta[at + x] = ThetaTraits<TH>::narrow(a[x]);
           }
           continue;
         }
-        float4 W[NF4], D[NF4];
-#pragma unroll
-        for (int f = 0; f < NF4; ++f) {
-          W[f] = *reinterpret_cast<const float4*>(som + col + 4 * f);
-          D[f] = *reinterpret_cast<const float4*>(sde + col + 4 * f);
-        }
-        float* wv = reinterpret_cast<float*>(&W[0]);
-        float* dv = reinterpret_cast<float*>(&D[0]);
+        const float4 W = *reinterpret_cast<const float4*>(som + col);
+        const float4 D = *reinterpret_cast<const float4*>(sde + col);
+        float wv[VEC] = {W.x, W.y, W.z, W.w}, dv[VEC] = {D.x, D.y, D.z, D.w};
 #pragma unroll
         for (int x = 0; x < VEC; ++x) bmuf_filter<TH>(a[x], wv[x], dv[x], t[x], P.eta, P.zeta);
         if (whole) {
-#pragma unroll
-          for (int f = 0; f < NF4; ++f) {
-            __stcs(reinterpret_cast<float4*>(P.delta + at) + f, D[f]);
-            __stcs(reinterpret_cast<float4*>(P.omega + at) + f, W[f]);
-          }
-          ThetaTraits<TH>::stg(theta + at, t);
+          __stcs(reinterpret_cast<float4*>(P.delta + at), make_float4(dv[0], dv[1], dv[2], dv[3]));
+          __stcs(reinterpret_cast<float4*>(P.omega + at), make_float4(wv[0], wv[1], wv[2], wv[3]));
+          ThetaTraits<TH>::stg_quad(theta + at, t);
         } else {
           // a vector that straddles the edge of the component: only the elements this tile owns
           for (int x = 0; x < VEC; ++x) {
@@ -951,7 +954,6 @@ gbmuf_status build_tensor_maps(gbmuf_ctx* ctx, const Launch& L) {
 gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
   const int K = ctx->cfg.K, q = ctx->cfg.q;
   const int esz = (int)theta_size(ctx);
-  const int VEC = 16 / esz;
   const bool bmuf = ctx->cfg.mode == GBMUF_MODE_BMUF;
   Launch L;
   L.flags = t.flags;
@@ -1004,8 +1006,8 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
   if (t.ncons) {
     L.ncons = t.ncons;
   } else {
-    int n = (L.T / VEC + 31) / 32 * 32;        // one vector per thread and row, within 128..512
-    L.ncons = n < 128 ? 128 : n > 512 ? 512 : n;
+    int n = (L.T / 4 + 31) / 32 * 32;          // one quad per thread and row, within 128..992
+    L.ncons = n < 128 ? 128 : n > 992 ? 992 : n;
   }
   *out = L;
   return GBMUF_OK;
