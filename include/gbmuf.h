@@ -216,6 +216,36 @@ gbmuf_status gbmuf_sync_round_noalloc(const gbmuf_config* cfg, void* theta_devic
                                       const int64_t* offsets_host, const uint8_t* comp_mask_host,
                                       uint64_t round, void* stream, int32_t* device_status_out);
 
+/* ---- one worker per GPU ("peer" form) ------------------------------------------------------------
+ * The deployment the paper describes: every worker owns a GPU and, at a synchronisation step,
+ * obtains the chosen neighbours' copies of each component (Algorithm 1, neighbour choice and
+ * averaging lines; Section 3, experimental platform).  Here worker `rank` holds its own theta in
+ * TWO buffers (a round reads one and writes the other), its omega and Delta ([ld] each), and
+ * pointers to every other worker's two theta buffers, mapped into this process (CUDA IPC / peer
+ * access; setting that up is the caller's business).  A round draws this worker's neighbours
+ * exactly as gbmuf_sync_round does for worker `rank` (same seed, round, global component index),
+ * and ONE kernel pulls their slices from peer memory (bulk copies without multicast), averages
+ * (own value first, then draw order), filters, writes omega and Delta in place and the new theta
+ * into the worker's other buffer.  Components that do not take part are copied to the other
+ * buffer unchanged, so after the round the other buffer is the worker's complete theta.
+ * Protocol: all workers call gbmuf_peer_sync_round(round, read_buffer = b), then synchronise
+ * with one another (every worker's kernel finished), then use b' = 1 - b for the next round.
+ * Within a round nobody writes a buffer that anybody reads, so no other ordering is needed.
+ * theta_bufs: host array of 2*K device pointers, theta_bufs[b*K + j] = buffer b of worker j
+ * (entry `rank` is this worker's own memory); all [ld] elements of theta's dtype, 128-byte
+ * aligned, valid until gbmuf_peer_destroy.  cfg: K = number of workers, N, ld, p, q <= 15, eta,
+ * zeta, mode, theta_dtype, seed, device, comp_base as for gbmuf_create.
+ * Errors as for the context calls; text via gbmuf_last_error(NULL) on the calling thread. */
+typedef struct gbmuf_peer gbmuf_peer;
+gbmuf_status gbmuf_peer_create(const gbmuf_config* cfg, int32_t rank, void* const* theta_bufs_host,
+                               float* omega_device, float* delta_device, gbmuf_peer** out);
+gbmuf_status gbmuf_peer_set_partition(gbmuf_peer* h, int32_t m, const int64_t* offsets_host,
+                                      const int32_t* periods_host);
+gbmuf_status gbmuf_peer_sync_round(gbmuf_peer* h, uint64_t round, const uint8_t* comp_mask_host,
+                                   int32_t read_buffer, void* stream);
+gbmuf_status gbmuf_peer_device_status(gbmuf_peer* h, void* stream, int32_t* out);
+gbmuf_status gbmuf_peer_destroy(gbmuf_peer* h);
+
 /* Sentence about the last error on this context ("" if none); valid until the next call on it.
  * With ctx == NULL: the last error of a failed gbmuf_create on this thread. */
 const char* gbmuf_last_error(const gbmuf_ctx* ctx);

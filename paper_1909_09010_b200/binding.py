@@ -24,7 +24,8 @@ EXPORTS = ["gbmuf_create", "gbmuf_set_partition", "gbmuf_init", "gbmuf_local_per
            "gbmuf_sync_round", "gbmuf_get_neighbors", "gbmuf_final_average", "gbmuf_device_status",
            "gbmuf_set_tuning", "gbmuf_get_launch_info", "gbmuf_last_error", "gbmuf_destroy",
            "gbmuf_sync_round_noalloc", "gbmuf_sync_round_host", "gbmuf_local_adagrad",
-           "gbmuf_selftest_wait_timeout"]
+           "gbmuf_selftest_wait_timeout", "gbmuf_peer_create", "gbmuf_peer_set_partition",
+           "gbmuf_peer_sync_round", "gbmuf_peer_device_status", "gbmuf_peer_destroy"]
 
 
 class Config(ctypes.Structure):
@@ -74,6 +75,11 @@ def lib() -> ctypes.CDLL:
                                            ctypes.POINTER(i32)]
     L.gbmuf_sync_round_host.argtypes = [ctypes.POINTER(Config), vp, vp, vp, i32, vp, vp, u64, i64]
     L.gbmuf_selftest_wait_timeout.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_double)]
+    L.gbmuf_peer_create.argtypes = [ctypes.POINTER(Config), i32, vp, vp, vp, ctypes.POINTER(vp)]
+    L.gbmuf_peer_set_partition.argtypes = [vp, i32, vp, vp]
+    L.gbmuf_peer_sync_round.argtypes = [vp, u64, vp, i32, vp]
+    L.gbmuf_peer_device_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
+    L.gbmuf_peer_destroy.argtypes = [vp]
     L.gbmuf_last_error.argtypes = [vp]
     L.gbmuf_last_error.restype = ctypes.c_char_p
     L.gbmuf_destroy.argtypes = [vp]
@@ -133,6 +139,55 @@ def sync_round_host(theta, omega, delta, offsets, rnd, *, K, N, ld, p, q, eta, z
                                      off.shape[0] - 1, _ptr(off), _ptr(mask), rnd, chunk_cols)
     if st != GBMUF_OK:
         raise GbmufError(st, lib().gbmuf_last_error(None).decode())
+
+
+class GbmufPeer:
+    """One worker of the one-worker-per-GPU form.  ``theta_bufs[b][j]`` is buffer b (0/1) of worker j
+    (tensors or raw device addresses; entry ``rank`` is this worker's own memory)."""
+
+    def __init__(self, rank, theta_bufs, omega, delta, *, K, N, ld, p, q, eta, zeta, seed=0,
+                 mode=MODE_BMUF, theta_dtype=F32, device=0, comp_base=0):
+        self._h = ctypes.c_void_p()
+        self.cfg = Config(K, N, ld, p, q, eta, zeta, mode, theta_dtype, seed, device, comp_base, 0)
+        self._keep = (theta_bufs, omega, delta)
+        addr = [(t if isinstance(t, int) else t.data_ptr()) for b in (0, 1) for t in theta_bufs[b]]
+        arr = (ctypes.c_void_p * (2 * K))(*addr)
+        st = lib().gbmuf_peer_create(ctypes.byref(self.cfg), rank, arr, _ptr(omega), _ptr(delta),
+                                     ctypes.byref(self._h))
+        if st != GBMUF_OK:
+            raise GbmufError(st, lib().gbmuf_last_error(None).decode())
+        self.m = 0
+
+    def _check(self, st):
+        if st != GBMUF_OK:
+            raise GbmufError(st, lib().gbmuf_last_error(None).decode())
+
+    def set_partition(self, offsets, periods=None):
+        off = np.ascontiguousarray(offsets, dtype=np.int64)
+        per = None if periods is None else np.ascontiguousarray(periods, dtype=np.int32)
+        self._check(lib().gbmuf_peer_set_partition(self._h, off.shape[0] - 1, _ptr(off), _ptr(per)))
+        self.m = off.shape[0] - 1
+
+    def sync_round(self, rnd, read_buffer, comp_mask=None, stream=None):
+        mask = None if comp_mask is None else np.ascontiguousarray(comp_mask, dtype=np.uint8)
+        self._check(lib().gbmuf_peer_sync_round(self._h, rnd, _ptr(mask), read_buffer, _stream(stream)))
+
+    def device_status(self, stream=None) -> int:
+        v = ctypes.c_int32(-1)
+        self._check(lib().gbmuf_peer_device_status(self._h, _stream(stream), ctypes.byref(v)))
+        return v.value
+
+    def destroy(self):
+        if self._h:
+            lib().gbmuf_peer_destroy(self._h)
+            self._h = ctypes.c_void_p()
+            self._keep = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
 
 
 class Gbmuf:

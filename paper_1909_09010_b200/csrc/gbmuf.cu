@@ -837,6 +837,233 @@ __global__ void __launch_bounds__(256) final_average_kernel(const TH* theta, TH*
 }
 
 // =================================================================================================
+// One worker per GPU ("peer" form): this GPU holds worker `rank`'s theta (two buffers, read one /
+// write the other), omega and Delta; the other workers' theta buffers are peer-mapped pointers.
+// For every participating component the worker's q neighbours are drawn exactly as in the
+// resident form, and the fused kernel pulls their slices straight from peer memory with
+// non-multicast bulk copies into the same shared-memory stage as its own theta, omega and Delta
+// slices, averages (own first, then draw order), filters, and writes omega and Delta in place and
+// the new theta into the OTHER buffer: peers that are still reading this worker's current buffer
+// never see a half-updated replica.  Components that do not take part are copied through to the
+// other buffer.  Every row of a stage passes through once, so stages are simply pipelined.
+// =================================================================================================
+struct PeerPlanParams {
+  int K, m, p, q, comp_base, rank, use_mask;
+  uint64_t seed, round;
+  const int32_t* periods;
+  const uint8_t* mask;
+  int32_t* nbr;    // [m][q] neighbours of worker `rank`
+  uint8_t* due;    // [m]
+};
+
+__global__ void __launch_bounds__(256) peer_plan_kernel(PeerPlanParams P) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= P.m) return;
+  P.due[i] = P.use_mask ? (P.mask[i] != 0) : (P.round % (uint64_t)P.periods[i] == 0);
+  if (P.q == 0) return;
+  int32_t a[kMaxCand];
+  const int c = ring_candidates(P.rank, P.K, P.p, a);
+  Philox4 r = {0, 0, 0, 0};
+  for (int j = 0; j < P.q && j < c; ++j) {
+    if ((j & 3) == 0) {
+      Philox4 ctr = {(uint32_t)P.round, (uint32_t)(P.round >> 32), (uint32_t)(P.comp_base + i),
+                     (uint32_t)P.rank | ((uint32_t)(j >> 2) << 16)};
+      r = philox4x32_10(ctr, (uint32_t)P.seed, (uint32_t)(P.seed >> 32) ^ kTagSampler);
+    }
+    const uint32_t u = (j & 3) == 0 ? r.x : (j & 3) == 1 ? r.y : (j & 3) == 2 ? r.z : r.w;
+    const int t = j + (int)__umulhi(u, (uint32_t)(c - j));
+    const int32_t tmp = a[j];
+    a[j] = a[t];
+    a[t] = tmp;
+    P.nbr[(size_t)i * P.q + j] = a[j];
+  }
+}
+
+struct PeerParams {
+  const void* const* theta_in;   // device array [K]: worker j's current theta buffer (peers included)
+  void* theta_out;               // this worker's other buffer
+  float* omega;                  // this worker's, [N]
+  float* delta;
+  const int64_t* off;            // [m+1]
+  const int32_t* tile_prefix;    // [m+1], over ALL components
+  const int32_t* nbr;            // [m][q]
+  const uint8_t* due;            // [m]
+  int32_t* status;
+  long long N;                   // columns; rows are read up to N rounded up to 8 (<= ld)
+  int rank, m, q, mode;
+  float eta, zeta, qp1, inv_qp1;
+  int inv_exact;
+  int T, stages, ncons;
+  uint32_t stage_stride, omega_off, delta_off, desc_off;   // stage: [q+1 theta rows | omega | Delta | desc]
+};
+
+template <typename TH>
+__global__ void __launch_bounds__(1024, 1) peer_round_kernel(const PeerParams P) {
+  constexpr int VEC = 4;
+  extern __shared__ __align__(128) unsigned char smem[];
+  const uint32_t bars = smem_u32(smem);            // [0,64) full, [64,128) empty
+  unsigned char* stage0 = smem + 128;
+  const int total = P.tile_prefix[P.m];
+  const int S = P.stages;
+  const bool bmuf = P.mode == GBMUF_MODE_BMUF;
+  const int my_tiles = (int)blockIdx.x < total ? (total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(bars + 8 * s, 1);
+      mbar_init(bars + 64 + 8 * s, P.ncons);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+
+  if (threadIdx.x < 32) {
+    // ------------------------------------------------------------------ producer warp
+    const int lane = threadIdx.x;
+    int comp = 0, pfx_lo = 0, pfx_hi = 0;
+    long long cb = 0, ce = 0;
+    if (my_tiles > 0) {
+      int lo_i = 0, hi_i = P.m;
+      while (hi_i - lo_i > 1) {
+        const int mid = (lo_i + hi_i) >> 1;
+        if (__ldg(P.tile_prefix + mid) <= (int)blockIdx.x) lo_i = mid; else hi_i = mid;
+      }
+      comp = lo_i;
+      pfx_lo = __ldg(P.tile_prefix + comp);
+      pfx_hi = __ldg(P.tile_prefix + comp + 1);
+      cb = __ldg(P.off + comp);
+      ce = __ldg(P.off + comp + 1);
+    }
+    int issued = 0;
+    bool ok = true;
+    const long long row_end = (P.N + kAlign - 1) & ~(long long)(kAlign - 1);
+    for (int it = 0; it < my_tiles; ++it) {
+      const int w = (int)blockIdx.x + it * (int)gridDim.x;
+      const int s = it % S;
+      if (it >= S) {
+        ok = mbar_wait_bounded(bars + 64 + 8 * s, ((it / S) - 1) & 1, P.status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+      }
+      if (w >= pfx_hi) {
+        while (w >= pfx_hi) {
+          ++comp;
+          pfx_lo = pfx_hi;
+          pfx_hi = __ldg(P.tile_prefix + comp + 1);
+        }
+        cb = __ldg(P.off + comp);
+        ce = __ldg(P.off + comp + 1);
+      }
+      const long long e0 = (cb & ~(long long)(kAlign - 1)) + (long long)(w - pfx_lo) * P.T;
+      long long load_end = (ce + kAlign - 1) & ~(long long)(kAlign - 1);
+      if (load_end > e0 + P.T) load_end = e0 + P.T;
+      if (load_end > row_end) load_end = row_end;
+      const uint32_t nelem = (uint32_t)(load_end - e0);
+      const uint32_t bytes_th = nelem * (uint32_t)sizeof(TH), bytes_f = nelem * 4u;
+      const bool due = __ldg(P.due + comp) != 0;
+      unsigned char* st = stage0 + (size_t)s * P.stage_stride;
+      if (lane == 0) {
+        TileDesc* d = reinterpret_cast<TileDesc*>(st + P.desc_off);
+        d->e0 = e0;
+        d->lo = cb > e0 ? cb : e0;
+        d->hi = ce < e0 + P.T ? ce : e0 + P.T;
+        d->comp = due ? comp : -1 - comp;            // negative: copy the component through
+      }
+      const uint32_t full = bars + 8 * s;
+      const int nrows = due ? P.q + 1 : 1;
+      if (lane == 0)
+        mbar_arrive_expect_tx(full, (uint32_t)nrows * bytes_th + ((due && bmuf) ? 2u * bytes_f : 0u));
+      __syncwarp();
+      const uint32_t sbase = smem_u32(st);
+      for (int r = lane; r < nrows; r += 32) {
+        const int src_worker = r == 0 ? P.rank : __ldg(P.nbr + (size_t)comp * P.q + (r - 1));
+        const TH* row = static_cast<const TH*>(P.theta_in[src_worker]);   // own or a peer's memory
+        bulk_load_row(sbase + (uint32_t)r * (uint32_t)P.T * (uint32_t)sizeof(TH), row + e0, bytes_th, full);
+      }
+      if (due && bmuf && lane == 0) {
+        bulk_load_row(sbase + P.omega_off, P.omega + e0, bytes_f, full);
+        bulk_load_row(sbase + P.delta_off, P.delta + e0, bytes_f, full);
+      }
+      issued = it + 1;
+    }
+    if (!ok) {
+      for (int it = issued > S ? issued - S : 0; it < issued; ++it)
+        mbar_wait_bounded(bars + 8 * (it % S), (it / S) & 1, P.status);
+    }
+    return;
+  }
+
+  // -------------------------------------------------------------------- consumer warps
+  const int c = threadIdx.x - 32;
+  const int nv = P.T / VEC, q = P.q, T = P.T;
+  TH* out = static_cast<TH*>(P.theta_out);
+  for (int it = 0; it < my_tiles; ++it) {
+    const int s = it % S;
+    if (!mbar_wait_bounded(bars + 8 * s, (it / S) & 1, P.status)) return;
+    unsigned char* st = stage0 + (size_t)s * P.stage_stride;
+    const TH* sth = reinterpret_cast<const TH*>(st);
+    const float* som = reinterpret_cast<const float*>(st + P.omega_off);
+    const float* sde = reinterpret_cast<const float*>(st + P.delta_off);
+    const TileDesc* d = reinterpret_cast<const TileDesc*>(st + P.desc_off);
+    const long long e0 = d->e0, lo = d->lo, hi = d->hi;
+    const bool due = d->comp >= 0;
+    for (int v = c; v < nv; v += P.ncons) {
+      const int col = v * VEC;
+      const long long e = e0 + col;
+      if (e >= hi || e + VEC <= lo) continue;
+      const bool whole = e >= lo && e + VEC <= hi;
+      float a[VEC], t[VEC];
+      ThetaTraits<TH>::lds_quad(sth + col, a);
+      if (!due) {                                         // not this round: carry theta over
+        if (whole) {
+          ThetaTraits<TH>::stg_quad(out + e, a);
+        } else {
+          for (int x = 0; x < VEC; ++x)
+            if (e + x >= lo && e + x < hi) out[e + x] = ThetaTraits<TH>::narrow(a[x]);
+        }
+        continue;
+      }
+      for (int j = 1; j <= q; ++j) {                      // neighbours in draw order
+        ThetaTraits<TH>::lds_quad(sth + (size_t)j * T + col, t);
+#pragma unroll
+        for (int x = 0; x < VEC; ++x) a[x] = __fadd_rn(a[x], t[x]);
+      }
+#pragma unroll
+      for (int x = 0; x < VEC; ++x)
+        a[x] = P.inv_exact ? __fmul_rn(a[x], P.inv_qp1) : __fdiv_rn(a[x], P.qp1);
+      if (!bmuf) {
+        if (whole) {
+          ThetaTraits<TH>::stg_quad(out + e, a);
+        } else {
+          for (int x = 0; x < VEC; ++x)
+            if (e + x >= lo && e + x < hi) out[e + x] = ThetaTraits<TH>::narrow(a[x]);
+        }
+        continue;
+      }
+      const float4 W = *reinterpret_cast<const float4*>(som + col);
+      const float4 D = *reinterpret_cast<const float4*>(sde + col);
+      float wv[VEC] = {W.x, W.y, W.z, W.w}, dv[VEC] = {D.x, D.y, D.z, D.w};
+#pragma unroll
+      for (int x = 0; x < VEC; ++x) bmuf_filter<TH>(a[x], wv[x], dv[x], t[x], P.eta, P.zeta);
+      if (whole) {
+        __stcs(reinterpret_cast<float4*>(P.delta + e), make_float4(dv[0], dv[1], dv[2], dv[3]));
+        __stcs(reinterpret_cast<float4*>(P.omega + e), make_float4(wv[0], wv[1], wv[2], wv[3]));
+        ThetaTraits<TH>::stg_quad(out + e, t);
+      } else {
+        for (int x = 0; x < VEC; ++x) {
+          if (e + x >= lo && e + x < hi) {
+            P.delta[e + x] = dv[x];
+            P.omega[e + x] = wv[x];
+            out[e + x] = ThetaTraits<TH>::narrow(t[x]);
+          }
+        }
+      }
+    }
+    mbar_arrive(bars + 64 + 8 * s);
+  }
+}
+
+// =================================================================================================
 // Host side
 // =================================================================================================
 thread_local std::string g_create_error;
@@ -1796,6 +2023,244 @@ gbmuf_status gbmuf_sync_round_host(const gbmuf_config* cfg, void* theta, float* 
   if (st == GBMUF_OK && worst != 0)
     st = fail(nullptr, GBMUF_ERR_TIMEOUT, "a bounded device-side wait expired; the host arrays are unspecified");
   return st;
+}
+
+
+// -------------------------------------------------------------------------------------------------
+// One worker per GPU: gbmuf_peer_*
+// -------------------------------------------------------------------------------------------------
+}  // extern "C"
+
+struct gbmuf_peer {
+  gbmuf_config cfg;
+  int rank = 0;
+  void* theta_own[2] = {nullptr, nullptr};
+  float* omega = nullptr;
+  float* delta = nullptr;
+  const void** d_theta_in[2] = {nullptr, nullptr};   // device arrays [K] of row pointers
+  int m = 0;
+  bool partitioned = false;
+  std::vector<int64_t> off;
+  std::vector<int32_t> periods;
+  unsigned char* tables = nullptr;   // offsets | prefix | periods | mask | due | nbr
+  size_t t_prefix = 0, t_periods = 0, t_mask = 0, t_due = 0, t_nbr = 0;
+  int32_t* d_status = nullptr;
+  long long total_tiles = 0;
+  int num_sms = 0, max_smem = 0;
+  int T = 0, stages = 0, ncons = 0;
+  uint32_t stage_stride = 0, omega_off = 0, delta_off = 0, desc_off = 0, smem = 0;
+};
+
+extern "C" {
+
+gbmuf_status gbmuf_peer_create(const gbmuf_config* cfg, int32_t rank, void* const* theta_bufs,
+                               float* omega, float* delta, gbmuf_peer** out) {
+  if (!cfg || !out || !theta_bufs) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "cfg, theta_bufs and out must not be NULL");
+  if (cfg->K < 1 || cfg->K > 65535 || rank < 0 || rank >= cfg->K)
+    return fail(nullptr, GBMUF_ERR_INVALID_ARG, "K must be in 1..65535 and 0 <= rank < K");
+  if (cfg->N < 1 || cfg->ld < cfg->N || cfg->ld % 32 != 0 || cfg->p < 0 || cfg->q < 0 || cfg->comp_base < 0 ||
+      (cfg->mode != GBMUF_MODE_BMUF && cfg->mode != GBMUF_MODE_MA) ||
+      (cfg->theta_dtype != GBMUF_F32 && cfg->theta_dtype != GBMUF_BF16) ||
+      !(cfg->eta == cfg->eta) || !(cfg->zeta == cfg->zeta) || cfg->device < 0)
+    return fail(nullptr, GBMUF_ERR_INVALID_ARG, "configuration out of range (see gbmuf_create)");
+  const int cand = host_candidates(cfg->K, cfg->p);
+  if (cfg->q > cand) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "q exceeds the ring neighbours min(2p, K-1)");
+  if (cand > kMaxCand) return fail(nullptr, GBMUF_ERR_UNSUPPORTED, "more than 64 ring neighbours per worker");
+  if (cfg->q > 15) return fail(nullptr, GBMUF_ERR_UNSUPPORTED, "more than 15 neighbours per draw in the peer form");
+  if (!omega || !delta || (((uintptr_t)omega | (uintptr_t)delta) % 128) != 0)
+    return fail(nullptr, GBMUF_ERR_INVALID_ARG, "omega and delta must be 128-byte aligned device pointers");
+  for (int b = 0; b < 2; ++b)
+    for (int j = 0; j < cfg->K; ++j) {
+      const void* ptr = theta_bufs[(size_t)b * cfg->K + j];
+      if (!ptr || (uintptr_t)ptr % 128 != 0)
+        return fail(nullptr, GBMUF_ERR_INVALID_ARG, "every theta buffer pointer must be non-NULL and 128-byte aligned");
+    }
+  if (theta_bufs[rank] == theta_bufs[(size_t)cfg->K + rank])
+    return fail(nullptr, GBMUF_ERR_INVALID_ARG, "the worker's two theta buffers must be different");
+  int ndev = 0;
+  cudaError_t e = cudaGetDeviceCount(&ndev);
+  if (e != cudaSuccess) return cuda_fail(nullptr, "cudaGetDeviceCount", e);
+  if (cfg->device >= ndev) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "no such CUDA device");
+  DeviceGuard guard(cfg->device);
+  if (!guard.ok) return fail(nullptr, GBMUF_ERR_CUDA, "cudaSetDevice failed");
+  gbmuf_peer* h = new (std::nothrow) gbmuf_peer();
+  if (!h) return fail(nullptr, GBMUF_ERR_ALLOC, "out of host memory");
+  h->cfg = *cfg; h->rank = rank; h->omega = omega; h->delta = delta;
+  h->theta_own[0] = theta_bufs[rank];
+  h->theta_own[1] = theta_bufs[(size_t)cfg->K + rank];
+  int v = 0;
+  cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, cfg->device); h->num_sms = v;
+  cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerBlockOptin, cfg->device); h->max_smem = v;
+  // launch shape: the widest power-of-two tile whose stage ((q+1) theta rows + omega + Delta)
+  // stays under 56 KB, so that four stages fit
+  const int esz = cfg->theta_dtype == GBMUF_F32 ? 4 : 2;
+  const bool bmuf = cfg->mode == GBMUF_MODE_BMUF;
+  auto stage_bytes = [&](int T) {
+    long long at = ((long long)(cfg->q + 1) * T * esz + 127) / 128 * 128;
+    h->omega_off = (uint32_t)at;
+    if (bmuf) at += (long long)T * 4;
+    h->delta_off = (uint32_t)at;
+    if (bmuf) at += (long long)T * 4;
+    h->desc_off = (uint32_t)at;
+    at += (long long)sizeof(TileDesc);
+    return (at + 127) / 128 * 128;
+  };
+  int T = 4096;
+  while (T > 64 && stage_bytes(T) > 56 * 1024) T >>= 1;
+  h->T = T;
+  h->stage_stride = (uint32_t)stage_bytes(T);
+  h->stages = (int)((h->max_smem - 128) / h->stage_stride);
+  if (h->stages > 4) h->stages = 4;
+  if (h->stages < 1) { delete h; return fail(nullptr, GBMUF_ERR_UNSUPPORTED, "a stage does not fit shared memory"); }
+  h->smem = 128 + (uint32_t)h->stages * h->stage_stride;
+  int n = (T / 4 + 31) / 32 * 32;
+  h->ncons = n < 128 ? 128 : n > 992 ? 992 : n;
+  e = cudaMalloc(&h->d_status, sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaMemset(h->d_status, 0, sizeof(int32_t));
+  for (int b = 0; b < 2 && e == cudaSuccess; ++b) {
+    e = cudaMalloc(&h->d_theta_in[b], (size_t)cfg->K * sizeof(void*));
+    if (e == cudaSuccess)
+      e = cudaMemcpy(h->d_theta_in[b], theta_bufs + (size_t)b * cfg->K, (size_t)cfg->K * sizeof(void*),
+                     cudaMemcpyHostToDevice);
+  }
+  if (e != cudaSuccess) {
+    cudaFree(h->d_status); cudaFree(h->d_theta_in[0]); cudaFree(h->d_theta_in[1]);
+    delete h;
+    return e == cudaErrorMemoryAllocation ? fail(nullptr, GBMUF_ERR_ALLOC, "peer pointer tables")
+                                          : cuda_fail(nullptr, "peer context set-up", e);
+  }
+  *out = h;
+  return GBMUF_OK;
+}
+
+gbmuf_status gbmuf_peer_set_partition(gbmuf_peer* h, int32_t m, const int64_t* offsets,
+                                      const int32_t* periods) {
+  if (!h) return GBMUF_ERR_INVALID_ARG;
+  if (m < 1 || m > 65536 || !offsets) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "m must be in 1..65536 and offsets not NULL");
+  if (offsets[0] != 0 || offsets[m] != h->cfg.N)
+    return fail(nullptr, GBMUF_ERR_INVALID_ARG, "offsets[0] must be 0 and offsets[m] must be N");
+  for (int i = 0; i < m; ++i) {
+    if (offsets[i + 1] <= offsets[i]) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "offsets must be strictly increasing");
+    if (periods && periods[i] < 1) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "periods must be >= 1");
+  }
+  DeviceGuard guard(h->cfg.device);
+  if (!guard.ok) return fail(nullptr, GBMUF_ERR_CUDA, "cudaSetDevice failed");
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return cuda_fail(nullptr, "cudaDeviceSynchronize", e);
+  cudaFree(h->tables);
+  h->tables = nullptr;
+  h->partitioned = false;
+  h->m = m;
+  h->off.assign(offsets, offsets + m + 1);
+  if (periods) h->periods.assign(periods, periods + m); else h->periods.assign(m, 1);
+  std::vector<int32_t> prefix((size_t)m + 1);
+  long long total = 0;
+  for (int i = 0; i < m; ++i) {              // every component has tiles: idle ones are copied through
+    prefix[i] = (int32_t)total;
+    const int64_t start = offsets[i] & ~(int64_t)(kAlign - 1);
+    total += (offsets[i + 1] - start + h->T - 1) / h->T;
+    if (total > 0x3fffffffLL) return fail(nullptr, GBMUF_ERR_UNSUPPORTED, "more than 2^30 - 1 tiles");
+  }
+  prefix[m] = (int32_t)total;
+  h->total_tiles = total;
+  auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+  h->t_prefix = up((size_t)(m + 1) * 8);
+  h->t_periods = h->t_prefix + up((size_t)(m + 1) * 4);
+  h->t_mask = h->t_periods + up((size_t)m * 4);
+  h->t_due = h->t_mask + up((size_t)m);
+  h->t_nbr = h->t_due + up((size_t)m);
+  const size_t bytes = h->t_nbr + up((size_t)m * (h->cfg.q > 0 ? h->cfg.q : 1) * 4);
+  e = cudaMalloc(&h->tables, bytes);
+  if (e == cudaSuccess) e = cudaMemcpy(h->tables, h->off.data(), (size_t)(m + 1) * 8, cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaMemcpy(h->tables + h->t_prefix, prefix.data(), (size_t)(m + 1) * 4, cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaMemcpy(h->tables + h->t_periods, h->periods.data(), (size_t)m * 4, cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) {
+    cudaFree(h->tables);
+    h->tables = nullptr;
+    return e == cudaErrorMemoryAllocation ? fail(nullptr, GBMUF_ERR_ALLOC, "partition tables") : cuda_fail(nullptr, "partition upload", e);
+  }
+  h->partitioned = true;
+  return GBMUF_OK;
+}
+
+gbmuf_status gbmuf_peer_sync_round(gbmuf_peer* h, uint64_t round, const uint8_t* comp_mask,
+                                   int32_t read_buffer, void* stream) {
+  if (!h) return GBMUF_ERR_INVALID_ARG;
+  if (!h->partitioned) return fail(nullptr, GBMUF_ERR_BAD_STATE, "gbmuf_peer_set_partition has not been called");
+  if (read_buffer != 0 && read_buffer != 1) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "read_buffer must be 0 or 1");
+  DeviceGuard guard(h->cfg.device);
+  if (!guard.ok) return fail(nullptr, GBMUF_ERR_CUDA, "cudaSetDevice failed");
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaError_t e;
+  if (comp_mask) {
+    e = cudaMemcpyAsync(h->tables + h->t_mask, comp_mask, (size_t)h->m, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(nullptr, "upload of the component mask", e);
+  }
+  PeerPlanParams Q;
+  Q.K = h->cfg.K; Q.m = h->m; Q.p = h->cfg.p; Q.q = h->cfg.q; Q.comp_base = h->cfg.comp_base;
+  Q.rank = h->rank; Q.use_mask = comp_mask ? 1 : 0; Q.seed = h->cfg.seed; Q.round = round;
+  Q.periods = reinterpret_cast<const int32_t*>(h->tables + h->t_periods);
+  Q.mask = h->tables + h->t_mask;
+  Q.nbr = reinterpret_cast<int32_t*>(h->tables + h->t_nbr);
+  Q.due = h->tables + h->t_due;
+  peer_plan_kernel<<<(h->m + 255) / 256, 256, 0, st>>>(Q);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(nullptr, "launch of the peer plan kernel", e);
+  PeerParams P;
+  P.theta_in = h->d_theta_in[read_buffer];
+  P.theta_out = h->theta_own[1 - read_buffer];
+  P.omega = h->omega; P.delta = h->delta;
+  P.off = reinterpret_cast<const int64_t*>(h->tables);
+  P.tile_prefix = reinterpret_cast<const int32_t*>(h->tables + h->t_prefix);
+  P.nbr = Q.nbr; P.due = Q.due; P.status = h->d_status;
+  P.N = h->cfg.N; P.rank = h->rank; P.m = h->m; P.q = h->cfg.q; P.mode = h->cfg.mode;
+  P.eta = h->cfg.eta; P.zeta = h->cfg.zeta;
+  const int qp1 = h->cfg.q + 1;
+  P.qp1 = (float)qp1; P.inv_qp1 = 1.0f / (float)qp1; P.inv_exact = (qp1 & (qp1 - 1)) == 0;
+  P.T = h->T; P.stages = h->stages; P.ncons = h->ncons;
+  P.stage_stride = h->stage_stride; P.omega_off = h->omega_off; P.delta_off = h->delta_off;
+  P.desc_off = h->desc_off;
+  const int grid = (int)(h->total_tiles < h->num_sms ? h->total_tiles : h->num_sms);
+  if (h->cfg.theta_dtype == GBMUF_F32) {
+    e = cudaFuncSetAttribute(peer_round_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, h->max_smem);
+    if (e == cudaSuccess) peer_round_kernel<float><<<grid, 32 + h->ncons, h->smem, st>>>(P);
+  } else {
+    e = cudaFuncSetAttribute(peer_round_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, h->max_smem);
+    if (e == cudaSuccess) peer_round_kernel<__nv_bfloat16><<<grid, 32 + h->ncons, h->smem, st>>>(P);
+  }
+  if (e == cudaSuccess) e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(nullptr, "launch of the peer round kernel", e);
+  return GBMUF_OK;
+}
+
+gbmuf_status gbmuf_peer_device_status(gbmuf_peer* h, void* stream, int32_t* out) {
+  if (!h || !out) return GBMUF_ERR_INVALID_ARG;
+  DeviceGuard guard(h->cfg.device);
+  if (!guard.ok) return fail(nullptr, GBMUF_ERR_CUDA, "cudaSetDevice failed");
+  cudaStream_t st = (cudaStream_t)stream;
+  int32_t v = 0;
+  cudaError_t e = cudaMemcpyAsync(&v, h->d_status, sizeof(v), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(h->d_status, 0, sizeof(v), st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return cuda_fail(nullptr, "read of the device status word", e);
+  *out = v;
+  return GBMUF_OK;
+}
+
+gbmuf_status gbmuf_peer_destroy(gbmuf_peer* h) {
+  if (!h) return GBMUF_OK;
+  gbmuf_status rc = GBMUF_OK;
+  {
+    DeviceGuard guard(h->cfg.device);
+    if (guard.ok) {
+      if (cudaDeviceSynchronize() != cudaSuccess) rc = GBMUF_ERR_CUDA;
+      cudaFree(h->tables); cudaFree(h->d_status); cudaFree(h->d_theta_in[0]); cudaFree(h->d_theta_in[1]);
+    } else {
+      rc = GBMUF_ERR_CUDA;
+    }
+  }
+  delete h;
+  return rc;
 }
 
 }  // extern "C"
