@@ -36,8 +36,8 @@ FALLBACK_HBM_GBS = 6650.0
 # + dram__bytes_write.sum divided by the replica-parameters of the captured launch; key = theta
 # dtype: 0 fp32 from workload profile16, 1 bf16 from profile16bf), valid only
 # for the kernel source it was taken from (source_sha() below).
-NCU_TRAFFIC = {"source_sha": "ca6a56ca1eb2", "bytes_per_replica_param": {0: 6.382624e9 / 268435536,
-                                                                   1: 5.309772e9 / 268435536}}
+NCU_TRAFFIC = {"source_sha": "9b5ad4df2841", "bytes_per_replica_param": {0: 6.383138e9 / 268435536,
+                                                                   1: 5.309694e9 / 268435536}}
 
 
 def algorithmic_bytes_per_replica_param(dtype: int, mode: int = 0) -> int:

@@ -159,7 +159,7 @@ gbmuf_status gbmuf_selftest_wait_timeout(gbmuf_ctx* ctx, void* stream, double* s
 /* Launch shape of the fused kernel (one persistent CTA per SM).  Any argument may be 0 to keep
  * the built-in choice.  consumer_threads: multiple of 32 in 32..992 (one more warp issues the
  * copies); tile_elems: elements of one component staged per work item for all K workers, a
- * multiple of 8 and, above 256, of 256; theta_stages: 1 or 2 tiles of theta resident per CTA;
+ * multiple of 8 and, above 256, of 256; theta_stages: 1..4 tiles of theta resident per CTA;
  * ring_slots: 2..8 rows of omega/Delta in flight; flags: bit 0 = 256-byte L2 promotion for the
  * theta loads (default 128).
  * Errors: INVALID_ARG, UNSUPPORTED (does not fit shared memory). */

@@ -321,7 +321,8 @@ struct TileDesc {
 
 constexpr int kMaxRing = 8;
 // barrier block at the start of shared memory (8 bytes each)
-constexpr uint32_t kBarThetaFull = 0, kBarThetaEmpty = 16, kBarRingFull = 32, kBarRingEmpty = 96;
+constexpr uint32_t kBarThetaFull = 0, kBarThetaEmpty = 32, kBarRingFull = 64, kBarRingEmpty = 128;
+constexpr int kMaxThetaStages = 4;
 constexpr uint32_t kBarBytes = 256;
 
 struct SyncParams {
@@ -338,7 +339,7 @@ struct SyncParams {
   int inv_exact;        // q+1 is a power of two: multiplying by 1/(q+1) equals dividing
   int T, BW, bw_shift, bw_mask;   // BW: columns per TMA box; column c of a tile is in box
                                   // c >> bw_shift at c & bw_mask
-  int stages, ring, ncons;        // theta stages (1 or 2), ring slots, consumer threads
+  int stages, ring, ncons;        // theta stages (1..4), ring slots, consumer threads
   uint32_t stage_stride, nbr_off, desc_off;   // theta stage: [theta boxes | nbr | desc]
   uint32_t ring_off, slot_stride;             // ring slot: [omega row T floats | Delta row T floats]
 };
@@ -506,6 +507,45 @@ sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_th
     const int* snb = reinterpret_cast<const int*>(st + P.nbr_off);
     const TileDesc* d = reinterpret_cast<const TileDesc*>(st + P.desc_off);
     const long long e0 = d->e0, lo = d->lo, hi = d->hi;
+    if (!bmuf) {
+      // gossip-MA: theta <- average.  No omega / Delta stream paces the workers, so each thread
+      // walks all workers for its group of elements; unrolled so that the shared-memory loads
+      // and divides of several workers overlap.
+      // With more threads than element groups the workers are split between thread groups:
+      // thread c takes group c % nv for workers c / nv, c / nv + kg, ...
+      const int kg = P.ncons > nv ? P.ncons / nv : 1;
+      const int k_first = P.ncons > nv ? c / nv : 0;
+      for (int v = P.ncons > nv ? c - k_first * nv : c; v < nv && k_first < kg; v += P.ncons) {
+        const int col = v * VEC;
+        const long long e = e0 + col;
+        if (e >= hi || e + VEC <= lo) continue;
+        const int b = col >> P.bw_shift, cin = col & P.bw_mask;
+        const int boxbase = b * box_elems + cin;
+        const bool whole = e >= lo && e + VEC <= hi;
+#pragma unroll 4
+        for (int k = k_first; k < P.K; k += kg) {
+          float a[VEC], t[VEC];
+          ThetaTraits<TH>::lds_quad(sth + boxbase + k * BW, a);
+          for (int j = 0; j < q; ++j) {
+            ThetaTraits<TH>::lds_quad(sth + boxbase + snb[k * q + j] * BW, t);
+#pragma unroll
+            for (int x = 0; x < VEC; ++x) a[x] = __fadd_rn(a[x], t[x]);
+          }
+#pragma unroll
+          for (int x = 0; x < VEC; ++x)
+            a[x] = P.inv_exact ? __fmul_rn(a[x], P.inv_qp1) : __fdiv_rn(a[x], P.qp1);
+          const long long at = (long long)k * P.ld + e;
+          if (whole) {
+            ThetaTraits<TH>::stg_quad(theta + at, a);
+          } else {
+            for (int x = 0; x < VEC; ++x)
+              if (e + x >= lo && e + x < hi) theta[at + x] = ThetaTraits<TH>::narrow(a[x]);
+          }
+        }
+      }
+      mbar_arrive(bars + kBarThetaEmpty + 8 * s);
+      continue;
+    }
     for (int k = 0; k < P.K; ++k) {
       const float* som = nullptr;
       const float* sde = nullptr;
@@ -1196,7 +1236,8 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
   auto total_bytes = [&](int T, int S, int R) {
     return (long long)kBarBytes + S * stage_bytes(T, nullptr) + (bmuf ? (long long)R * 2 * T * 4 : 0);
   };
-  const int want_stages = t.stages ? t.stages : 1;
+  // gossip-MA stages only theta, so it can afford (and needs) a second stage to overlap
+  int want_stages = t.stages ? t.stages : (bmuf ? 1 : 2);
   auto ring_for = [&](int T) {   // slots used with tile T: the caller's, else as many as fit up to 4
     if (!bmuf) return 0;
     if (t.ring) return t.ring;
@@ -1206,6 +1247,7 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
   };
   if (t.T) {
     L.T = t.T;
+    if (!t.stages && want_stages > 1 && total_bytes(L.T, want_stages, ring_for(L.T)) > cap) want_stages = 1;
   } else {
     // The widest power-of-two tile (longest contiguous run per row) that fits: measured DRAM
     // efficiency keeps growing with the run length up to 16 KB, and a tile that is a whole
@@ -1220,7 +1262,7 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
   if (L.T > 256 && L.T % 256 != 0)
     return fail(ctx, GBMUF_ERR_INVALID_ARG, "tile_elems above 256 must be a multiple of 256");
   L.BW = L.T < 256 ? L.T : 256;                // a tensor-map box is at most 256 elements wide
-  L.stages = t.stages ? t.stages : 1;
+  L.stages = want_stages;
   if ((long long)K * L.T * esz >= (1 << 20) || total_bytes(L.T, L.stages, L.ring) > cap)
     return fail(ctx, GBMUF_ERR_UNSUPPORTED,
                 "the theta stage(s) (K rows of the tile) and the omega/Delta ring do not fit the "
@@ -1235,6 +1277,8 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
   } else {
     int n = (L.T / 4 + 31) / 32 * 32;          // one quad per thread and row, within 128..992
     L.ncons = n < 128 ? 128 : n > 992 ? 992 : n;
+    if (!bmuf && L.T / 4 >= 32 && L.T / 4 <= 496)
+      L.ncons = (L.T / 4) * (992 / (L.T / 4));  // gossip-MA: thread groups share out the workers
   }
   *out = L;
   return GBMUF_OK;
@@ -1436,7 +1480,7 @@ gbmuf_status gbmuf_set_tuning(gbmuf_ctx* ctx, int32_t ncons, int32_t tile_elems,
                               int32_t ring, int32_t flags) {
   if (!ctx) return GBMUF_ERR_INVALID_ARG;
   if (ncons < 0 || ncons > 992 || ncons % 32 != 0 || tile_elems < 0 || tile_elems > (1 << 16) ||
-      stages < 0 || stages > 2 || ring < 0 || ring > kMaxRing || ring == 1 || flags < 0 || flags > 1)
+      stages < 0 || stages > kMaxThetaStages || ring < 0 || ring > kMaxRing || ring == 1 || flags < 0 || flags > 1)
     return fail(ctx, GBMUF_ERR_INVALID_ARG, "tuning value out of range");
   Tuning t;
   t.ncons = ncons; t.T = tile_elems; t.stages = stages; t.ring = ring; t.flags = flags;
