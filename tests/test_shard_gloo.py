@@ -1,6 +1,6 @@
 """The multi-GPU plan on CPU: the path shards by column range with no data exchange.  Two gloo
 ranks each take their share from the shard planner, run the round on it alone (here with the
-oracle, the GPU library being out of reach on a CPU machine), and the pieces must reassemble to the
+oracle, since these ranks have no GPU), and the pieces must reassemble to the
 unsharded result; the timing reduction the bench uses is the max over ranks."""
 import os
 import socket
