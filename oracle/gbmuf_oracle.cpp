@@ -127,7 +127,7 @@ int gbo_candidate_list(int k, int K, int p, int32_t* out) {
   return candidate_list(k, K, p, out);
 }
 
-// Algorithm 1, "randomly choose q neighbors k_1..k_q": an independent uniform draw of q
+// Algorithm 1, the neighbour-choice line (k_1..k_q): an independent uniform draw of q
 // distinct nodes out of worker k's ring neighbours for every (round, worker k, component i).
 // Partial Fisher-Yates over the candidate list; the j-th swap index uses one 32-bit Philox
 // word reduced to [0, c-j) by multiply-shift.

@@ -57,7 +57,7 @@ constexpr int kMaxCand = 64;                   // largest candidate set min(2p, 
 constexpr int kAlign = 8;                      // tiles start on multiples of 8 elements (>= 16 B)
 
 // =================================================================================================
-// Round set-up: neighbour draws (Algorithm 1: "randomly choose q neighbors k_1..k_q") and the
+// Round set-up: neighbour draws (Algorithm 1, the neighbour-choice line: k_1..k_q) and the
 // work-list of this round.
 // =================================================================================================
 struct SetupParams {

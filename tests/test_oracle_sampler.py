@@ -1,5 +1,5 @@
 """Pins of the oracle's ring topology (Definition 1) and neighbour sampler (Algorithm 1,
-"randomly choose q neighbors")."""
+the neighbour-choice line)."""
 import itertools
 
 import numpy as np
