@@ -205,6 +205,19 @@ def run_gpu(args, w):
     del theta0
     lr, sigma = w.lr or 0.1, w.sigma or 1e-3
     g.local_perturb(0, lr, sigma, 1)
+    if args.local_step == "adagrad":
+        # the experiments' optimiser on a fixed synthetic gradient (std 1e-2); the recurrent
+        # components (here: those of 1 Mi to 8 Mi elements) form the clipped group
+        grad = torch.empty((K, ld), dtype=torch.float32, device=dev).normal_(0.0, 1e-2)
+        accum = torch.full((K, ld), 0.1, dtype=torch.float32, device=dev)
+        sizes = [w.offsets[i + 1] - w.offsets[i] for i in range(w.m)]
+        clip_mask = [1 if n <= (1 << 23) and n >= (1 << 20) else 0 for n in sizes]
+
+        def local_step(step):
+            g.local_adagrad(grad, accum, lr, eps=1e-8, clip_norm=10.0, clip_mask=clip_mask)
+    else:
+        def local_step(step):
+            g.local_perturb(step, lr, sigma, 1)
     torch.cuda.synchronize()
     info = g.launch_info()
 
@@ -217,7 +230,7 @@ def run_gpu(args, w):
            torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     rnd = 1
     for _ in range(args.warmup):
-        g.local_perturb(rnd, lr, sigma, 1)
+        local_step(rnd)
         g.sync_round(rnd)
         rnd += 1
     barrier()
@@ -228,7 +241,7 @@ def run_gpu(args, w):
     for i in range(args.steps):
         a, b, c = ev[i]
         a.record()
-        g.local_perturb(rnd, lr, sigma, 1)      # the synthetic local step: outside the timed interval
+        local_step(rnd)                         # the local step: outside the timed interval
         b.record()
         g.sync_round(rnd)                       # set-up kernel + fused kernel
         c.record()
@@ -302,7 +315,8 @@ def run_gpu(args, w):
                            "parallelism": f"element-range shards x{world}, no collective",
                            "l2": "inputs_larger_than_l2 (state %.1f GB per GPU)" %
                                  ((K * ld * (8 + (4 if w.dtype == 0 else 2))) / 1e9),
-                           "launch": info, "local_step_ms": sum(pert_ms) / len(pert_ms),
+                           "launch": info, "local_step": args.local_step,
+                           "local_step_ms": sum(pert_ms) / len(pert_ms),
                            "round_plus_local_step_ms": (sum(pert_ms) + sum(sync_ms)) / len(sync_ms),
                            "sync_ms_min": min(sync_ms), "sync_ms_max": max(sync_ms),
                            "device_status": status},
@@ -311,7 +325,8 @@ def run_gpu(args, w):
                              "frac_of_nominal_8TBs": achieved / 8000.0,
                              "algorithmic_bytes_per_replica_param": bpe, "traffic": traffic,
                              "kernel": "sync_fused_kernel"},
-                "clocks": clocks, "gpu_launches": 3 * args.steps, "e2e": e2e}
+                "clocks": clocks,
+                "gpu_launches": (3 if args.local_step == "perturb" else 5) * args.steps, "e2e": e2e}
         if not args.no_cpu_baseline and world == 1:
             times, units_cpu = time_oracle_rounds(w, args.ref_cols, 3)
             t = sum(times) / len(times)
@@ -337,6 +352,8 @@ def main():
     ap.add_argument("--tuning", default="", help="consumer_threads,tile_elems,theta_stages,ring_slots,flags")
     ap.add_argument("--ref-cols", type=int, default=1 << 23,
                     help="columns of the workload the CPU oracle is timed on")
+    ap.add_argument("--local-step", default="perturb", choices=["perturb", "adagrad"],
+                    help="what moves the replicas between rounds (launched outside the timed interval)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-cols", type=int, default=1 << 27,
