@@ -161,7 +161,8 @@ gbmuf_status gbmuf_selftest_wait_timeout(gbmuf_ctx* ctx, void* stream, double* s
  * copies); tile_elems: elements of one component staged per work item for all K workers, a
  * multiple of 8 and, above 256, of 256; theta_stages: 1..4 tiles of theta resident per CTA;
  * ring_slots: 2..8 rows of omega/Delta in flight; flags: bit 0 = 256-byte L2 promotion for the
- * theta loads (default 128).
+ * theta loads (default 128); bit 1 = keep the theta tile in tensor memory (fp32 theta,
+ * gossip-BMUF mode, 4 <= K <= 128; tile_elems then a multiple of 512 with K * tile_elems / 128 <= 512).
  * Errors: INVALID_ARG, UNSUPPORTED (does not fit shared memory). */
 gbmuf_status gbmuf_set_tuning(gbmuf_ctx* ctx, int32_t consumer_threads, int32_t tile_elems,
                               int32_t theta_stages, int32_t ring_slots, int32_t flags);

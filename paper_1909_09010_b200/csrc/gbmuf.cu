@@ -614,6 +614,254 @@ sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_th
   }
 }
 
+// =================================================================================================
+// Variant of the fused round that keeps the theta tile in tensor memory (TMEM) instead of shared
+// memory (fp32 theta, gossip-BMUF mode).  A K x T fp32 tile of up to 256 KB does not fit shared
+// memory next to anything else, but it is exactly what the 512 columns x 128 lanes of an SM's
+// tensor memory hold.  Every row of theta, omega and Delta streams through one ring of
+// shared-memory slots (two rows of T floats per slot): first the K theta rows of a tile, which
+// each consumer thread moves from the slot into its own TMEM cells (tcgen05.st), then, worker by
+// worker, omega and Delta, for which the thread reads its own and the drawn neighbours' theta
+// back from those cells (tcgen05.ld).  A thread only ever reads cells it wrote itself, so TMEM
+// needs no synchronisation between threads, and the run per row can be twice as long as with a
+// shared-memory tile.
+//
+// TMEM addressing: a warp reaches the 32 lanes 32 * (warp id % 4) ..; with the .32x32b.x4 shape
+// each thread moves the 4 consecutive 32-bit columns of its lane that start at the given column.
+// Element group g (4 elements) of a tile lives in lane g % 128, columns ((g / 128) * K + row) * 4.
+// The allocation is released by the warp that made it after every thread has reached the end of
+// the kernel; no path returns early.
+// =================================================================================================
+struct TmemParams {
+  const float* theta_in;   // same array as theta (read side)
+  float* theta;
+  float* omega;
+  float* delta;
+  const int64_t* off;
+  const int32_t* tile_prefix;
+  const int32_t* nbr;      // [m][K][q]
+  int32_t* status;
+  long long ld;
+  int K, m, q;
+  float eta, zeta, qp1, inv_qp1;
+  int inv_exact;
+  int T, ring, ncols;      // T multiple of 512; ring slots of 2*T floats; TMEM columns (power of 2)
+  uint32_t ring_off, meta_off, meta_stride;   // meta ring (4 entries): [TileDesc | nbr K*q ints]
+};
+
+__device__ __forceinline__ void tmem_store4(uint32_t taddr, const float (&x)[4]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};" ::"r"(taddr),
+               "r"(__float_as_uint(x[0])), "r"(__float_as_uint(x[1])), "r"(__float_as_uint(x[2])),
+               "r"(__float_as_uint(x[3]))
+               : "memory");
+}
+__device__ __forceinline__ void tmem_load4(uint32_t taddr, float (&x)[4]) {
+  uint32_t a, b, c, d;
+  // load and wait in one statement: the registers are only valid after the wait, and nothing may
+  // be scheduled between the two
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];\n\t"
+      "tcgen05.wait::ld.sync.aligned;"
+      : "=r"(a), "=r"(b), "=r"(c), "=r"(d)
+      : "r"(taddr)
+      : "memory");
+  x[0] = __uint_as_float(a); x[1] = __uint_as_float(b); x[2] = __uint_as_float(c); x[3] = __uint_as_float(d);
+}
+
+__global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParams P) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  // [0,64) ring full, [64,128) ring empty, [128,132) TMEM base address
+  const uint32_t bars = smem_u32(smem);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 128);
+  unsigned char* ring0 = smem + P.ring_off;
+  unsigned char* meta0 = smem + P.meta_off;
+  const int total = P.tile_prefix[P.m];
+  const int R = P.ring, K = P.K, q = P.q, T = P.T;
+  const int my_tiles = (int)blockIdx.x < total ? (total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+  const int ntheta = (K + 1) / 2;           // theta items per tile (two rows each)
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int r = 0; r < R; ++r) {
+      mbar_init(bars + 8 * r, 1);
+      mbar_init(bars + 64 + 8 * r, 512);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"((uint32_t)P.ncols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer warp
+    int comp = 0, pfx_lo = 0, pfx_hi = 0;
+    long long cb = 0, ce = 0;
+    if (my_tiles > 0) {
+      int lo_i = 0, hi_i = P.m;
+      while (hi_i - lo_i > 1) {
+        const int mid = (lo_i + hi_i) >> 1;
+        if (__ldg(P.tile_prefix + mid) <= (int)blockIdx.x) lo_i = mid; else hi_i = mid;
+      }
+      comp = lo_i;
+      pfx_lo = __ldg(P.tile_prefix + comp);
+      pfx_hi = __ldg(P.tile_prefix + comp + 1);
+      cb = __ldg(P.off + comp);
+      ce = __ldg(P.off + comp + 1);
+    }
+    int gi = 0;              // ring items requested so far
+    bool ok = true;
+    for (int it = 0; it < my_tiles && ok; ++it) {
+      const int w = (int)blockIdx.x + it * (int)gridDim.x;
+      if (w >= pfx_hi) {
+        while (w >= pfx_hi) {
+          ++comp;
+          pfx_lo = pfx_hi;
+          pfx_hi = __ldg(P.tile_prefix + comp + 1);
+        }
+        cb = __ldg(P.off + comp);
+        ce = __ldg(P.off + comp + 1);
+      }
+      const long long e0 = (cb & ~(long long)(kAlign - 1)) + (long long)(w - pfx_lo) * T;
+      long long run = P.ld - e0;
+      if (run > T) run = T;
+      const uint32_t bytes = (uint32_t)run * 4u;
+      // tile descriptor + neighbour table into the meta ring (4 entries: the consumers are never
+      // more than a ring of items, i.e. less than one tile, behind)
+      unsigned char* meta = meta0 + (size_t)(it & 3) * P.meta_stride;
+      TileDesc* d = reinterpret_cast<TileDesc*>(meta);
+      int* snb = reinterpret_cast<int*>(meta + sizeof(TileDesc));
+      if (d->comp != comp || it < 4) {
+        const int32_t* gnb = P.nbr + (size_t)comp * K * q;
+        for (int x = lane; x < K * q; x += 32) snb[x] = __ldg(gnb + x);
+      }
+      __syncwarp();
+      if (lane == 0) {
+        d->e0 = e0;
+        d->lo = cb > e0 ? cb : e0;
+        d->hi = ce < e0 + T ? ce : e0 + T;
+        d->comp = comp;
+      }
+      __syncwarp();
+      for (int item = 0; item < ntheta + K && ok; ++item, ++gi) {
+        const int slot = gi % R;
+        if (gi >= R) {
+          bool fine = mbar_wait_bounded(bars + 64 + 8 * slot, ((gi / R) - 1) & 1, P.status);
+          ok = __all_sync(0xffffffffu, fine);
+          if (!ok) break;
+        }
+        if (lane == 0) {
+          const uint32_t full = bars + 8 * slot;
+          const uint32_t dst = smem_u32(ring0 + (size_t)slot * (size_t)T * 8);
+          if (item < ntheta) {
+            const int r0 = 2 * item, rows = (r0 + 1 < K) ? 2 : 1;
+            mbar_arrive_expect_tx(full, (uint32_t)rows * bytes);
+            bulk_load_row(dst, P.theta_in + (long long)r0 * P.ld + e0, bytes, full);
+            if (rows == 2) bulk_load_row(dst + (uint32_t)T * 4u, P.theta_in + (long long)(r0 + 1) * P.ld + e0, bytes, full);
+          } else {
+            const long long at = (long long)(item - ntheta) * P.ld + e0;
+            mbar_arrive_expect_tx(full, 2u * bytes);
+            bulk_load_row(dst, P.omega + at, bytes, full);
+            bulk_load_row(dst + (uint32_t)T * 4u, P.delta + at, bytes, full);
+          }
+        }
+      }
+    }
+    if (!ok) {
+      for (int j = gi > R ? gi - R : 0; j < gi; ++j)
+        mbar_wait_bounded(bars + 8 * (j % R), (j / R) & 1, P.status);
+    }
+  } else {
+    // -------------------------------------------------------------------- consumer warps (16)
+    // lanes this warp reaches, and which of the four warps of that lane quarter it is
+    const int quarter = warp & 3, sub = (warp - 1) >> 2;
+    const uint32_t tlane = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    const int ngroups = T / 512;                  // element groups of 128 x 4 per row
+    int gi = 0;
+    bool ok = true;
+    for (int it = 0; it < my_tiles && ok; ++it) {
+      const unsigned char* meta = meta0 + (size_t)(it & 3) * P.meta_stride;
+      const TileDesc* d = reinterpret_cast<const TileDesc*>(meta);
+      const int* snb = reinterpret_cast<const int*>(meta + sizeof(TileDesc));
+      long long e0 = 0, lo = 0, hi = 0;
+      for (int item = 0; item < ntheta + K && ok; ++item, ++gi) {
+        const int slot = gi % R;
+        bool fine = mbar_wait_bounded(bars + 8 * slot, (gi / R) & 1, P.status);
+        ok = __all_sync(0xffffffffu, fine);
+        if (!ok) break;
+        if (item == 0) { e0 = d->e0; lo = d->lo; hi = d->hi; }
+        const float* row0 = reinterpret_cast<const float*>(ring0 + (size_t)slot * (size_t)T * 8);
+        const float* row1 = row0 + T;
+        if (item < ntheta) {
+          // deposit two theta rows into this thread's TMEM cells
+          const int r0 = 2 * item;
+          for (int g = sub; g < ngroups; g += 4) {
+            const int col = (g * 128 + quarter * 32 + lane) * 4;
+            float x[4];
+            ThetaTraits<float>::lds_quad(row0 + col, x);
+            tmem_store4(tlane + (uint32_t)((g * K + r0) * 4), x);
+            if (r0 + 1 < K) {
+              ThetaTraits<float>::lds_quad(row1 + col, x);
+              tmem_store4(tlane + (uint32_t)((g * K + r0 + 1) * 4), x);
+            }
+          }
+          asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        } else {
+          const int k = item - ntheta;
+          for (int g = sub; g < ngroups; g += 4) {
+            const int col = (g * 128 + quarter * 32 + lane) * 4;
+            const long long e = e0 + col;
+            float a[4], t[4];
+            tmem_load4(tlane + (uint32_t)((g * K + k) * 4), a);
+            for (int j = 0; j < q; ++j) {
+              tmem_load4(tlane + (uint32_t)((g * K + snb[k * q + j]) * 4), t);
+#pragma unroll
+              for (int x = 0; x < 4; ++x) a[x] = __fadd_rn(a[x], t[x]);
+            }
+            if (e >= hi || e + 4 <= lo) continue;
+#pragma unroll
+            for (int x = 0; x < 4; ++x)
+              a[x] = P.inv_exact ? __fmul_rn(a[x], P.inv_qp1) : __fdiv_rn(a[x], P.qp1);
+            const float4 W = *reinterpret_cast<const float4*>(row0 + col);
+            const float4 D = *reinterpret_cast<const float4*>(row1 + col);
+            float wv[4] = {W.x, W.y, W.z, W.w}, dv[4] = {D.x, D.y, D.z, D.w};
+#pragma unroll
+            for (int x = 0; x < 4; ++x) bmuf_filter<float>(a[x], wv[x], dv[x], t[x], P.eta, P.zeta);
+            const long long at = (long long)k * P.ld + e;
+            if (e >= lo && e + 4 <= hi) {
+              __stcs(reinterpret_cast<float4*>(P.delta + at), make_float4(dv[0], dv[1], dv[2], dv[3]));
+              __stcs(reinterpret_cast<float4*>(P.omega + at), make_float4(wv[0], wv[1], wv[2], wv[3]));
+              __stcs(reinterpret_cast<float4*>(P.theta + at), make_float4(t[0], t[1], t[2], t[3]));
+            } else {
+              for (int x = 0; x < 4; ++x) {
+                if (e + x >= lo && e + x < hi) {
+                  P.delta[at + x] = dv[x];
+                  P.omega[at + x] = wv[x];
+                  P.theta[at + x] = t[x];
+                }
+              }
+            }
+          }
+        }
+        mbar_arrive(bars + 64 + 8 * slot);
+      }
+    }
+  }
+  // every thread arrives here; only then is the tensor memory given back
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 0) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)P.ncols) : "memory");
+  }
+}
+
 // Self-test of the bounded wait: one warp waits on a barrier that nothing will ever signal.  The
 // wait must expire, set the status word and return; nothing here can hang or trap.
 __global__ void wait_timeout_selftest_kernel(int32_t* status, int32_t* returned) {
@@ -1115,6 +1363,8 @@ struct Tuning {
 struct Launch {
   int ncons, stages, ring, T, BW, flags;
   uint32_t stage_stride, nbr_off, desc_off, ring_off, slot_stride, smem;
+  int tmem_cols;                     // TMEM variant: columns to allocate (0 = shared-memory tile)
+  uint32_t meta_off, meta_stride;
 };
 
 int host_candidates(int K, int p) {
@@ -1224,7 +1474,34 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
   const bool bmuf = ctx->cfg.mode == GBMUF_MODE_BMUF;
   Launch L;
   L.flags = t.flags;
+  L.tmem_cols = 0; L.meta_off = 0; L.meta_stride = 0;
   const long long cap = ctx->max_smem < ctx->smem_per_sm - 1024 ? ctx->max_smem : ctx->smem_per_sm - 1024;
+  if (t.flags & 2) {
+    // theta tile in tensor memory: fp32 theta, gossip-BMUF, 4 <= K, K * (T/512) * 4 <= 512 columns
+    if (esz != 4 || !bmuf || K < 4 || K > 128)
+      return fail(ctx, GBMUF_ERR_UNSUPPORTED, "the tensor-memory variant needs fp32 theta, BMUF mode and 4 <= K <= 128");
+    int T = t.T ? t.T : 4096;
+    while (!t.T && T > 512 && (T / 512) * K * 4 > 512) T >>= 1;
+    if (T < 512 || T % 512 != 0 || (T / 512) * K * 4 > 512)
+      return fail(ctx, GBMUF_ERR_INVALID_ARG, "tensor-memory variant: tile_elems must be a multiple of 512 with K * tile_elems / 128 <= 512");
+    L.T = T; L.BW = 256; L.stages = 1; L.ncons = 512;
+    L.meta_off = 256;
+    L.meta_stride = (uint32_t)(((long long)sizeof(TileDesc) + (long long)K * q * 4 + 127) / 128 * 128);
+    L.ring_off = L.meta_off + 4 * L.meta_stride;
+    L.slot_stride = (uint32_t)(8 * T);
+    int R = t.ring ? t.ring : 6;
+    while (!t.ring && R > 2 && (long long)L.ring_off + (long long)R * L.slot_stride > cap) --R;
+    if ((long long)L.ring_off + (long long)R * L.slot_stride > cap || R < 2)
+      return fail(ctx, GBMUF_ERR_UNSUPPORTED, "tensor-memory variant: the ring does not fit shared memory");
+    L.ring = R;
+    L.smem = (uint32_t)(L.ring_off + (long long)R * L.slot_stride);
+    int cols = 32;
+    while (cols < (T / 512) * K * 4) cols <<= 1;
+    L.tmem_cols = cols;
+    L.stage_stride = 0; L.nbr_off = 0; L.desc_off = 0;
+    *out = L;
+    return GBMUF_OK;
+  }
   auto stage_bytes = [&](int T, Launch* l) {
     long long at = ((long long)K * T * esz + 15) / 16 * 16;
     if (l) l->nbr_off = (uint32_t)at;
@@ -1480,7 +1757,7 @@ gbmuf_status gbmuf_set_tuning(gbmuf_ctx* ctx, int32_t ncons, int32_t tile_elems,
                               int32_t ring, int32_t flags) {
   if (!ctx) return GBMUF_ERR_INVALID_ARG;
   if (ncons < 0 || ncons > 992 || ncons % 32 != 0 || tile_elems < 0 || tile_elems > (1 << 16) ||
-      stages < 0 || stages > kMaxThetaStages || ring < 0 || ring > kMaxRing || ring == 1 || flags < 0 || flags > 1)
+      stages < 0 || stages > kMaxThetaStages || ring < 0 || ring > kMaxRing || ring == 1 || flags < 0 || flags > 3)
     return fail(ctx, GBMUF_ERR_INVALID_ARG, "tuning value out of range");
   Tuning t;
   t.ncons = ncons; t.T = tile_elems; t.stages = stages; t.ring = ring; t.flags = flags;
@@ -1642,6 +1919,21 @@ gbmuf_status gbmuf_sync_round(gbmuf_ctx* ctx, uint64_t round, const uint8_t* com
                    ctx->d_prefix, ctx->d_nbr, ctx->d_status, &P);
   const long long cap = (long long)ctx->num_sms;              // one persistent CTA per SM
   const int grid = (int)(total < cap ? total : cap);
+  if (L.tmem_cols > 0) {
+    TmemParams Q;
+    Q.theta_in = (const float*)ctx->theta; Q.theta = (float*)ctx->theta; Q.omega = ctx->omega; Q.delta = ctx->delta;
+    Q.off = ctx->d_off; Q.tile_prefix = ctx->d_prefix; Q.nbr = ctx->d_nbr; Q.status = ctx->d_status;
+    Q.ld = ctx->cfg.ld; Q.K = ctx->cfg.K; Q.m = ctx->m; Q.q = ctx->cfg.q;
+    Q.eta = P.eta; Q.zeta = P.zeta; Q.qp1 = P.qp1; Q.inv_qp1 = P.inv_qp1; Q.inv_exact = P.inv_exact;
+    Q.T = L.T; Q.ring = L.ring; Q.ncols = L.tmem_cols;
+    Q.ring_off = L.ring_off; Q.meta_off = L.meta_off; Q.meta_stride = L.meta_stride;
+    cudaError_t e2 = cudaFuncSetAttribute(sync_fused_tmem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem);
+    if (e2 != cudaSuccess) return cuda_fail(ctx, "cudaFuncSetAttribute", e2);
+    sync_fused_tmem_kernel<<<grid, 544, L.smem, st>>>(Q);
+    e2 = cudaGetLastError();
+    if (e2 != cudaSuccess) return cuda_fail(ctx, "launch of the tensor-memory round kernel", e2);
+    return GBMUF_OK;
+  }
   if (ctx->cfg.theta_dtype == GBMUF_F32) return launch_sync<float>(ctx, P, grid, st, &ctx->attr_set[0]);
   return launch_sync<__nv_bfloat16>(ctx, P, grid, st, &ctx->attr_set[1]);
 }
