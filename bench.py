@@ -36,8 +36,8 @@ FALLBACK_HBM_GBS = 6650.0
 # + dram__bytes_write.sum divided by the replica-parameters of the captured launch; key = theta
 # dtype: 0 fp32 from workload profile16, 1 bf16 from profile16bf), valid only
 # for the kernel source it was taken from (source_sha() below).
-NCU_TRAFFIC = {"source_sha": "9b5ad4df2841", "bytes_per_replica_param": {0: 6.383138e9 / 268435536,
-                                                                   1: 5.309694e9 / 268435536}}
+NCU_TRAFFIC = {"source_sha": "fad09bdc3844", "bytes_per_replica_param": {0: 6.383452e9 / 268435536,
+                                                                   1: 5.309491e9 / 268435536}}
 
 
 def algorithmic_bytes_per_replica_param(dtype: int, mode: int = 0) -> int:
@@ -103,11 +103,12 @@ class ClockSampler:
 
 def source_sha() -> str:
     """Fingerprint of the fused kernel's source: the part of csrc/gbmuf.cu from the barrier /
-    bulk-copy primitives to the end of sync_fused_kernel (theta traits and filter included)."""
+    bulk-copy primitives to the end of sync_fused_kernel (theta traits and filter included;
+    the opt-in tensor-memory variant that follows it is not part of it)."""
     with open(os.path.join(ROOT, "paper_1909_09010_b200", "csrc", "gbmuf.cu"), "rb") as f:
         text = f.read()
     a = text.index(b"// Shared-memory barrier and bulk-copy primitives")
-    b = text.index(b"// Synthetic local step")
+    b = text.index(b"// Variant of the fused round that keeps the theta tile in tensor memory")
     return hashlib.sha256(text[a:b]).hexdigest()[:12]
 
 
