@@ -128,7 +128,9 @@ gbmuf_status gbmuf_local_adagrad(gbmuf_ctx* ctx, const float* grad_device, float
  * G = theta_bar - R, with R the component as the worker's previous sync left it (theta_0 before
  * any); Delta <- eta Delta + zeta G; omega <- omega + Delta; theta <- omega + eta Delta.
  * R is not stored: it is recomputed as store(omega + eta Delta) from the values before the round,
- * which is bit-for-bit the expression that produced it.  In MA mode theta <- theta_bar only.
+ * which is bit-for-bit the expression that produced it (so a caller that fills omega and Delta
+ * itself, rather than through gbmuf_init and earlier rounds, thereby defines R).  In MA mode
+ * theta <- theta_bar only.
  * Everything happens in place in one pass; components not taking part are not touched.
  * Requires set_partition.  Errors: BAD_STATE, INVALID_ARG, CUDA. */
 gbmuf_status gbmuf_sync_round(gbmuf_ctx* ctx, uint64_t round, const uint8_t* comp_mask_host,
