@@ -103,12 +103,12 @@ class ClockSampler:
 
 def source_sha() -> str:
     """Fingerprint of the fused kernel's source: the part of csrc/gbmuf.cu from the barrier /
-    bulk-copy primitives to the end of sync_fused_kernel (theta traits and filter included;
-    the opt-in tensor-memory variant that follows it is not part of it)."""
+    bulk-copy primitives to the end of the fused round kernels (theta traits, filter, the
+    shared-memory-tile kernel and the tensor-memory-tile kernel)."""
     with open(os.path.join(ROOT, "paper_1909_09010_b200", "csrc", "gbmuf.cu"), "rb") as f:
         text = f.read()
     a = text.index(b"// Shared-memory barrier and bulk-copy primitives")
-    b = text.index(b"// Variant of the fused round that keeps the theta tile in tensor memory")
+    b = text.index(b"// Self-test of the bounded wait")
     return hashlib.sha256(text[a:b]).hexdigest()[:12]
 
 
@@ -325,7 +325,7 @@ def run_gpu(args, w):
                              "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                              "frac_of_nominal_8TBs": achieved / 8000.0,
                              "algorithmic_bytes_per_replica_param": bpe, "traffic": traffic,
-                             "kernel": "sync_fused_kernel"},
+                             "kernel": "sync_fused_tmem_kernel" if info.get("variant") == "tmem" else "sync_fused_kernel"},
                 "clocks": clocks,
                 "gpu_launches": (3 if args.local_step == "perturb" else 5) * args.steps, "e2e": e2e}
         if not args.no_cpu_baseline and world == 1:

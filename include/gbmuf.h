@@ -159,18 +159,22 @@ gbmuf_status gbmuf_device_status(gbmuf_ctx* ctx, void* stream, int32_t* out);
 gbmuf_status gbmuf_selftest_wait_timeout(gbmuf_ctx* ctx, void* stream, double* seconds_out);
 
 /* Launch shape of the fused kernel (one persistent CTA per SM).  Any argument may be 0 to keep
- * the built-in choice.  consumer_threads: multiple of 32 in 32..992 (one more warp issues the
- * copies); tile_elems: elements of one component staged per work item for all K workers, a
- * multiple of 8 and, above 256, of 256; theta_stages: 1..4 tiles of theta resident per CTA;
- * ring_slots: 2..8 rows of omega/Delta in flight; flags: bit 0 = 256-byte L2 promotion for the
- * theta loads (default 128); bit 1 = keep the theta tile in tensor memory (fp32 theta,
- * gossip-BMUF mode, 4 <= K <= 128; tile_elems then a multiple of 512 with K * tile_elems / 128 <= 512).
- * Errors: INVALID_ARG, UNSUPPORTED (does not fit shared memory). */
+ * the built-in choice.  Two variants exist.  (a) theta tile in tensor memory, outputs through bulk
+ * stores: chosen automatically for fp32 theta in gossip-BMUF mode with 4 <= K <= 128; tile_elems
+ * must then be a multiple of 512 with K * tile_elems / 128 <= 512; ring_slots (2..8) is the number
+ * of shared-memory slots every row streams through.  (b) theta tile in shared memory: everything
+ * else, and whenever consumer_threads or theta_stages is given or flags bit 3 is set;
+ * consumer_threads: multiple of 32 in 32..992 (one more warp issues the copies); tile_elems: a
+ * multiple of 8 and, above 256, of 256; theta_stages: 1..4; ring_slots: 2..8 rows of omega/Delta in
+ * flight.  flags: bit 0 = 256-byte L2 promotion for the theta loads of (b); bit 1 = force (a),
+ * bit 2 (with bit 1) = with bulk stores (without: stores from registers); bit 3 = force (b).
+ * Errors: INVALID_ARG, UNSUPPORTED (does not fit, or (a) forced where it does not apply). */
 gbmuf_status gbmuf_set_tuning(gbmuf_ctx* ctx, int32_t consumer_threads, int32_t tile_elems,
                               int32_t theta_stages, int32_t ring_slots, int32_t flags);
 
 /* What the next full round would launch: tiles (work items), grid and block size, dynamic shared
- * memory in bytes, elements per tile, theta stages.  Any out pointer may be NULL.  Requires
+ * memory in bytes, elements per tile, theta stages in shared memory (0 = the theta tile is kept in
+ * tensor memory).  Any out pointer may be NULL.  Requires
  * set_partition. */
 gbmuf_status gbmuf_get_launch_info(gbmuf_ctx* ctx, int64_t* tiles, int32_t* grid, int32_t* block,
                                    int32_t* smem_bytes, int32_t* tile_elems, int32_t* stages);

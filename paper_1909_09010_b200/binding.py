@@ -271,7 +271,8 @@ class Gbmuf:
                                                 ctypes.byref(b), ctypes.byref(s), ctypes.byref(t),
                                                 ctypes.byref(st)))
         return {"tiles": tiles.value, "grid": g.value, "block": b.value, "smem_bytes": s.value,
-                "tile_elems": t.value, "stages": st.value}
+                "tile_elems": t.value, "stages": st.value,
+                "variant": "tmem" if st.value == 0 else "smem"}
 
     def last_error(self) -> str:
         return lib().gbmuf_last_error(self._h).decode()

@@ -645,8 +645,10 @@ struct TmemParams {
   int K, m, q;
   float eta, zeta, qp1, inv_qp1;
   int inv_exact;
-  int T, ring, ncols;      // T multiple of 512; ring slots of 2*T floats; TMEM columns (power of 2)
+  int T, ring, ncols;      // T multiple of 512; ring slots of 2 (3 with bulk stores) rows of T floats;
+                           // TMEM columns (power of 2)
   uint32_t ring_off, meta_off, meta_stride;   // meta ring (4 entries): [TileDesc | nbr K*q ints]
+  uint32_t slot_stride;    // bytes per ring slot
 };
 
 __device__ __forceinline__ void tmem_store4(uint32_t taddr, const float (&x)[4]) {
@@ -668,11 +670,18 @@ __device__ __forceinline__ void tmem_load4(uint32_t taddr, float (&x)[4]) {
   x[0] = __uint_as_float(a); x[1] = __uint_as_float(b); x[2] = __uint_as_float(c); x[3] = __uint_as_float(d);
 }
 
+// BULK: the outputs leave through bulk stores from the ring slot (a third row holds the new theta)
+// instead of st.global from registers.
+struct SlotInfo { long long e0, lo, hi; int k; int pad; };   // what the producer must know to retire a slot
+
+template <bool BULK>
 __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParams P) {
   extern __shared__ __align__(128) unsigned char smem[];
-  // [0,64) ring full, [64,128) ring empty, [128,132) TMEM base address
+  // [0,64) ring full, [64,128) ring empty (consumers done), [128,132) TMEM base address,
+  // [192,448) per-slot retire information (BULK)
   const uint32_t bars = smem_u32(smem);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 128);
+  SlotInfo* sinfo = reinterpret_cast<SlotInfo*>(smem + 192);
   unsigned char* ring0 = smem + P.ring_off;
   unsigned char* meta0 = smem + P.meta_off;
   const int total = P.tile_prefix[P.m];
@@ -718,6 +727,31 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
     }
     int gi = 0;              // ring items requested so far
     bool ok = true;
+    // BULK: item j is finished by the consumers -> send its results out of the slot.  One bulk
+    // group per item (an empty one for theta items) so that "all but the newest group have been
+    // read" means exactly "the slot about to be refilled is free".
+    auto retire = [&](int j) -> bool {
+      const int slot = j % R;
+      bool fine = mbar_wait_bounded(bars + 64 + 8 * slot, (j / R) & 1, P.status);
+      if (!__all_sync(0xffffffffu, fine)) return false;
+      if (lane == 0) {
+        const SlotInfo si = sinfo[slot];
+        if (si.k >= 0) {
+          const long long sb = (si.lo + 3) & ~3LL, se = si.hi & ~3LL;   // whole groups of 4 inside the tile
+          if (se > sb) {
+            const uint32_t src = smem_u32(ring0 + (size_t)slot * P.slot_stride) + (uint32_t)(sb - si.e0) * 4u;
+            const uint32_t nbytes = (uint32_t)(se - sb) * 4u;
+            const long long at = (long long)si.k * P.ld + sb;
+            asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(P.omega + at), "r"(src), "r"(nbytes) : "memory");
+            asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(P.delta + at), "r"(src + (uint32_t)T * 4u), "r"(nbytes) : "memory");
+            asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(P.theta + at), "r"(src + (uint32_t)T * 8u), "r"(nbytes) : "memory");
+          }
+        }
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+      }
+      __syncwarp();
+      return true;
+    };
     for (int it = 0; it < my_tiles && ok; ++it) {
       const int w = (int)blockIdx.x + it * (int)gridDim.x;
       if (w >= pfx_hi) {
@@ -752,14 +786,26 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
       __syncwarp();
       for (int item = 0; item < ntheta + K && ok; ++item, ++gi) {
         const int slot = gi % R;
-        if (gi >= R) {
+        if (BULK) {
+          if (gi >= R - 1) ok = retire(gi - (R - 1));       // consumers done with it; its stores go out
+          if (!ok) break;
+          if (gi >= R && lane == 0)                          // the slot's own stores have read it
+            asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+          __syncwarp();
+        } else if (gi >= R) {
           bool fine = mbar_wait_bounded(bars + 64 + 8 * slot, ((gi / R) - 1) & 1, P.status);
           ok = __all_sync(0xffffffffu, fine);
           if (!ok) break;
         }
         if (lane == 0) {
           const uint32_t full = bars + 8 * slot;
-          const uint32_t dst = smem_u32(ring0 + (size_t)slot * (size_t)T * 8);
+          const uint32_t dst = smem_u32(ring0 + (size_t)slot * P.slot_stride);
+          if (BULK) {
+            sinfo[slot].e0 = e0;
+            sinfo[slot].lo = cb > e0 ? cb : e0;
+            sinfo[slot].hi = ce < e0 + T ? ce : e0 + T;
+            sinfo[slot].k = item < ntheta ? -1 : item - ntheta;
+          }
           if (item < ntheta) {
             const int r0 = 2 * item, rows = (r0 + 1 < K) ? 2 : 1;
             mbar_arrive_expect_tx(full, (uint32_t)rows * bytes);
@@ -773,6 +819,11 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
           }
         }
       }
+    }
+    if (BULK) {
+      for (int j = gi > R - 1 ? gi - (R - 1) : 0; j < gi && ok; ++j) ok = retire(j);
+      if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+      __syncwarp();
     }
     if (!ok) {
       for (int j = gi > R ? gi - R : 0; j < gi; ++j)
@@ -797,8 +848,9 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
         ok = __all_sync(0xffffffffu, fine);
         if (!ok) break;
         if (item == 0) { e0 = d->e0; lo = d->lo; hi = d->hi; }
-        const float* row0 = reinterpret_cast<const float*>(ring0 + (size_t)slot * (size_t)T * 8);
-        const float* row1 = row0 + T;
+        float* row0 = reinterpret_cast<float*>(ring0 + (size_t)slot * P.slot_stride);
+        float* row1 = row0 + T;
+        float* row2 = row1 + T;   // BULK: the new theta
         if (item < ntheta) {
           // deposit two theta rows into this thread's TMEM cells
           const int r0 = 2 * item;
@@ -836,9 +888,15 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
             for (int x = 0; x < 4; ++x) bmuf_filter<float>(a[x], wv[x], dv[x], t[x], P.eta, P.zeta);
             const long long at = (long long)k * P.ld + e;
             if (e >= lo && e + 4 <= hi) {
-              __stcs(reinterpret_cast<float4*>(P.delta + at), make_float4(dv[0], dv[1], dv[2], dv[3]));
-              __stcs(reinterpret_cast<float4*>(P.omega + at), make_float4(wv[0], wv[1], wv[2], wv[3]));
-              __stcs(reinterpret_cast<float4*>(P.theta + at), make_float4(t[0], t[1], t[2], t[3]));
+              if (BULK) {
+                *reinterpret_cast<float4*>(row0 + col) = make_float4(wv[0], wv[1], wv[2], wv[3]);
+                *reinterpret_cast<float4*>(row1 + col) = make_float4(dv[0], dv[1], dv[2], dv[3]);
+                *reinterpret_cast<float4*>(row2 + col) = make_float4(t[0], t[1], t[2], t[3]);
+              } else {
+                __stcs(reinterpret_cast<float4*>(P.delta + at), make_float4(dv[0], dv[1], dv[2], dv[3]));
+                __stcs(reinterpret_cast<float4*>(P.omega + at), make_float4(wv[0], wv[1], wv[2], wv[3]));
+                __stcs(reinterpret_cast<float4*>(P.theta + at), make_float4(t[0], t[1], t[2], t[3]));
+              }
             } else {
               for (int x = 0; x < 4; ++x) {
                 if (e + x >= lo && e + x < hi) {
@@ -850,6 +908,7 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
             }
           }
         }
+        if (BULK && item >= ntheta) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         mbar_arrive(bars + 64 + 8 * slot);
       }
     }
@@ -1401,7 +1460,6 @@ struct gbmuf_ctx {
   Tuning tuning;
   Launch launch;
   CUtensorMap map_theta;   // boxes [K rows][launch.BW columns] over theta
-  bool attr_set[2] = {false, false};
   std::string err;
 };
 
@@ -1476,32 +1534,53 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
   L.flags = t.flags;
   L.tmem_cols = 0; L.meta_off = 0; L.meta_stride = 0;
   const long long cap = ctx->max_smem < ctx->smem_per_sm - 1024 ? ctx->max_smem : ctx->smem_per_sm - 1024;
-  if (t.flags & 2) {
-    // theta tile in tensor memory: fp32 theta, gossip-BMUF, 4 <= K, K * (T/512) * 4 <= 512 columns
-    if (esz != 4 || !bmuf || K < 4 || K > 128)
-      return fail(ctx, GBMUF_ERR_UNSUPPORTED, "the tensor-memory variant needs fp32 theta, BMUF mode and 4 <= K <= 128");
-    int T = t.T ? t.T : 4096;
-    while (!t.T && T > 512 && (T / 512) * K * 4 > 512) T >>= 1;
-    if (T < 512 || T % 512 != 0 || (T / 512) * K * 4 > 512)
+  // Variant: flags bit 3 forces the shared-memory theta tile, bit 1 forces the tensor-memory tile
+  // (bit 2: with bulk stores); with neither, the tensor-memory tile with bulk stores is used
+  // wherever it applies (fp32 theta, gossip-BMUF, 4 <= K <= 128) -- it is the faster one.
+  const bool tmem_ok = esz == 4 && bmuf && K >= 4 && K <= 128;
+  // (automatic choice only when the caller has not asked for anything specific to the
+  // shared-memory tile: consumer threads, theta stages, or a tile width it cannot have)
+  const bool auto_tmem = !(t.flags & 8) && tmem_ok && t.ncons == 0 && t.stages == 0 &&
+                         (t.T == 0 || (t.T % 512 == 0 && (t.T / 512) * K * 4 <= 512));
+  const bool want_tmem = (t.flags & 2) || auto_tmem;
+  if ((t.flags & 2) && !tmem_ok)
+    return fail(ctx, GBMUF_ERR_UNSUPPORTED, "the tensor-memory variant needs fp32 theta, BMUF mode and 4 <= K <= 128");
+  if (want_tmem) {
+    const bool bulk = (t.flags & 2) ? (t.flags & 4) != 0 : true;
+    const bool forced = (t.flags & 2) != 0;
+    // theta tile in tensor memory: K * (T/512) * 4 <= 512 columns; T a multiple of 512
+    int T = t.T ? t.T : 3584;
+    while (!t.T && T > 512 && (T / 512) * K * 4 > 512) T -= 512;
+    bool fits = T >= 512 && T % 512 == 0 && (T / 512) * K * 4 <= 512;
+    if (!fits && (forced || t.T))
       return fail(ctx, GBMUF_ERR_INVALID_ARG, "tensor-memory variant: tile_elems must be a multiple of 512 with K * tile_elems / 128 <= 512");
-    L.T = T; L.BW = 256; L.stages = 1; L.ncons = 512;
-    L.meta_off = 256;
-    L.meta_stride = (uint32_t)(((long long)sizeof(TileDesc) + (long long)K * q * 4 + 127) / 128 * 128);
-    L.ring_off = L.meta_off + 4 * L.meta_stride;
-    L.slot_stride = (uint32_t)(8 * T);
-    int R = t.ring ? t.ring : 6;
-    while (!t.ring && R > 2 && (long long)L.ring_off + (long long)R * L.slot_stride > cap) --R;
-    if ((long long)L.ring_off + (long long)R * L.slot_stride > cap || R < 2)
-      return fail(ctx, GBMUF_ERR_UNSUPPORTED, "tensor-memory variant: the ring does not fit shared memory");
-    L.ring = R;
-    L.smem = (uint32_t)(L.ring_off + (long long)R * L.slot_stride);
-    int cols = 32;
-    while (cols < (T / 512) * K * 4) cols <<= 1;
-    L.tmem_cols = cols;
-    L.stage_stride = 0; L.nbr_off = 0; L.desc_off = 0;
-    *out = L;
-    return GBMUF_OK;
+    if (fits) {
+      L.T = T; L.BW = 256; L.stages = 1; L.ncons = 512;
+      L.flags = (t.flags & 1) | 2 | (bulk ? 4 : 0);
+      L.meta_off = 512;
+      L.meta_stride = (uint32_t)(((long long)sizeof(TileDesc) + (long long)K * q * 4 + 127) / 128 * 128);
+      L.ring_off = L.meta_off + 4 * L.meta_stride;
+      L.slot_stride = (uint32_t)((bulk ? 12 : 8) * T);
+      int R = t.ring ? t.ring : (bulk ? 5 : 3);
+      while (!t.ring && R > 3 && (long long)L.ring_off + (long long)R * L.slot_stride > cap) --R;
+      while (!t.ring && R < 8 && (long long)R * L.slot_stride < 160 * 1024 &&
+             (long long)L.ring_off + (long long)(R + 1) * L.slot_stride <= cap) ++R;   // small slots: more of them
+      const bool ring_fits = (long long)L.ring_off + (long long)R * L.slot_stride <= cap && R >= 2;
+      if (!ring_fits && (forced || t.ring))
+        return fail(ctx, GBMUF_ERR_UNSUPPORTED, "tensor-memory variant: the ring does not fit shared memory");
+      if (ring_fits) {
+        L.ring = R;
+        L.smem = (uint32_t)(L.ring_off + (long long)R * L.slot_stride);
+        int cols = 32;
+        while (cols < (T / 512) * K * 4) cols <<= 1;
+        L.tmem_cols = cols;
+        L.stage_stride = 0; L.nbr_off = 0; L.desc_off = 0;
+        *out = L;
+        return GBMUF_OK;
+      }
+    }
   }
+  L.flags = t.flags & 1;
   auto stage_bytes = [&](int T, Launch* l) {
     long long at = ((long long)K * T * esz + 15) / 16 * 16;
     if (l) l->nbr_off = (uint32_t)at;
@@ -1574,21 +1653,6 @@ long long host_total_tiles(const gbmuf_ctx* ctx, uint64_t round, const uint8_t* 
   return total;
 }
 
-template <typename TH>
-gbmuf_status launch_sync(gbmuf_ctx* ctx, const SyncParams& P, int grid, cudaStream_t st, bool* attr) {
-  auto kern = sync_fused_kernel<TH>;
-  if (!*attr) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         ctx->max_smem);
-    if (e != cudaSuccess) return cuda_fail(ctx, "cudaFuncSetAttribute", e);
-    *attr = true;
-  }
-  kern<<<grid, 32 + P.ncons, ctx->launch.smem, st>>>(P, ctx->map_theta);
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return cuda_fail(ctx, "launch of the fused round kernel", e);
-  return GBMUF_OK;
-}
-
 // Everything the fused kernel needs to know about one launch.
 void fill_sync_params(const gbmuf_config& cfg, const Launch& L, void* theta, float* omega,
                       float* delta, long long ld, int m, const int64_t* off, const int32_t* prefix,
@@ -1604,6 +1668,42 @@ void fill_sync_params(const gbmuf_config& cfg, const Launch& L, void* theta, flo
   else { P->bw_shift = 30; P->bw_mask = (1 << 30) - 1; }          // one box
   P->stage_stride = L.stage_stride; P->nbr_off = L.nbr_off; P->desc_off = L.desc_off;
   P->ring_off = L.ring_off; P->slot_stride = L.slot_stride;
+}
+
+// Launches the fused round in the variant the launch shape names.  `ctx` supplies the error
+// slot, the device limits and (shared-memory variant) the tensor map of theta.
+gbmuf_status launch_round(gbmuf_ctx* ctx, const gbmuf_config& cfg, const Launch& L, void* theta,
+                          float* omega, float* delta, long long ld, int m, const int64_t* off,
+                          const int32_t* prefix, const int32_t* nbr, int32_t* status,
+                          long long total, cudaStream_t st) {
+  const int grid = (int)(total < ctx->num_sms ? total : ctx->num_sms);   // one persistent CTA per SM
+  SyncParams P;
+  fill_sync_params(cfg, L, theta, omega, delta, ld, m, off, prefix, nbr, status, &P);
+  cudaError_t e;
+  if (L.tmem_cols > 0) {
+    TmemParams Q;
+    Q.theta_in = (const float*)theta; Q.theta = (float*)theta; Q.omega = omega; Q.delta = delta;
+    Q.off = off; Q.tile_prefix = prefix; Q.nbr = nbr; Q.status = status;
+    Q.ld = ld; Q.K = cfg.K; Q.m = m; Q.q = cfg.q;
+    Q.eta = P.eta; Q.zeta = P.zeta; Q.qp1 = P.qp1; Q.inv_qp1 = P.inv_qp1; Q.inv_exact = P.inv_exact;
+    Q.T = L.T; Q.ring = L.ring; Q.ncols = L.tmem_cols;
+    Q.ring_off = L.ring_off; Q.meta_off = L.meta_off; Q.meta_stride = L.meta_stride; Q.slot_stride = L.slot_stride;
+    auto kern = (L.flags & 4) ? sync_fused_tmem_kernel<true> : sync_fused_tmem_kernel<false>;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem);
+    if (e != cudaSuccess) return cuda_fail(ctx, "cudaFuncSetAttribute", e);
+    kern<<<grid, 544, L.smem, st>>>(Q);
+  } else if (cfg.theta_dtype == GBMUF_F32) {
+    e = cudaFuncSetAttribute(sync_fused_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem);
+    if (e != cudaSuccess) return cuda_fail(ctx, "cudaFuncSetAttribute", e);
+    sync_fused_kernel<float><<<grid, 32 + L.ncons, L.smem, st>>>(P, ctx->map_theta);
+  } else {
+    e = cudaFuncSetAttribute(sync_fused_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem);
+    if (e != cudaSuccess) return cuda_fail(ctx, "cudaFuncSetAttribute", e);
+    sync_fused_kernel<__nv_bfloat16><<<grid, 32 + L.ncons, L.smem, st>>>(P, ctx->map_theta);
+  }
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(ctx, "launch of the fused round kernel", e);
+  return GBMUF_OK;
 }
 
 void fill_setup(const gbmuf_ctx* ctx, uint64_t round, bool use_mask, bool plan, int32_t* nbr,
@@ -1757,7 +1857,7 @@ gbmuf_status gbmuf_set_tuning(gbmuf_ctx* ctx, int32_t ncons, int32_t tile_elems,
                               int32_t ring, int32_t flags) {
   if (!ctx) return GBMUF_ERR_INVALID_ARG;
   if (ncons < 0 || ncons > 992 || ncons % 32 != 0 || tile_elems < 0 || tile_elems > (1 << 16) ||
-      stages < 0 || stages > kMaxThetaStages || ring < 0 || ring > kMaxRing || ring == 1 || flags < 0 || flags > 3)
+      stages < 0 || stages > kMaxThetaStages || ring < 0 || ring > kMaxRing || ring == 1 || flags < 0 || flags > 15 || ((flags & 4) && !(flags & 2)) || ((flags & 8) && (flags & 2)))
     return fail(ctx, GBMUF_ERR_INVALID_ARG, "tuning value out of range");
   Tuning t;
   t.ncons = ncons; t.T = tile_elems; t.stages = stages; t.ring = ring; t.flags = flags;
@@ -1785,7 +1885,7 @@ gbmuf_status gbmuf_get_launch_info(gbmuf_ctx* ctx, int64_t* tiles, int32_t* grid
   if (block) *block = 32 + ctx->launch.ncons;
   if (smem) *smem = (int32_t)ctx->launch.smem;
   if (tile_elems) *tile_elems = ctx->launch.T;
-  if (stages) *stages = ctx->launch.stages;
+  if (stages) *stages = ctx->launch.tmem_cols > 0 ? 0 : ctx->launch.stages;
   return GBMUF_OK;
 }
 
@@ -1914,28 +2014,8 @@ gbmuf_status gbmuf_sync_round(gbmuf_ctx* ctx, uint64_t round, const uint8_t* com
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, "launch of the round set-up kernel", e);
 
-  SyncParams P;
-  fill_sync_params(ctx->cfg, L, ctx->theta, ctx->omega, ctx->delta, ctx->cfg.ld, ctx->m, ctx->d_off,
-                   ctx->d_prefix, ctx->d_nbr, ctx->d_status, &P);
-  const long long cap = (long long)ctx->num_sms;              // one persistent CTA per SM
-  const int grid = (int)(total < cap ? total : cap);
-  if (L.tmem_cols > 0) {
-    TmemParams Q;
-    Q.theta_in = (const float*)ctx->theta; Q.theta = (float*)ctx->theta; Q.omega = ctx->omega; Q.delta = ctx->delta;
-    Q.off = ctx->d_off; Q.tile_prefix = ctx->d_prefix; Q.nbr = ctx->d_nbr; Q.status = ctx->d_status;
-    Q.ld = ctx->cfg.ld; Q.K = ctx->cfg.K; Q.m = ctx->m; Q.q = ctx->cfg.q;
-    Q.eta = P.eta; Q.zeta = P.zeta; Q.qp1 = P.qp1; Q.inv_qp1 = P.inv_qp1; Q.inv_exact = P.inv_exact;
-    Q.T = L.T; Q.ring = L.ring; Q.ncols = L.tmem_cols;
-    Q.ring_off = L.ring_off; Q.meta_off = L.meta_off; Q.meta_stride = L.meta_stride;
-    cudaError_t e2 = cudaFuncSetAttribute(sync_fused_tmem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem);
-    if (e2 != cudaSuccess) return cuda_fail(ctx, "cudaFuncSetAttribute", e2);
-    sync_fused_tmem_kernel<<<grid, 544, L.smem, st>>>(Q);
-    e2 = cudaGetLastError();
-    if (e2 != cudaSuccess) return cuda_fail(ctx, "launch of the tensor-memory round kernel", e2);
-    return GBMUF_OK;
-  }
-  if (ctx->cfg.theta_dtype == GBMUF_F32) return launch_sync<float>(ctx, P, grid, st, &ctx->attr_set[0]);
-  return launch_sync<__nv_bfloat16>(ctx, P, grid, st, &ctx->attr_set[1]);
+  return launch_round(ctx, ctx->cfg, L, ctx->theta, ctx->omega, ctx->delta, ctx->cfg.ld, ctx->m, ctx->d_off,
+                      ctx->d_prefix, ctx->d_nbr, ctx->d_status, total, st);
 }
 
 gbmuf_status gbmuf_get_neighbors(gbmuf_ctx* ctx, uint64_t round, int32_t* out) {
@@ -2167,12 +2247,8 @@ gbmuf_status gbmuf_sync_round_noalloc(const gbmuf_config* cfg, void* theta, floa
     e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(nullptr, "launch of the round set-up kernel", e);
 
-    SyncParams P;
-    fill_sync_params(*cfg, L, theta, omega, delta, cfg->ld, m, S.off, S.tile_prefix, S.nbr, d_status, &P);
-    const int grid = (int)(total < tmp.num_sms ? total : tmp.num_sms);
-    bool attr = false;
-    st = cfg->theta_dtype == GBMUF_F32 ? launch_sync<float>(&tmp, P, grid, cs, &attr)
-                                       : launch_sync<__nv_bfloat16>(&tmp, P, grid, cs, &attr);
+    st = launch_round(&tmp, *cfg, L, theta, omega, delta, cfg->ld, m, S.off, S.tile_prefix, S.nbr, d_status,
+                      total, cs);
     if (st != GBMUF_OK) { g_create_error = tmp.err; return st; }
   }
   if (device_status_out) {
@@ -2329,12 +2405,8 @@ gbmuf_status gbmuf_sync_round_host(const gbmuf_config* cfg, void* theta, float* 
     e = cudaGetLastError();
     if (e != cudaSuccess) { st = cuda_fail(nullptr, "launch of the round set-up kernel", e); break; }
     const Launch& L = hs.ctx.launch;
-    SyncParams P;
-    fill_sync_params(*cfg, L, hs.ctx.theta, hs.ctx.omega, hs.ctx.delta, chunk_cols, mc, S.off,
-                     S.tile_prefix, S.nbr, reinterpret_cast<int32_t*>(hs.tables + t_status), &P);
-    const int grid = (int)(total < hs.ctx.num_sms ? total : hs.ctx.num_sms);
-    st = esz == 4 ? launch_sync<float>(&hs.ctx, P, grid, cs, &hs.ctx.attr_set[0])
-                  : launch_sync<__nv_bfloat16>(&hs.ctx, P, grid, cs, &hs.ctx.attr_set[1]);
+    st = launch_round(&hs.ctx, *cfg, L, hs.ctx.theta, hs.ctx.omega, hs.ctx.delta, chunk_cols, mc, S.off,
+                      S.tile_prefix, S.nbr, reinterpret_cast<int32_t*>(hs.tables + t_status), total, cs);
     if (st != GBMUF_OK) { g_create_error = hs.ctx.err; break; }
     e = cudaMemcpy2DAsync((char*)theta + (size_t)c0 * esz, (size_t)cfg->ld * esz, hs.ctx.theta,
                           (size_t)chunk_cols * esz, w_th, K, cudaMemcpyDeviceToHost, cs);

@@ -37,16 +37,17 @@ def _restart_invariant(pr, eta):
     return ok
 
 
-@pytest.mark.parametrize("name,over", [("wikitext103", {}), ("longrun", {}),
-                                       ("sweep", dict(C=256, q=4, eta=0.5)),
-                                       ("sweep", dict(C=64, q=1, eta=0.9))])
-def test_full_size_sampled_parity(name, over):
+@pytest.mark.parametrize("name,over,tuning", [("wikitext103", {}, None), ("longrun", {}, None),
+                                              ("sweep", dict(C=256, q=4, eta=0.5), None),
+                                              ("sweep", dict(C=64, q=1, eta=0.9), None),
+                                              ("wikitext103", {}, dict(flags=8))])
+def test_full_size_sampled_parity(name, over, tuning):
     w = workloads.get(name, **over)
     dev = torch.device("cuda:0")
     theta0 = workloads.theta0_torch(w, dev)
     if w.dtype == 1:
         theta0 = theta0.to(torch.bfloat16)
-    pr = Pair(case_of(w), theta0, slices=_slices(w))
+    pr = Pair(case_of(w), theta0, slices=_slices(w), tuning=tuning)
     try:
         info = pr.g.launch_info()
         assert info["grid"] == torch.cuda.get_device_properties(0).multi_processor_count

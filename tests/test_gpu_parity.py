@@ -75,6 +75,9 @@ RAGGED = [
 def test_ragged_shapes(K, offsets, p, q, dtype):
     case = Case(K=K, offsets=offsets, p=p, q=q, eta=0.875, zeta=1.0, dtype=dtype, seed=K * 31 + q)
     run(case, random_theta0(case.N, seed=K, dtype=dtype), rounds=3, sigma=5e-2)
+    if dtype == 0 and 4 <= K <= 128:      # the default was the tensor-memory tile: also the shared-memory one
+        run(case, random_theta0(case.N, seed=K, dtype=dtype), rounds=3, sigma=5e-2, tuning=dict(flags=8),
+            check_nbr=False)
 
 
 @pytest.mark.parametrize("tuning", [
@@ -337,9 +340,11 @@ def test_random_shapes_property():
         dtype = data.draw(st_.integers(0, 1))
         mode = data.draw(st_.sampled_from([0, 0, 0, 1]))
         tile = data.draw(st_.sampled_from([0, 64, 256, 512]))
+        force_smem = data.draw(st_.booleans())
         case = Case(K=K, offsets=offsets, p=p, q=q, eta=eta, zeta=zeta, dtype=dtype,
                     seed=data.draw(st_.integers(0, 2 ** 63)), mode=mode)
-        tuning = dict(tile_elems=tile, consumer_threads=data.draw(st_.sampled_from([64, 256]))) if tile else None
+        tuning = dict(tile_elems=tile, consumer_threads=data.draw(st_.sampled_from([64, 256]))) if tile else \
+            (dict(flags=8) if force_smem else None)
         run(case, random_theta0(N, seed=K + N, dtype=dtype), rounds=2, sigma=5e-2, tuning=tuning)
 
     inner()
@@ -444,16 +449,17 @@ def test_special_values_propagate_identically(dtype):
         pr.close()
 
 
+@pytest.mark.parametrize("flags", [2, 6])          # 6: outputs leave through bulk stores
 @pytest.mark.parametrize("K,p,q,tile,ring", [(16, 3, 2, 0, 0), (8, 2, 2, 2048, 4), (5, 2, 4, 1024, 3),
                                               (4, 1, 1, 512, 8), (16, 3, 6, 1024, 2), (32, 4, 3, 2048, 0)])
-def test_tensor_memory_variant(K, p, q, tile, ring):
+def test_tensor_memory_variant(K, p, q, tile, ring, flags):
     """The variant that parks the theta tile in tensor memory gives the same bits: several tiles
     per CTA, ragged component edges, masks, odd K (a half-filled last theta item)."""
     offsets = (0, 100_003, 100_004, 350_001, 777_777)
     case = Case(K=K, offsets=offsets, p=p, q=q, eta=0.875, zeta=1.0, dtype=0, seed=K + q)
     masks = [None, [1, 0, 1, 1], None]
     run(case, random_theta0(case.N, seed=K, dtype=0), rounds=3, sigma=5e-2, masks=masks,
-        tuning=dict(tile_elems=tile, ring_slots=ring, flags=2), check_nbr=False)
+        tuning=dict(tile_elems=tile, ring_slots=ring, flags=flags), check_nbr=False)
 
 
 def test_tensor_memory_variant_is_refused_where_it_does_not_apply():
