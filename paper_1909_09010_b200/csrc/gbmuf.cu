@@ -1561,10 +1561,12 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
       L.meta_stride = (uint32_t)(((long long)sizeof(TileDesc) + (long long)K * q * 4 + 127) / 128 * 128);
       L.ring_off = L.meta_off + 4 * L.meta_stride;
       L.slot_stride = (uint32_t)((bulk ? 12 : 8) * T);
-      int R = t.ring ? t.ring : (bulk ? 5 : 3);
-      while (!t.ring && R > 3 && (long long)L.ring_off + (long long)R * L.slot_stride > cap) --R;
-      while (!t.ring && R < 8 && (long long)R * L.slot_stride < 160 * 1024 &&
-             (long long)L.ring_off + (long long)(R + 1) * L.slot_stride <= cap) ++R;   // small slots: more of them
+      // Ring depth: 4 slots of the default width measured best (3 starve the pipeline, 5 and more
+      // put too much in flight; even counts did better than odd ones); narrower slots: more of them.
+      int R = t.ring ? t.ring : (bulk ? 4 : 3);
+      while (!t.ring && R > 2 && (long long)L.ring_off + (long long)R * L.slot_stride > cap) --R;
+      while (!t.ring && bulk && R + 2 <= 8 && (long long)R * L.slot_stride < 160 * 1024 &&
+             (long long)L.ring_off + (long long)(R + 2) * L.slot_stride <= cap) R += 2;
       const bool ring_fits = (long long)L.ring_off + (long long)R * L.slot_stride <= cap && R >= 2;
       if (!ring_fits && (forced || t.ring))
         return fail(ctx, GBMUF_ERR_UNSUPPORTED, "tensor-memory variant: the ring does not fit shared memory");
