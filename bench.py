@@ -34,9 +34,10 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of the fused kernel per replica-parameter from an ncu capture (dram__bytes_read.sum
 # + dram__bytes_write.sum divided by the replica-parameters of the captured launch; key = theta
-# dtype: 0 fp32 from workload profile16, 1 bf16 from profile16bf), valid only
+# dtype: 0 fp32 from workload profile16 (tensor-memory kernel), 1 bf16 from profile16bf
+# (shared-memory kernel)), valid only
 # for the kernel source it was taken from (source_sha() below).
-NCU_TRAFFIC = {"source_sha": "fad09bdc3844", "bytes_per_replica_param": {0: 6.383452e9 / 268435536,
+NCU_TRAFFIC = {"source_sha": "b3ec2c12f686", "bytes_per_replica_param": {0: 6.383429e9 / 268435536,
                                                                    1: 5.309491e9 / 268435536}}
 
 
