@@ -160,9 +160,10 @@ gbmuf_status gbmuf_selftest_wait_timeout(gbmuf_ctx* ctx, void* stream, double* s
 
 /* Launch shape of the fused kernel (one persistent CTA per SM).  Any argument may be 0 to keep
  * the built-in choice.  Two variants exist.  (a) theta tile in tensor memory, outputs through bulk
- * stores: chosen automatically for fp32 theta in gossip-BMUF mode with 4 <= K <= 128; tile_elems
- * must then be a multiple of 512 with K * tile_elems / 128 <= 512; ring_slots (2..8) is the number
- * of shared-memory slots every row streams through.  (b) theta tile in shared memory: everything
+ * stores: chosen automatically in gossip-BMUF mode with 4 <= K <= 128; tile_elems must then be a
+ * multiple of 512 whose K rows fit the 512 columns of tensor memory (K * tile_elems / 128 <= 512
+ * for fp32 theta, <= 1024 for bf16); ring_slots (2..8, at most three tiles' worth of rows) is the
+ * number of shared-memory slots every row streams through.  (b) theta tile in shared memory: everything
  * else, and whenever consumer_threads or theta_stages is given or flags bit 3 is set;
  * consumer_threads: multiple of 32 in 32..992 (one more warp issues the copies); tile_elems: a
  * multiple of 8 and, above 256, of 256; theta_stages: 1..4; ring_slots: 2..8 rows of omega/Delta in

@@ -616,25 +616,29 @@ sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_th
 
 // =================================================================================================
 // Variant of the fused round that keeps the theta tile in tensor memory (TMEM) instead of shared
-// memory (fp32 theta, gossip-BMUF mode).  A K x T fp32 tile of up to 256 KB does not fit shared
-// memory next to anything else, but it is exactly what the 512 columns x 128 lanes of an SM's
-// tensor memory hold.  Every row of theta, omega and Delta streams through one ring of
-// shared-memory slots (two rows of T floats per slot): first the K theta rows of a tile, which
-// each consumer thread moves from the slot into its own TMEM cells (tcgen05.st), then, worker by
-// worker, omega and Delta, for which the thread reads its own and the drawn neighbours' theta
-// back from those cells (tcgen05.ld).  A thread only ever reads cells it wrote itself, so TMEM
-// needs no synchronisation between threads, and the run per row can be twice as long as with a
-// shared-memory tile.
+// memory.  A K x T fp32 tile of up to 256 KB does not fit shared memory next to anything else,
+// but it is exactly what the 512 columns x 128 lanes of an SM's tensor memory hold.  Every row of
+// theta, omega and Delta streams through one ring of shared-memory slots: first the K theta rows
+// of a tile (several per slot), which each consumer thread moves from the slot into its own TMEM
+// cells (tcgen05.st), then the output items, for which the thread reads its own and the drawn
+// neighbours' theta back from those cells (tcgen05.ld).  A thread only ever reads cells it wrote
+// itself, so TMEM needs no synchronisation between threads, and the run per row can be about
+// twice as long as with a shared-memory tile.
 //
-// TMEM addressing: a warp reaches the 32 lanes 32 * (warp id % 4) ..; with the .32x32b.x4 shape
-// each thread moves the 4 consecutive 32-bit columns of its lane that start at the given column.
-// Element group g (4 elements) of a tile lives in lane g % 128, columns ((g / 128) * K + row) * 4.
-// The allocation is released by the warp that made it after every thread has reached the end of
-// the kernel; no path returns early.
+// (gossip-BMUF mode only.  The same schedule was tried for gossip-MA, whose output items carry
+// only averages: its consumers, 16 warps of serial TMEM round trips, could not keep up with 8
+// bytes per element and it ran at 60 % of the shared-memory schedule's speed.)
+//
+// TMEM addressing: a warp reaches the 32 lanes 32 * (warp id % 4) ..; with the .32x32b.xN shape
+// each thread moves the N consecutive 32-bit columns of its lane that start at the given column.
+// Four consecutive elements of a row are one cell: 4 columns for fp32, 2 for bf16 (kept packed).
+// Element group g (4 elements) of a tile lives in lane g % 128, columns ((g / 128) * K + row) *
+// cell width.  The allocation is released by the warp that made it after every thread has
+// reached the end of the kernel; no path returns early.
 // =================================================================================================
 struct TmemParams {
-  const float* theta_in;   // same array as theta (read side)
-  float* theta;
+  const void* theta_in;    // same array as theta (read side)
+  void* theta;
   float* omega;
   float* delta;
   const int64_t* off;
@@ -645,37 +649,93 @@ struct TmemParams {
   int K, m, q;
   float eta, zeta, qp1, inv_qp1;
   int inv_exact;
-  int T, ring, ncols;      // T multiple of 512; ring slots of 2 (3 with bulk stores) rows of T floats;
-                           // TMEM columns (power of 2)
+  int T, ring, ncols;      // T multiple of 512; ring slots; TMEM columns (power of 2)
   uint32_t ring_off, meta_off, meta_stride;   // meta ring (4 entries): [TileDesc | nbr K*q ints]
   uint32_t slot_stride;    // bytes per ring slot
 };
 
-__device__ __forceinline__ void tmem_store4(uint32_t taddr, const float (&x)[4]) {
-  asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};" ::"r"(taddr),
-               "r"(__float_as_uint(x[0])), "r"(__float_as_uint(x[1])), "r"(__float_as_uint(x[2])),
-               "r"(__float_as_uint(x[3]))
-               : "memory");
-}
-__device__ __forceinline__ void tmem_load4(uint32_t taddr, float (&x)[4]) {
-  uint32_t a, b, c, d;
-  // load and wait in one statement: the registers are only valid after the wait, and nothing may
-  // be scheduled between the two
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];\n\t"
-      "tcgen05.wait::ld.sync.aligned;"
-      : "=r"(a), "=r"(b), "=r"(c), "=r"(d)
-      : "r"(taddr)
-      : "memory");
-  x[0] = __uint_as_float(a); x[1] = __uint_as_float(b); x[2] = __uint_as_float(c); x[3] = __uint_as_float(d);
+// Four consecutive theta elements of one row <-> this thread's TMEM cell.  Load and wait sit in
+// ONE asm statement because the registers are only valid after the wait and nothing may be
+// scheduled between the two.  (Several loads per wait were measured slower, not faster.)
+template <typename TH> struct TmemCell;
+template <> struct TmemCell<float> {
+  static constexpr int COLS = 4;
+  static __device__ __forceinline__ void deposit(uint32_t taddr, const float* src) {
+    const float4 v = *reinterpret_cast<const float4*>(src);
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};" ::"r"(taddr),
+                 "r"(__float_as_uint(v.x)), "r"(__float_as_uint(v.y)), "r"(__float_as_uint(v.z)),
+                 "r"(__float_as_uint(v.w))
+                 : "memory");
+  }
+  static __device__ __forceinline__ void fetch(uint32_t taddr, float (&x)[4]) {
+    uint32_t a, b, c, d;
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(a), "=r"(b), "=r"(c), "=r"(d)
+        : "r"(taddr)
+        : "memory");
+    x[0] = __uint_as_float(a); x[1] = __uint_as_float(b); x[2] = __uint_as_float(c); x[3] = __uint_as_float(d);
+  }
+  static __device__ __forceinline__ void sts_quad(float* dst, const float (&x)[4]) {
+    *reinterpret_cast<float4*>(dst) = make_float4(x[0], x[1], x[2], x[3]);
+  }
+};
+template <> struct TmemCell<__nv_bfloat16> {
+  static constexpr int COLS = 2;
+  static __device__ __forceinline__ void deposit(uint32_t taddr, const __nv_bfloat16* src) {
+    const uint2 v = *reinterpret_cast<const uint2*>(src);
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x2.b32 [%0], {%1, %2};" ::"r"(taddr), "r"(v.x), "r"(v.y)
+                 : "memory");
+  }
+  static __device__ __forceinline__ void fetch(uint32_t taddr, float (&x)[4]) {
+    uint32_t a, b;
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x2.b32 {%0, %1}, [%2];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(a), "=r"(b)
+        : "r"(taddr)
+        : "memory");
+    x[0] = __uint_as_float(a << 16); x[1] = __uint_as_float(a & 0xFFFF0000u);
+    x[2] = __uint_as_float(b << 16); x[3] = __uint_as_float(b & 0xFFFF0000u);
+  }
+  static __device__ __forceinline__ void sts_quad(__nv_bfloat16* dst, const float (&x)[4]) {
+    uint2 t;
+    __nv_bfloat162 h;
+    h = __floats2bfloat162_rn(x[0], x[1]); t.x = *reinterpret_cast<uint32_t*>(&h);
+    h = __floats2bfloat162_rn(x[2], x[3]); t.y = *reinterpret_cast<uint32_t*>(&h);
+    *reinterpret_cast<uint2*>(dst) = t;
+  }
+};
+
+// Sum of worker k's own cell and its q drawn neighbours' cells of element group `cell0` (the
+// TMEM address of row 0's cell), own first, then draw order, each addition rounded.
+template <typename TH>
+__device__ __forceinline__ void tmem_gather(uint32_t cell0, int k, const int* nb, int q, float (&a)[4]) {
+  constexpr int CW = TmemCell<TH>::COLS;
+  TmemCell<TH>::fetch(cell0 + (uint32_t)(k * CW), a);
+  for (int j = 0; j < q; ++j) {
+    float t[4];
+    TmemCell<TH>::fetch(cell0 + (uint32_t)(nb[j] * CW), t);
+#pragma unroll
+    for (int x = 0; x < 4; ++x) a[x] = __fadd_rn(a[x], t[x]);
+  }
 }
 
-// BULK: the outputs leave through bulk stores from the ring slot (a third row holds the new theta)
-// instead of st.global from registers.
-struct SlotInfo { long long e0, lo, hi; int k; int pad; };   // what the producer must know to retire a slot
+// What the producer must know to send a finished slot out: the staged range starts at e0, whole
+// 16-byte pieces of the rows cover [sb, se); k < 0: a load item, nothing to send.
+struct SlotInfo { long long e0, sb, se; int k; int pad; };
 
-template <bool BULK>
+// Slot layout.  Load item: IN_ROWS rows of T theta elements.  Output item (one per worker):
+// [omega T floats | Delta T floats | (BULK) new theta T elements].
+// BULK: the outputs leave through bulk stores from the ring slot instead of st.global from
+// registers.
+template <typename TH, bool BULK>
 __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParams P) {
+  constexpr int EB = (int)sizeof(TH);
+  constexpr int CW = TmemCell<TH>::COLS;
+  constexpr int IN_ROWS = 8 / EB;                    // theta rows per load item
+  constexpr long long ALN = 16 / EB;                 // elements per 16 bytes of theta
   extern __shared__ __align__(128) unsigned char smem[];
   // [0,64) ring full, [64,128) ring empty (consumers done), [128,132) TMEM base address,
   // [192,448) per-slot retire information (BULK)
@@ -684,16 +744,19 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
   SlotInfo* sinfo = reinterpret_cast<SlotInfo*>(smem + 192);
   unsigned char* ring0 = smem + P.ring_off;
   unsigned char* meta0 = smem + P.meta_off;
+  TH* const theta = reinterpret_cast<TH*>(P.theta);
+  const TH* const theta_in = reinterpret_cast<const TH*>(P.theta_in);
   const int total = P.tile_prefix[P.m];
   const int R = P.ring, K = P.K, q = P.q, T = P.T;
   const int my_tiles = (int)blockIdx.x < total ? (total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
-  const int ntheta = (K + 1) / 2;           // theta items per tile (two rows each)
+  const int ntheta = (K + IN_ROWS - 1) / IN_ROWS;                  // load items per tile
+  const int nout = K;                                              // output items per tile
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
     for (int r = 0; r < R; ++r) {
       mbar_init(bars + 8 * r, 1);
-      mbar_init(bars + 64 + 8 * r, 512);
+      mbar_init(bars + 64 + 8 * r, 512);                 // every consumer thread arrives
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -728,7 +791,7 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
     int gi = 0;              // ring items requested so far
     bool ok = true;
     // BULK: item j is finished by the consumers -> send its results out of the slot.  One bulk
-    // group per item (an empty one for theta items) so that "all but the newest group have been
+    // group per item (an empty one for load items) so that "all but the newest group have been
     // read" means exactly "the slot about to be refilled is free".
     auto retire = [&](int j) -> bool {
       const int slot = j % R;
@@ -736,16 +799,13 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
       if (!__all_sync(0xffffffffu, fine)) return false;
       if (lane == 0) {
         const SlotInfo si = sinfo[slot];
-        if (si.k >= 0) {
-          const long long sb = (si.lo + 3) & ~3LL, se = si.hi & ~3LL;   // whole groups of 4 inside the tile
-          if (se > sb) {
-            const uint32_t src = smem_u32(ring0 + (size_t)slot * P.slot_stride) + (uint32_t)(sb - si.e0) * 4u;
-            const uint32_t nbytes = (uint32_t)(se - sb) * 4u;
-            const long long at = (long long)si.k * P.ld + sb;
-            asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(P.omega + at), "r"(src), "r"(nbytes) : "memory");
-            asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(P.delta + at), "r"(src + (uint32_t)T * 4u), "r"(nbytes) : "memory");
-            asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(P.theta + at), "r"(src + (uint32_t)T * 8u), "r"(nbytes) : "memory");
-          }
+        if (si.k >= 0 && si.se > si.sb) {
+          const uint32_t base = smem_u32(ring0 + (size_t)slot * P.slot_stride);
+          const uint32_t skip = (uint32_t)(si.sb - si.e0), n = (uint32_t)(si.se - si.sb);
+          const long long at = (long long)si.k * P.ld + si.sb;
+          asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(P.omega + at), "r"(base + skip * 4u), "r"(n * 4u) : "memory");
+          asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(P.delta + at), "r"(base + (uint32_t)T * 4u + skip * 4u), "r"(n * 4u) : "memory");
+          asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(theta + at), "r"(base + (uint32_t)T * 8u + skip * EB), "r"(n * EB) : "memory");
         }
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
       }
@@ -766,9 +826,9 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
       const long long e0 = (cb & ~(long long)(kAlign - 1)) + (long long)(w - pfx_lo) * T;
       long long run = P.ld - e0;
       if (run > T) run = T;
-      const uint32_t bytes = (uint32_t)run * 4u;
+      const long long lo = cb > e0 ? cb : e0, hi = ce < e0 + T ? ce : e0 + T;
       // tile descriptor + neighbour table into the meta ring (4 entries: the consumers are never
-      // more than a ring of items, i.e. less than one tile, behind)
+      // more than a ring of items, i.e. at most three tiles, behind)
       unsigned char* meta = meta0 + (size_t)(it & 3) * P.meta_stride;
       TileDesc* d = reinterpret_cast<TileDesc*>(meta);
       int* snb = reinterpret_cast<int*>(meta + sizeof(TileDesc));
@@ -779,12 +839,12 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
       __syncwarp();
       if (lane == 0) {
         d->e0 = e0;
-        d->lo = cb > e0 ? cb : e0;
-        d->hi = ce < e0 + T ? ce : e0 + T;
+        d->lo = lo;
+        d->hi = hi;
         d->comp = comp;
       }
       __syncwarp();
-      for (int item = 0; item < ntheta + K && ok; ++item, ++gi) {
+      for (int item = 0; item < ntheta + nout && ok; ++item, ++gi) {
         const int slot = gi % R;
         if (BULK) {
           if (gi >= R - 1) ok = retire(gi - (R - 1));       // consumers done with it; its stores go out
@@ -801,18 +861,24 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
           const uint32_t full = bars + 8 * slot;
           const uint32_t dst = smem_u32(ring0 + (size_t)slot * P.slot_stride);
           if (BULK) {
-            sinfo[slot].e0 = e0;
-            sinfo[slot].lo = cb > e0 ? cb : e0;
-            sinfo[slot].hi = ce < e0 + T ? ce : e0 + T;
-            sinfo[slot].k = item < ntheta ? -1 : item - ntheta;
+            SlotInfo si;
+            si.e0 = e0;
+            si.sb = (lo + ALN - 1) & ~(ALN - 1);
+            si.se = hi & ~(ALN - 1);
+            si.k = item < ntheta ? -1 : item - ntheta;
+            si.pad = 0;
+            sinfo[slot] = si;
           }
           if (item < ntheta) {
-            const int r0 = 2 * item, rows = (r0 + 1 < K) ? 2 : 1;
+            const int r0 = IN_ROWS * item;
+            const int rows = K - r0 < IN_ROWS ? K - r0 : IN_ROWS;
+            const uint32_t bytes = (uint32_t)run * EB;
             mbar_arrive_expect_tx(full, (uint32_t)rows * bytes);
-            bulk_load_row(dst, P.theta_in + (long long)r0 * P.ld + e0, bytes, full);
-            if (rows == 2) bulk_load_row(dst + (uint32_t)T * 4u, P.theta_in + (long long)(r0 + 1) * P.ld + e0, bytes, full);
+            for (int r = 0; r < rows; ++r)
+              bulk_load_row(dst + (uint32_t)r * (uint32_t)T * EB, theta_in + (long long)(r0 + r) * P.ld + e0, bytes, full);
           } else {
             const long long at = (long long)(item - ntheta) * P.ld + e0;
+            const uint32_t bytes = (uint32_t)run * 4u;
             mbar_arrive_expect_tx(full, 2u * bytes);
             bulk_load_row(dst, P.omega + at, bytes, full);
             bulk_load_row(dst + (uint32_t)T * 4u, P.delta + at, bytes, full);
@@ -832,6 +898,7 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
   } else {
     // -------------------------------------------------------------------- consumer warps (16)
     // lanes this warp reaches, and which of the four warps of that lane quarter it is
+    // (24 consumer warps were measured slower than 16)
     const int quarter = warp & 3, sub = (warp - 1) >> 2;
     const uint32_t tlane = tmem_base + ((uint32_t)(quarter * 32) << 16);
     const int ngroups = T / 512;                  // element groups of 128 x 4 per row
@@ -841,42 +908,41 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
       const unsigned char* meta = meta0 + (size_t)(it & 3) * P.meta_stride;
       const TileDesc* d = reinterpret_cast<const TileDesc*>(meta);
       const int* snb = reinterpret_cast<const int*>(meta + sizeof(TileDesc));
-      long long e0 = 0, lo = 0, hi = 0;
-      for (int item = 0; item < ntheta + K && ok; ++item, ++gi) {
+      long long e0 = 0, lo = 0, hi = 0, sb = 0, se = 0;
+      for (int item = 0; item < ntheta + nout && ok; ++item, ++gi) {
         const int slot = gi % R;
         bool fine = mbar_wait_bounded(bars + 8 * slot, (gi / R) & 1, P.status);
         ok = __all_sync(0xffffffffu, fine);
         if (!ok) break;
-        if (item == 0) { e0 = d->e0; lo = d->lo; hi = d->hi; }
-        float* row0 = reinterpret_cast<float*>(ring0 + (size_t)slot * P.slot_stride);
-        float* row1 = row0 + T;
-        float* row2 = row1 + T;   // BULK: the new theta
+        if (item == 0) {
+          e0 = d->e0; lo = d->lo; hi = d->hi;
+          sb = (lo + ALN - 1) & ~(ALN - 1);       // whole 16-byte pieces of theta inside the tile
+          se = hi & ~(ALN - 1);
+        }
+        unsigned char* const sbase = ring0 + (size_t)slot * P.slot_stride;
         if (item < ntheta) {
-          // deposit two theta rows into this thread's TMEM cells
-          const int r0 = 2 * item;
+          // deposit the theta rows of this item into this thread's TMEM cells
+          const int r0 = IN_ROWS * item;
+          const TH* rows_in = reinterpret_cast<const TH*>(sbase);
           for (int g = sub; g < ngroups; g += 4) {
             const int col = (g * 128 + quarter * 32 + lane) * 4;
-            float x[4];
-            ThetaTraits<float>::lds_quad(row0 + col, x);
-            tmem_store4(tlane + (uint32_t)((g * K + r0) * 4), x);
-            if (r0 + 1 < K) {
-              ThetaTraits<float>::lds_quad(row1 + col, x);
-              tmem_store4(tlane + (uint32_t)((g * K + r0 + 1) * 4), x);
-            }
+#pragma unroll
+            for (int r = 0; r < IN_ROWS; ++r)
+              if (r0 + r < K)
+                TmemCell<TH>::deposit(tlane + (uint32_t)((g * K + r0 + r) * CW), rows_in + (size_t)r * T + col);
           }
           asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         } else {
           const int k = item - ntheta;
+          float* row0 = reinterpret_cast<float*>(sbase);
+          float* row1 = row0 + T;
+          TH* row2 = reinterpret_cast<TH*>(row1 + T);      // BULK: the new theta
           for (int g = sub; g < ngroups; g += 4) {
             const int col = (g * 128 + quarter * 32 + lane) * 4;
             const long long e = e0 + col;
             float a[4], t[4];
-            tmem_load4(tlane + (uint32_t)((g * K + k) * 4), a);
-            for (int j = 0; j < q; ++j) {
-              tmem_load4(tlane + (uint32_t)((g * K + snb[k * q + j]) * 4), t);
-#pragma unroll
-              for (int x = 0; x < 4; ++x) a[x] = __fadd_rn(a[x], t[x]);
-            }
+            __syncwarp();                          // lanes that left the last group early rejoin
+            tmem_gather<TH>(tlane + (uint32_t)(g * K * CW), k, snb + k * q, q, a);
             if (e >= hi || e + 4 <= lo) continue;
 #pragma unroll
             for (int x = 0; x < 4; ++x)
@@ -885,24 +951,22 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
             const float4 D = *reinterpret_cast<const float4*>(row1 + col);
             float wv[4] = {W.x, W.y, W.z, W.w}, dv[4] = {D.x, D.y, D.z, D.w};
 #pragma unroll
-            for (int x = 0; x < 4; ++x) bmuf_filter<float>(a[x], wv[x], dv[x], t[x], P.eta, P.zeta);
+            for (int x = 0; x < 4; ++x) bmuf_filter<TH>(a[x], wv[x], dv[x], t[x], P.eta, P.zeta);
             const long long at = (long long)k * P.ld + e;
-            if (e >= lo && e + 4 <= hi) {
-              if (BULK) {
-                *reinterpret_cast<float4*>(row0 + col) = make_float4(wv[0], wv[1], wv[2], wv[3]);
-                *reinterpret_cast<float4*>(row1 + col) = make_float4(dv[0], dv[1], dv[2], dv[3]);
-                *reinterpret_cast<float4*>(row2 + col) = make_float4(t[0], t[1], t[2], t[3]);
-              } else {
-                __stcs(reinterpret_cast<float4*>(P.delta + at), make_float4(dv[0], dv[1], dv[2], dv[3]));
-                __stcs(reinterpret_cast<float4*>(P.omega + at), make_float4(wv[0], wv[1], wv[2], wv[3]));
-                __stcs(reinterpret_cast<float4*>(P.theta + at), make_float4(t[0], t[1], t[2], t[3]));
-              }
+            if (BULK && e >= sb && e + 4 <= se) {
+              *reinterpret_cast<float4*>(row0 + col) = make_float4(wv[0], wv[1], wv[2], wv[3]);
+              *reinterpret_cast<float4*>(row1 + col) = make_float4(dv[0], dv[1], dv[2], dv[3]);
+              TmemCell<TH>::sts_quad(row2 + col, t);
+            } else if (!BULK && e >= lo && e + 4 <= hi) {
+              __stcs(reinterpret_cast<float4*>(P.delta + at), make_float4(dv[0], dv[1], dv[2], dv[3]));
+              __stcs(reinterpret_cast<float4*>(P.omega + at), make_float4(wv[0], wv[1], wv[2], wv[3]));
+              ThetaTraits<TH>::stg_quad(theta + at, t);
             } else {
               for (int x = 0; x < 4; ++x) {
                 if (e + x >= lo && e + x < hi) {
                   P.delta[at + x] = dv[x];
                   P.omega[at + x] = wv[x];
-                  P.theta[at + x] = t[x];
+                  theta[at + x] = ThetaTraits<TH>::narrow(t[x]);
                 }
               }
             }
@@ -1536,45 +1600,54 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
   const long long cap = ctx->max_smem < ctx->smem_per_sm - 1024 ? ctx->max_smem : ctx->smem_per_sm - 1024;
   // Variant: flags bit 3 forces the shared-memory theta tile, bit 1 forces the tensor-memory tile
   // (bit 2: with bulk stores); with neither, the tensor-memory tile with bulk stores is used
-  // wherever it applies (fp32 theta, gossip-BMUF, 4 <= K <= 128) -- it is the faster one.
-  const bool tmem_ok = esz == 4 && bmuf && K >= 4 && K <= 128;
+  // wherever it applies (gossip-BMUF, 4 <= K <= 128) -- it is the faster one.
+  const int cw = esz == 4 ? 4 : 2;                       // TMEM columns per group of 4 elements
+  const bool tmem_ok = bmuf && K >= 4 && K <= 128;
   // (automatic choice only when the caller has not asked for anything specific to the
   // shared-memory tile: consumer threads, theta stages, or a tile width it cannot have)
   const bool auto_tmem = !(t.flags & 8) && tmem_ok && t.ncons == 0 && t.stages == 0 &&
-                         (t.T == 0 || (t.T % 512 == 0 && (t.T / 512) * K * 4 <= 512));
+                         (t.T == 0 || (t.T % 512 == 0 && (t.T / 512) * K * cw <= 512));
   const bool want_tmem = (t.flags & 2) || auto_tmem;
   if ((t.flags & 2) && !tmem_ok)
-    return fail(ctx, GBMUF_ERR_UNSUPPORTED, "the tensor-memory variant needs fp32 theta, BMUF mode and 4 <= K <= 128");
+    return fail(ctx, GBMUF_ERR_UNSUPPORTED, "the tensor-memory variant needs gossip-BMUF mode and 4 <= K <= 128");
   if (want_tmem) {
     const bool bulk = (t.flags & 2) ? (t.flags & 4) != 0 : true;
     const bool forced = (t.flags & 2) != 0;
-    // theta tile in tensor memory: K * (T/512) * 4 <= 512 columns; T a multiple of 512
-    int T = t.T ? t.T : 3584;
-    while (!t.T && T > 512 && (T / 512) * K * 4 > 512) T -= 512;
-    bool fits = T >= 512 && T % 512 == 0 && (T / 512) * K * 4 <= 512;
+    // theta tile in tensor memory: K * (T/512) * cw <= 512 columns; T a multiple of 512
+    // default width: measured best with 16 replicas (fp32: 3584 x 4 slots; bf16: 3072 x 6 slots)
+    int T = t.T ? t.T : (esz == 4 ? 3584 : 3072);
+    while (!t.T && T > 512 && (T / 512) * K * cw > 512) T -= 512;
+    bool fits = T >= 512 && T % 512 == 0 && (T / 512) * K * cw <= 512;
     if (!fits && (forced || t.T))
-      return fail(ctx, GBMUF_ERR_INVALID_ARG, "tensor-memory variant: tile_elems must be a multiple of 512 with K * tile_elems / 128 <= 512");
+      return fail(ctx, GBMUF_ERR_INVALID_ARG, "tensor-memory variant: tile_elems must be a multiple of 512 whose K rows fit 512 columns of tensor memory");
     if (fits) {
-      L.T = T; L.BW = 256; L.stages = 1; L.ncons = 512;
+      L.T = T; L.BW = 256; L.stages = 1;
+      L.ncons = 512;
       L.flags = (t.flags & 1) | 2 | (bulk ? 4 : 0);
       L.meta_off = 512;
       L.meta_stride = (uint32_t)(((long long)sizeof(TileDesc) + (long long)K * q * 4 + 127) / 128 * 128);
       L.ring_off = L.meta_off + 4 * L.meta_stride;
-      L.slot_stride = (uint32_t)((bulk ? 12 : 8) * T);
+      L.slot_stride = (uint32_t)((bulk ? 8 + esz : 8) * T);
+      // ring items per tile; the 4-entry descriptor ring needs the producer to stay within three
+      // tiles of the consumers, i.e. a ring no deeper than three tiles' worth of items
+      const int in_rows = 8 / esz;
+      const int per_tile = (K + in_rows - 1) / in_rows + K;
+      const int ring_cap = 3 * per_tile < kMaxRing ? 3 * per_tile : kMaxRing;
       // Ring depth: 4 slots of the default width measured best (3 starve the pipeline, 5 and more
       // put too much in flight; even counts did better than odd ones); narrower slots: more of them.
       int R = t.ring ? t.ring : (bulk ? 4 : 3);
       while (!t.ring && R > 2 && (long long)L.ring_off + (long long)R * L.slot_stride > cap) --R;
-      while (!t.ring && bulk && R + 2 <= 8 && (long long)R * L.slot_stride < 160 * 1024 &&
+      while (!t.ring && bulk && R + 2 <= ring_cap && (long long)R * L.slot_stride < 160 * 1024 &&
              (long long)L.ring_off + (long long)(R + 2) * L.slot_stride <= cap) R += 2;
-      const bool ring_fits = (long long)L.ring_off + (long long)R * L.slot_stride <= cap && R >= 2;
+      if (!t.ring && R > ring_cap) R = ring_cap;
+      const bool ring_fits = (long long)L.ring_off + (long long)R * L.slot_stride <= cap && R >= 2 && R <= ring_cap;
       if (!ring_fits && (forced || t.ring))
-        return fail(ctx, GBMUF_ERR_UNSUPPORTED, "tensor-memory variant: the ring does not fit shared memory");
+        return fail(ctx, GBMUF_ERR_UNSUPPORTED, "tensor-memory variant: the ring does not fit shared memory (or is deeper than three tiles)");
       if (ring_fits) {
         L.ring = R;
         L.smem = (uint32_t)(L.ring_off + (long long)R * L.slot_stride);
         int cols = 32;
-        while (cols < (T / 512) * K * 4) cols <<= 1;
+        while (cols < (T / 512) * K * cw) cols <<= 1;
         L.tmem_cols = cols;
         L.stage_stride = 0; L.nbr_off = 0; L.desc_off = 0;
         *out = L;
@@ -1684,13 +1757,18 @@ gbmuf_status launch_round(gbmuf_ctx* ctx, const gbmuf_config& cfg, const Launch&
   cudaError_t e;
   if (L.tmem_cols > 0) {
     TmemParams Q;
-    Q.theta_in = (const float*)theta; Q.theta = (float*)theta; Q.omega = omega; Q.delta = delta;
+    Q.theta_in = theta; Q.theta = theta; Q.omega = omega; Q.delta = delta;
     Q.off = off; Q.tile_prefix = prefix; Q.nbr = nbr; Q.status = status;
     Q.ld = ld; Q.K = cfg.K; Q.m = m; Q.q = cfg.q;
     Q.eta = P.eta; Q.zeta = P.zeta; Q.qp1 = P.qp1; Q.inv_qp1 = P.inv_qp1; Q.inv_exact = P.inv_exact;
     Q.T = L.T; Q.ring = L.ring; Q.ncols = L.tmem_cols;
     Q.ring_off = L.ring_off; Q.meta_off = L.meta_off; Q.meta_stride = L.meta_stride; Q.slot_stride = L.slot_stride;
-    auto kern = (L.flags & 4) ? sync_fused_tmem_kernel<true> : sync_fused_tmem_kernel<false>;
+    const bool bulk = (L.flags & 4) != 0, bf = cfg.theta_dtype != GBMUF_F32;
+    void (*kern)(const TmemParams);
+    if (bf)
+      kern = bulk ? sync_fused_tmem_kernel<__nv_bfloat16, true> : sync_fused_tmem_kernel<__nv_bfloat16, false>;
+    else
+      kern = bulk ? sync_fused_tmem_kernel<float, true> : sync_fused_tmem_kernel<float, false>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem);
     if (e != cudaSuccess) return cuda_fail(ctx, "cudaFuncSetAttribute", e);
     kern<<<grid, 544, L.smem, st>>>(Q);

@@ -450,15 +450,16 @@ def test_special_values_propagate_identically(dtype):
 
 
 @pytest.mark.parametrize("flags", [2, 6])          # 6: outputs leave through bulk stores
+@pytest.mark.parametrize("dtype", [0, 1])
 @pytest.mark.parametrize("K,p,q,tile,ring", [(16, 3, 2, 0, 0), (8, 2, 2, 2048, 4), (5, 2, 4, 1024, 3),
                                               (4, 1, 1, 512, 8), (16, 3, 6, 1024, 2), (32, 4, 3, 2048, 0)])
-def test_tensor_memory_variant(K, p, q, tile, ring, flags):
+def test_tensor_memory_variant(K, p, q, tile, ring, dtype, flags):
     """The variant that parks the theta tile in tensor memory gives the same bits: several tiles
-    per CTA, ragged component edges, masks, odd K (a half-filled last theta item)."""
+    per CTA, ragged component edges, masks, odd K (a partly filled last theta item)."""
     offsets = (0, 100_003, 100_004, 350_001, 777_777)
-    case = Case(K=K, offsets=offsets, p=p, q=q, eta=0.875, zeta=1.0, dtype=0, seed=K + q)
+    case = Case(K=K, offsets=offsets, p=p, q=q, eta=0.875, zeta=1.0, dtype=dtype, seed=K + q)
     masks = [None, [1, 0, 1, 1], None]
-    run(case, random_theta0(case.N, seed=K, dtype=0), rounds=3, sigma=5e-2, masks=masks,
+    run(case, random_theta0(case.N, seed=K, dtype=dtype), rounds=3, sigma=5e-2, masks=masks,
         tuning=dict(tile_elems=tile, ring_slots=ring, flags=flags), check_nbr=False)
 
 
@@ -470,9 +471,9 @@ def test_tensor_memory_variant_is_refused_where_it_does_not_apply():
         g.set_tuning(flags=2)                      # fewer than 4 workers
     assert e.value.status == binding.ERR_UNSUPPORTED
     g.destroy()
-    thb = torch.zeros((8, 1024), dtype=torch.bfloat16, device=dev)
-    f = torch.zeros((8, 1024), device=dev)
-    g = binding.Gbmuf(thb, f, f.clone(), K=8, N=1024, ld=1024, p=1, q=1, eta=0.9, zeta=1.0, theta_dtype=1)
+    th = torch.zeros((8, 1024), device=dev)
+    g = binding.Gbmuf(th, th.clone(), th.clone(), K=8, N=1024, ld=1024, p=1, q=1, eta=0.9, zeta=1.0,
+                      mode=binding.MODE_MA)
     with pytest.raises(binding.GbmufError):
-        g.set_tuning(flags=2)                      # bf16 theta
+        g.set_tuning(flags=6)                      # gossip-MA
     g.destroy()
