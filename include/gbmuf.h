@@ -158,6 +158,17 @@ gbmuf_status gbmuf_device_status(gbmuf_ctx* ctx, void* stream, int32_t* out);
  * fully usable.  No fault, trap or unbounded loop is involved. */
 gbmuf_status gbmuf_selftest_wait_timeout(gbmuf_ctx* ctx, void* stream, double* seconds_out);
 
+/* Self-test of the averaging division.  Algorithm 1's averaging line divides a sum by q+1; the
+ * kernels compute that quotient for a small integer divisor that is not a power of two as
+ * q0 = RN(s * RN(1/b)), r = fma(-b, q0, s), RN(q0 + r * RN(1/b)) when the exponent of s is in the
+ * middle range, and with the division instruction sequence otherwise.  The result must equal the
+ * IEEE-754 quotient rounded to nearest even in every bit.  This call evaluates both over ALL 2^32
+ * bit patterns of s for the given divisor (2..256) and writes the number of patterns whose
+ * results differ to *mismatches_out (host) and the smallest such pattern to *first_bad_out (host,
+ * may be NULL; 0xFFFFFFFF if none).  Synchronises the stream.  Errors: INVALID_ARG, CUDA. */
+gbmuf_status gbmuf_selftest_divide(gbmuf_ctx* ctx, int32_t divisor, void* stream,
+                                   uint64_t* mismatches_out, uint32_t* first_bad_out);
+
 /* Launch shape of the fused kernel (one persistent CTA per SM).  Any argument may be 0 to keep
  * the built-in choice.  Two variants exist.  (a) theta tile in tensor memory, outputs through bulk
  * stores: chosen automatically in gossip-BMUF mode with 4 <= K <= 128; tile_elems must then be a

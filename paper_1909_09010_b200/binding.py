@@ -24,7 +24,7 @@ EXPORTS = ["gbmuf_create", "gbmuf_set_partition", "gbmuf_init", "gbmuf_local_per
            "gbmuf_sync_round", "gbmuf_get_neighbors", "gbmuf_final_average", "gbmuf_device_status",
            "gbmuf_set_tuning", "gbmuf_get_launch_info", "gbmuf_last_error", "gbmuf_destroy",
            "gbmuf_sync_round_noalloc", "gbmuf_sync_round_host", "gbmuf_local_adagrad",
-           "gbmuf_selftest_wait_timeout", "gbmuf_peer_create", "gbmuf_peer_set_partition",
+           "gbmuf_selftest_wait_timeout", "gbmuf_selftest_divide", "gbmuf_peer_create", "gbmuf_peer_set_partition",
            "gbmuf_peer_sync_round", "gbmuf_peer_device_status", "gbmuf_peer_destroy"]
 
 
@@ -75,6 +75,7 @@ def lib() -> ctypes.CDLL:
                                            ctypes.POINTER(i32)]
     L.gbmuf_sync_round_host.argtypes = [ctypes.POINTER(Config), vp, vp, vp, i32, vp, vp, u64, i64]
     L.gbmuf_selftest_wait_timeout.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_double)]
+    L.gbmuf_selftest_divide.argtypes = [vp, i32, vp, ctypes.POINTER(u64), ctypes.POINTER(ctypes.c_uint32)]
     L.gbmuf_peer_create.argtypes = [ctypes.POINTER(Config), i32, vp, vp, vp, ctypes.POINTER(vp)]
     L.gbmuf_peer_set_partition.argtypes = [vp, i32, vp, vp]
     L.gbmuf_peer_sync_round.argtypes = [vp, u64, vp, i32, vp]
@@ -259,6 +260,14 @@ class Gbmuf:
         sec = ctypes.c_double(0.0)
         self._check(lib().gbmuf_selftest_wait_timeout(self._h, _stream(stream), ctypes.byref(sec)))
         return sec.value
+
+    def selftest_divide(self, divisor: int, stream=None) -> tuple[int, int]:
+        """Compares the kernels' averaging division with the plain division over all 2^32
+        dividends; returns (number of differing patterns, smallest differing pattern)."""
+        bad, first = ctypes.c_uint64(0), ctypes.c_uint32(0)
+        self._check(lib().gbmuf_selftest_divide(self._h, divisor, _stream(stream), ctypes.byref(bad),
+                                                ctypes.byref(first)))
+        return bad.value, first.value
 
     def set_tuning(self, consumer_threads=0, tile_elems=0, theta_stages=0, ring_slots=0, flags=0):
         self._check(lib().gbmuf_set_tuning(self._h, consumer_threads, tile_elems, theta_stages,

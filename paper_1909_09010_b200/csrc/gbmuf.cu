@@ -23,6 +23,7 @@
 #include <cstring>
 #include <new>
 #include <string>
+#include <type_traits>
 #include <vector>
 
 #include "gbmuf.h"
@@ -344,6 +345,41 @@ struct SyncParams {
   uint32_t ring_off, slot_stride;             // ring slot: [omega row T floats | Delta row T floats]
 };
 
+// The division of the gossip average, s / (q+1), for four elements.  The result is that of the
+// IEEE-754 division rounded to nearest even, bit for bit, for every input; only the route differs:
+//  - q+1 a power of two: multiplying by 1/(q+1) is exact;
+//  - otherwise, for the small integer divisor b = q+1 and y = RN(1/b): q0 = RN(s*y), the exact
+//    residual r = fma(-b, q0, s), then RN(q0 + r*y) (Markstein's correction step).  It is taken
+//    only when the exponent of s is in the middle range, where no intermediate can overflow,
+//    underflow or be subnormal; zeros, subnormals, huge values, infinities and NaNs go through the
+//    division instruction sequence.  gbmuf_selftest_divide compares this routine with the plain
+//    division over all 2^32 bit patterns for a given divisor.
+// Costs 3 arithmetic instructions per element instead of about 10; gossip-MA with q+1 = 3 was
+// limited by the divide.
+// Exponent test: the result has one of its two top bits set iff the biased exponent of s is
+// outside [64, 191], i.e. unless 2^-63 <= |s| < 2^65; results of several values may be OR-ed.
+__device__ __forceinline__ uint32_t outside_mid_range(float s) {
+  return (__float_as_uint(s) & 0x7F800000u) - 0x20000000u;
+}
+__device__ __forceinline__ float divide_corrected(float s, float b, float y) {
+  const float q0 = __fmul_rn(s, y);
+  const float r = __fmaf_rn(-b, q0, s);
+  return __fmaf_rn(r, y, q0);
+}
+__device__ __forceinline__ void average_divide(float (&a)[4], float b, float y, int y_exact) {
+  if (y_exact) {
+#pragma unroll
+    for (int x = 0; x < 4; ++x) a[x] = __fmul_rn(a[x], y);
+  } else if (!((outside_mid_range(a[0]) | outside_mid_range(a[1]) | outside_mid_range(a[2]) |
+                outside_mid_range(a[3])) & 0xC0000000u)) {
+#pragma unroll
+    for (int x = 0; x < 4; ++x) a[x] = divide_corrected(a[x], b, y);
+  } else {
+#pragma unroll
+    for (int x = 0; x < 4; ++x) a[x] = __fdiv_rn(a[x], b);
+  }
+}
+
 // Block-momentum filter for one element (Algorithm 1: G, Delta, omega, theta lines).  The
 // block-start value is recomputed from the pre-round omega and Delta.
 template <typename TH>
@@ -510,38 +546,65 @@ sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_th
     if (!bmuf) {
       // gossip-MA: theta <- average.  No omega / Delta stream paces the workers, so each thread
       // walks all workers for its group of elements; unrolled so that the shared-memory loads
-      // and divides of several workers overlap.
+      // and the arithmetic of several workers overlap.
       // With more threads than element groups the workers are split between thread groups:
       // thread c takes group c % nv for workers c / nv, c / nv + kg, ...
-      const int kg = P.ncons > nv ? P.ncons / nv : 1;
-      const int k_first = P.ncons > nv ? c / nv : 0;
-      for (int v = P.ncons > nv ? c - k_first * nv : c; v < nv && k_first < kg; v += P.ncons) {
-        const int col = v * VEC;
-        const long long e = e0 + col;
-        if (e >= hi || e + VEC <= lo) continue;
-        const int b = col >> P.bw_shift, cin = col & P.bw_mask;
-        const int boxbase = b * box_elems + cin;
-        const bool whole = e >= lo && e + VEC <= hi;
+      // The division (see average_divide) is kept free of branches inside the loop, which is
+      // what lets the unrolled workers overlap: a pass either multiplies by an exact reciprocal
+      // (DIV 0), or takes the corrected-product route for every element while OR-ing the exponent
+      // tests (DIV 1), or divides plainly (DIV 2).  If a DIV 1 pass met a sum outside the middle
+      // range, the thread repeats its share of the tile with DIV 2 from the still-staged theta,
+      // overwriting what it stored.
+      // Each thread takes 16 bytes of theta per row here: 4 fp32 or 8 bf16 elements.
+      constexpr int MV = ThetaTraits<TH>::VEC;
+      const int nvm = P.T / MV;
+      const int kg = P.ncons > nvm ? P.ncons / nvm : 1;
+      const int k_first = P.ncons > nvm ? c / nvm : 0;
+      auto ma_pass = [&](auto div_tag) -> bool {
+        constexpr int DIV = decltype(div_tag)::value;
+        uint32_t oor = 0;
+        for (int v = P.ncons > nvm ? c - k_first * nvm : c; v < nvm && k_first < kg; v += P.ncons) {
+          const int col = v * MV;
+          const long long e = e0 + col;
+          if (e >= hi || e + MV <= lo) continue;
+          const int b = col >> P.bw_shift, cin = col & P.bw_mask;
+          const int boxbase = b * box_elems + cin;
+          const bool whole = e >= lo && e + MV <= hi;
 #pragma unroll 4
-        for (int k = k_first; k < P.K; k += kg) {
-          float a[VEC], t[VEC];
-          ThetaTraits<TH>::lds_quad(sth + boxbase + k * BW, a);
-          for (int j = 0; j < q; ++j) {
-            ThetaTraits<TH>::lds_quad(sth + boxbase + snb[k * q + j] * BW, t);
+          for (int k = k_first; k < P.K; k += kg) {
+            float a[MV], t[MV];
+            ThetaTraits<TH>::lds(sth + boxbase + k * BW, a);
+            for (int j = 0; j < q; ++j) {
+              ThetaTraits<TH>::lds(sth + boxbase + snb[k * q + j] * BW, t);
 #pragma unroll
-            for (int x = 0; x < VEC; ++x) a[x] = __fadd_rn(a[x], t[x]);
-          }
+              for (int x = 0; x < MV; ++x) a[x] = __fadd_rn(a[x], t[x]);
+            }
 #pragma unroll
-          for (int x = 0; x < VEC; ++x)
-            a[x] = P.inv_exact ? __fmul_rn(a[x], P.inv_qp1) : __fdiv_rn(a[x], P.qp1);
-          const long long at = (long long)k * P.ld + e;
-          if (whole) {
-            ThetaTraits<TH>::stg_quad(theta + at, a);
-          } else {
-            for (int x = 0; x < VEC; ++x)
-              if (e + x >= lo && e + x < hi) theta[at + x] = ThetaTraits<TH>::narrow(a[x]);
+            for (int x = 0; x < MV; ++x) {
+              if (DIV == 0) {
+                a[x] = __fmul_rn(a[x], P.inv_qp1);
+              } else if (DIV == 1) {
+                oor |= outside_mid_range(a[x]);
+                a[x] = divide_corrected(a[x], P.qp1, P.inv_qp1);
+              } else {
+                a[x] = __fdiv_rn(a[x], P.qp1);
+              }
+            }
+            const long long at = (long long)k * P.ld + e;
+            if (whole) {
+              ThetaTraits<TH>::stg(theta + at, a);
+            } else {
+              for (int x = 0; x < MV; ++x)
+                if (e + x >= lo && e + x < hi) theta[at + x] = ThetaTraits<TH>::narrow(a[x]);
+            }
           }
         }
+        return (oor & 0xC0000000u) != 0;
+      };
+      if (P.inv_exact) {
+        ma_pass(std::integral_constant<int, 0>{});
+      } else if (ma_pass(std::integral_constant<int, 1>{})) {
+        ma_pass(std::integral_constant<int, 2>{});
       }
       mbar_arrive(bars + kBarThetaEmpty + 8 * s);
       continue;
@@ -571,9 +634,7 @@ sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_th
 #pragma unroll
           for (int x = 0; x < VEC; ++x) a[x] = __fadd_rn(a[x], t[x]);
         }
-#pragma unroll
-        for (int x = 0; x < VEC; ++x)
-          a[x] = P.inv_exact ? __fmul_rn(a[x], P.inv_qp1) : __fdiv_rn(a[x], P.qp1);
+        average_divide(a, P.qp1, P.inv_qp1, P.inv_exact);
         const long long at = (long long)k * P.ld + e;
         const bool whole = e >= lo && e + VEC <= hi;
         if (!bmuf) {                                       // gossip-MA: theta <- average
@@ -944,9 +1005,7 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
             __syncwarp();                          // lanes that left the last group early rejoin
             tmem_gather<TH>(tlane + (uint32_t)(g * K * CW), k, snb + k * q, q, a);
             if (e >= hi || e + 4 <= lo) continue;
-#pragma unroll
-            for (int x = 0; x < 4; ++x)
-              a[x] = P.inv_exact ? __fmul_rn(a[x], P.inv_qp1) : __fdiv_rn(a[x], P.qp1);
+            average_divide(a, P.qp1, P.inv_qp1, P.inv_exact);
             const float4 W = *reinterpret_cast<const float4*>(row0 + col);
             const float4 D = *reinterpret_cast<const float4*>(row1 + col);
             float wv[4] = {W.x, W.y, W.z, W.w}, dv[4] = {D.x, D.y, D.z, D.w};
@@ -982,6 +1041,37 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
   __syncthreads();
   if (warp == 0) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)P.ncols) : "memory");
+  }
+}
+
+// Self-test of average_divide: runs its correction route (never the power-of-two shortcut) and
+// the plain division over all 2^32 bit patterns of the dividend, four consecutive patterns per
+// call as in the round kernels, and counts the patterns whose results differ in any bit.
+__global__ void __launch_bounds__(256) divide_selftest_kernel(float b, float y, unsigned long long* mismatches,
+                                                              unsigned int* first_bad) {
+  const unsigned long long nquads = 1ull << 30;
+  unsigned int bad = 0, first = 0xFFFFFFFFu;
+  for (unsigned long long qd = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; qd < nquads;
+       qd += (unsigned long long)gridDim.x * blockDim.x) {
+    float a[4], ref[4];
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+      a[x] = __uint_as_float((unsigned int)(qd * 4 + x));
+      ref[x] = __fdiv_rn(a[x], b);
+    }
+    average_divide(a, b, y, 0);
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+      if (__float_as_uint(a[x]) != __float_as_uint(ref[x])) {
+        ++bad;
+        const unsigned int pat = (unsigned int)(qd * 4 + x);
+        if (pat < first) first = pat;
+      }
+    }
+  }
+  if (bad) {
+    atomicAdd(mismatches, (unsigned long long)bad);
+    atomicMin(first_bad, first);
   }
 }
 
@@ -1439,9 +1529,7 @@ __global__ void __launch_bounds__(1024, 1) peer_round_kernel(const PeerParams P)
 #pragma unroll
         for (int x = 0; x < VEC; ++x) a[x] = __fadd_rn(a[x], t[x]);
       }
-#pragma unroll
-      for (int x = 0; x < VEC; ++x)
-        a[x] = P.inv_exact ? __fmul_rn(a[x], P.inv_qp1) : __fdiv_rn(a[x], P.qp1);
+      average_divide(a, P.qp1, P.inv_qp1, P.inv_exact);
       if (!bmuf) {
         if (whole) {
           ThetaTraits<TH>::stg_quad(out + e, a);
@@ -1708,8 +1796,11 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
   } else {
     int n = (L.T / 4 + 31) / 32 * 32;          // one quad per thread and row, within 128..992
     L.ncons = n < 128 ? 128 : n > 992 ? 992 : n;
-    if (!bmuf && L.T / 4 >= 32 && L.T / 4 <= 496)
-      L.ncons = (L.T / 4) * (992 / (L.T / 4));  // gossip-MA: thread groups share out the workers
+    if (!bmuf) {                               // gossip-MA: 16 bytes of theta per thread and row,
+      const int per = L.T / (16 / esz);        // and thread groups that share out the workers
+      if (per >= 32 && per <= 496) L.ncons = per * (992 / per);
+      else { n = (per + 31) / 32 * 32; L.ncons = n < 128 ? 128 : n > 992 ? 992 : n; }
+    }
   }
   *out = L;
   return GBMUF_OK;
@@ -2172,6 +2263,35 @@ gbmuf_status gbmuf_selftest_wait_timeout(gbmuf_ctx* ctx, void* stream, double* s
   if (e != cudaSuccess) return cuda_fail(ctx, "wait-timeout self-test", e);
   if (seconds_out) *seconds_out = ms / 1e3;
   if (ret != 2) return fail(ctx, GBMUF_ERR_BAD_STATE, "the self-test wait did not expire as it should");
+  return GBMUF_OK;
+}
+
+gbmuf_status gbmuf_selftest_divide(gbmuf_ctx* ctx, int32_t divisor, void* stream,
+                                   uint64_t* mismatches_out, uint32_t* first_bad_out) {
+  if (!ctx) return GBMUF_ERR_INVALID_ARG;
+  if (!mismatches_out) return fail(ctx, GBMUF_ERR_INVALID_ARG, "mismatches_out must not be NULL");
+  if (divisor < 2 || divisor > 256)
+    return fail(ctx, GBMUF_ERR_INVALID_ARG, "divisor must be in 2..256");
+  DeviceGuard guard(ctx->cfg.device);
+  if (!guard.ok) return fail(ctx, GBMUF_ERR_CUDA, "cudaSetDevice failed");
+  cudaStream_t st = (cudaStream_t)stream;
+  unsigned long long* d_buf = nullptr;             // [0] mismatches, [1] first bad pattern (low word)
+  cudaError_t e = cudaMalloc(&d_buf, 2 * sizeof(unsigned long long));
+  const unsigned long long init[2] = {0ull, 0xFFFFFFFFull};
+  if (e == cudaSuccess) e = cudaMemcpyAsync(d_buf, init, sizeof(init), cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess) {
+    const float b = (float)divisor;
+    divide_selftest_kernel<<<ctx->num_sms * 8, 256, 0, st>>>(b, 1.0f / b, d_buf,
+                                                             reinterpret_cast<unsigned int*>(d_buf + 1));
+    e = cudaGetLastError();
+  }
+  unsigned long long res[2] = {0ull, 0ull};
+  if (e == cudaSuccess) e = cudaMemcpyAsync(res, d_buf, sizeof(res), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  cudaFree(d_buf);
+  if (e != cudaSuccess) return cuda_fail(ctx, "divide self-test", e);
+  *mismatches_out = (uint64_t)res[0];
+  if (first_bad_out) *first_bad_out = (uint32_t)(res[1] & 0xFFFFFFFFull);
   return GBMUF_OK;
 }
 

@@ -400,8 +400,9 @@ def test_expired_wait_is_reported_not_hung():
         pr.close()
 
 
+@pytest.mark.parametrize("mode", [binding.MODE_BMUF, binding.MODE_MA])
 @pytest.mark.parametrize("dtype", [0, 1])
-def test_special_values_propagate_identically(dtype):
+def test_special_values_propagate_identically(dtype, mode):
     """Denormals (no flush-to-zero), signed zeros, infinities, NaN and extreme magnitudes go
     through the round as IEEE arithmetic dictates: bit-equal with the oracle wherever the result
     is not NaN, NaN exactly where the oracle has NaN."""
@@ -415,7 +416,7 @@ def test_special_values_propagate_identically(dtype):
     theta0[1001:1200] = (g.integers(-2000, 2000, size=199) * 1e-42).astype(np.float32)   # a denormal stretch
     if dtype == 1:
         theta0 = oracle.f32_to_bf16(theta0)
-    case = Case(K=K, offsets=offsets, p=2, q=2, eta=0.9, zeta=1.0, dtype=dtype, seed=3)
+    case = Case(K=K, offsets=offsets, p=2, q=2, eta=0.9, zeta=1.0, dtype=dtype, seed=3, mode=mode)
     pr = Pair(case, theta0)
     try:
         drift = (g.standard_normal((K, N)) * 0.05).astype(np.float32)
@@ -444,7 +445,11 @@ def test_special_values_propagate_identically(dtype):
             d = st.delta[np.isfinite(st.delta)]
             saw_denormal = saw_denormal or bool((np.abs(d[d != 0]) < 1.1754944e-38).any())
         assert np.isnan(st.theta if dtype == 0 else oracle.bf16_to_f32(st.theta)).any()
-        assert saw_denormal or dtype == 1, "the test never produced a denormal Delta"
+        if mode == binding.MODE_BMUF:
+            assert saw_denormal or dtype == 1, "the test never produced a denormal Delta"
+        elif dtype == 0:
+            t = st.theta[np.isfinite(st.theta)]
+            assert (np.abs(t[t != 0]) < 1.1754944e-38).any(), "no denormal average was produced"
     finally:
         pr.close()
 
@@ -461,6 +466,23 @@ def test_tensor_memory_variant(K, p, q, tile, ring, dtype, flags):
     masks = [None, [1, 0, 1, 1], None]
     run(case, random_theta0(case.N, seed=K, dtype=dtype), rounds=3, sigma=5e-2, masks=masks,
         tuning=dict(tile_elems=tile, ring_slots=ring, flags=flags), check_nbr=False)
+
+
+def test_averaging_division_equals_the_ieee_division_for_every_dividend():
+    """The kernels divide the gossip sum by q+1 through a multiply and a residual correction;
+    for every divisor they can meet (q+1 <= 65) and some beyond, all 2^32 dividends -- zeros,
+    subnormals, infinities and NaNs included -- give the bits of the plain division."""
+    dev = torch.device("cuda:0")
+    th = torch.zeros((2, 1024), device=dev)
+    g = binding.Gbmuf(th, th.clone(), th.clone(), K=2, N=1024, ld=1024, p=1, q=1, eta=0.9, zeta=1.0)
+    try:
+        for b in list(range(2, 66)) + [96, 100, 127, 129, 255, 256]:
+            bad, first = g.selftest_divide(b)
+            assert bad == 0, f"divisor {b}: {bad} dividends differ, first pattern {first:#010x}"
+        with pytest.raises(binding.GbmufError):
+            g.selftest_divide(1)
+    finally:
+        g.destroy()
 
 
 def test_tensor_memory_variant_is_refused_where_it_does_not_apply():
