@@ -1200,69 +1200,186 @@ __global__ void clip_scale_kernel(const double* partial, int K, int nblk, float 
   scale[k] = __fdiv_rn(clip_norm, norm > clip_norm ? norm : clip_norm);
 }
 
+// The element-wise Adagrad update as a streaming kernel: 20 bytes per replica-parameter (fp32
+// theta) and nothing else, so it is built like the fused round: persistent CTAs, a producer warp
+// that has the copy engine fetch [gradient | accumulator | theta] chunks of one worker's row into a
+// ring of shared-memory slots, 16 consumer warps that update accumulator and theta inside the slot,
+// and bulk stores that send the two rows back.  Chunks are T consecutive elements of one row;
+// consecutive CTAs take consecutive chunks.  Rows are read up to the padded stride (a multiple of
+// 16 bytes); stores cover whole 16-byte pieces below N, the few elements after the last whole
+// piece are stored by the thread that computed them, and the padding is never written.
+struct AdagradParams {
+  void* theta;
+  const float* grad;
+  float* accum;
+  const float* scale;      // [K] clip factor per worker, or NULL
+  int32_t* status;
+  long long N, ld;
+  int K, T, ring, chunks_per_row, groups;   // groups: consumer thread groups (1, 2 or 4)
+  uint32_t ring_off, slot_stride;
+  float lr, eps;
+  ClipRanges R;
+};
+
+// What producer and consumers share about the chunk in a slot: it starts at element e0 of worker
+// k's row and ends before hi (<= N); whole 16-byte pieces end at se; `where` places it relative
+// to the clip ranges (0 outside all, 1 inside one, 2 mixed) and sc is the worker's clip factor.
+struct AdagradSlot { long long e0, hi, se; int k; int where; float sc; int pad; };
+
 template <typename TH>
-__global__ void __launch_bounds__(256) adagrad_kernel(TH* theta, const float* grad, float* accum,
-                                                      int K, long long N, long long ld, float lr,
-                                                      float eps, const float* scale, ClipRanges R) {
-  constexpr int VEC = ThetaTraits<TH>::VEC;
-  const long long nvec = (N + VEC - 1) / VEC;
-  const int k = blockIdx.y;                 // one grid row per worker
-  for (long long iv = (long long)blockIdx.x * blockDim.x + threadIdx.x; iv < nvec;
-       iv += (long long)gridDim.x * blockDim.x) {
-    const long long e = iv * VEC;
-    const long long at = (long long)k * ld + e;
-    const int n = N - e < VEC ? (int)(N - e) : VEC;
-    const float sc = scale ? scale[k] : 1.0f;
-    float th[VEC], g[VEC], a[VEC];
-    if (n == VEC) {
-      ThetaTraits<TH>::lds(theta + at, th);
-#pragma unroll
-      for (int h = 0; h < VEC / 4; ++h) {
-        const float4 gv = __ldcs(reinterpret_cast<const float4*>(grad + at) + h);
-        const float4 av = __ldcs(reinterpret_cast<const float4*>(accum + at) + h);
-        g[4 * h] = gv.x; g[4 * h + 1] = gv.y; g[4 * h + 2] = gv.z; g[4 * h + 3] = gv.w;
-        a[4 * h] = av.x; a[4 * h + 1] = av.y; a[4 * h + 2] = av.z; a[4 * h + 3] = av.w;
-      }
-    } else {
-      for (int x = 0; x < n; ++x) {
-        th[x] = ThetaTraits<TH>::widen(theta[at + x]);
-        g[x] = grad[at + x];
-        a[x] = accum[at + x];
-      }
+__global__ void __launch_bounds__(544, 1) adagrad_stream_kernel(const AdagradParams P) {
+  constexpr int EB = (int)sizeof(TH);
+  constexpr long long ALN = 16 / EB;                 // elements per 16 bytes of theta
+  extern __shared__ __align__(128) unsigned char smem[];
+  // [0,64) slot full, [64,128) slot done (consumers), [128,512) per-slot chunk descriptors
+  const uint32_t bars = smem_u32(smem);
+  AdagradSlot* sinfo = reinterpret_cast<AdagradSlot*>(smem + 128);
+  unsigned char* ring0 = smem + P.ring_off;
+  TH* const theta = reinterpret_cast<TH*>(P.theta);
+  const int R = P.ring, T = P.T;
+  const long long total = (long long)P.chunks_per_row * P.K;
+  const int my_chunks = (long long)blockIdx.x < total
+                            ? (int)((total - (long long)blockIdx.x + (long long)gridDim.x - 1) / (long long)gridDim.x)
+                            : 0;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int r = 0; r < R; ++r) {
+      mbar_init(bars + 8 * r, 1);
+      mbar_init(bars + 64 + 8 * r, 512 / P.groups);      // every thread of one consumer group arrives
     }
-    // where the vector lies relative to the clip ranges: 0 outside all, 1 inside one, 2 straddling
-    int where = 0;
-    if (scale) {
-      for (int r = 0; r < R.n; ++r) {
-        if (e >= R.begin[r] && e + VEC <= R.end[r]) where = 1;
-        else if (e < R.end[r] && e + VEC > R.begin[r] && where == 0) where = 2;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer warp
+    bool ok = true;
+    // chunk j is finished by the consumers -> send accumulator and theta out of the slot.  One
+    // bulk group per chunk, so that "all but the newest group have been read" means exactly
+    // "the slot about to be refilled is free".
+    auto retire = [&](int j) -> bool {
+      const int slot = j % R;
+      bool fine = mbar_wait_bounded(bars + 64 + 8 * slot, (j / R) & 1, P.status);
+      if (!__all_sync(0xffffffffu, fine)) return false;
+      if (lane == 0) {
+        const AdagradSlot si = sinfo[slot];
+        if (si.se > si.e0) {
+          const uint32_t base = smem_u32(ring0 + (size_t)slot * P.slot_stride);
+          const uint32_t n = (uint32_t)(si.se - si.e0);
+          const long long at = (long long)si.k * P.ld + si.e0;
+          asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(P.accum + at), "r"(base + (uint32_t)T * 4u), "r"(n * 4u) : "memory");
+          asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(theta + at), "r"(base + (uint32_t)T * 8u), "r"(n * EB) : "memory");
+        }
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
       }
+      __syncwarp();
+      return true;
+    };
+    // this CTA's chunks are w = blockIdx.x + it * gridDim.x: keep (row, chunk in row) incrementally
+    int k = (int)(blockIdx.x / (unsigned)P.chunks_per_row);
+    int cin = (int)(blockIdx.x % (unsigned)P.chunks_per_row);
+    const int dk = (int)(gridDim.x / (unsigned)P.chunks_per_row), dc = (int)(gridDim.x % (unsigned)P.chunks_per_row);
+    float sc = (P.scale && lane == 0 && my_chunks > 0) ? __ldg(P.scale + k) : 1.0f;
+    int it = 0;
+    for (; it < my_chunks && ok; ++it) {
+      const long long e0 = (long long)cin * T;
+      long long run = P.ld - e0;                         // a row ends at ld: never read past it
+      if (run > T) run = T;
+      const long long hi = e0 + T < P.N ? e0 + T : P.N;
+      const int slot = it % R;
+      if (it >= R - 1) ok = retire(it - (R - 1));        // consumers done with it; its stores go out
+      if (!ok) break;
+      if (it >= R && lane == 0)                          // the slot's own stores have read it
+        asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) {
+        AdagradSlot si;
+        si.e0 = e0; si.hi = hi; si.se = hi & ~(ALN - 1); si.k = k; si.where = 0; si.sc = sc; si.pad = 0;
+        if (P.scale) {
+          for (int r = 0; r < P.R.n; ++r) {
+            if (e0 >= P.R.begin[r] && hi <= P.R.end[r]) si.where = 1;
+            else if (e0 < P.R.end[r] && hi > P.R.begin[r] && si.where == 0) si.where = 2;
+          }
+        }
+        sinfo[slot] = si;
+        const uint32_t full = bars + 8 * slot;
+        const uint32_t dst = smem_u32(ring0 + (size_t)slot * P.slot_stride);
+        const long long at = (long long)k * P.ld + e0;
+        mbar_arrive_expect_tx(full, (uint32_t)run * (8u + EB));
+        bulk_load_row(dst, P.grad + at, (uint32_t)run * 4u, full);
+        bulk_load_row(dst + (uint32_t)T * 4u, P.accum + at, (uint32_t)run * 4u, full);
+        bulk_load_row(dst + (uint32_t)T * 8u, theta + at, (uint32_t)run * EB, full);
+      }
+      // next chunk of this CTA
+      const int k_before = k;
+      k += dk; cin += dc;
+      if (cin >= P.chunks_per_row) { cin -= P.chunks_per_row; ++k; }
+      if (P.scale && lane == 0 && k != k_before && it + 1 < my_chunks) sc = __ldg(P.scale + k);
     }
+    for (int j = it > R - 1 ? it - (R - 1) : 0; j < it && ok; ++j) ok = retire(j);
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    __syncwarp();
+    if (!ok) {
+      // leave only after the copies already requested into this CTA's shared memory have landed
+      for (int j = it > R ? it - R : 0; j < it; ++j)
+        mbar_wait_bounded(bars + 8 * (j % R), (j / R) & 1, P.status);
+    }
+    return;
+  }
+
+  // -------------------------------------------------------------------- consumer warps (16)
+  // The consumer threads form `groups` groups that take chunks in turn, so that several chunks
+  // are being updated at once: one chunk's chain of loads, square root, divide and stores is
+  // long, and a single group would make the ring wait for it.
+  const int gsize = 512 / P.groups;
+  const int grp = (threadIdx.x - 32) / gsize, c = (threadIdx.x - 32) - grp * gsize;
+  for (int it = grp; it < my_chunks; it += P.groups) {
+    const int slot = it % R;
+    if (!mbar_wait_bounded(bars + 8 * slot, (it / R) & 1, P.status)) return;
+    const AdagradSlot si = sinfo[slot];
+    const long long e0 = si.e0, hi = si.hi, se = si.se;
+    const int where = si.where;
+    const float sc = si.sc;
+    float* sg = reinterpret_cast<float*>(ring0 + (size_t)slot * P.slot_stride);
+    float* sa = sg + T;
+    TH* sth = reinterpret_cast<TH*>(sa + T);
+#pragma unroll 2
+    for (int col = c * 4; col < T; col += gsize * 4) {
+      const long long e = e0 + col;
+      if (e >= hi) break;
+      const float4 gv = *reinterpret_cast<const float4*>(sg + col);
+      const float4 av = *reinterpret_cast<const float4*>(sa + col);
+      float g[4] = {gv.x, gv.y, gv.z, gv.w}, a[4] = {av.x, av.y, av.z, av.w}, th[4];
+      ThetaTraits<TH>::lds_quad(sth + col, th);
 #pragma unroll
-    for (int x = 0; x < VEC; ++x) {
-      if (x < n) {
+      for (int x = 0; x < 4; ++x) {
         bool inside = where == 1;
         if (where == 2)
-          for (int r = 0; r < R.n; ++r) inside = inside || (e + x >= R.begin[r] && e + x < R.end[r]);
+          for (int r = 0; r < P.R.n; ++r) inside = inside || (e + x >= P.R.begin[r] && e + x < P.R.end[r]);
         float gx = g[x];
         if (inside) gx = __fmul_rn(gx, sc);
         a[x] = __fadd_rn(a[x], __fmul_rn(gx, gx));
-        const float denom = __fadd_rn(__fsqrt_rn(a[x]), eps);
-        th[x] = ThetaTraits<TH>::round_store(__fsub_rn(th[x], __fdiv_rn(__fmul_rn(lr, gx), denom)));
+        const float denom = __fadd_rn(__fsqrt_rn(a[x]), P.eps);
+        th[x] = __fsub_rn(th[x], __fdiv_rn(__fmul_rn(P.lr, gx), denom));
+      }
+      if (e + 4 <= se) {
+        *reinterpret_cast<float4*>(sa + col) = make_float4(a[0], a[1], a[2], a[3]);
+        TmemCell<TH>::sts_quad(sth + col, th);
+      } else {
+        // after the last whole 16-byte piece of the row: only the elements below N
+        const long long at = (long long)si.k * P.ld + e;
+        for (int x = 0; x < 4; ++x) {
+          if (e + x < hi) {
+            P.accum[at + x] = a[x];
+            theta[at + x] = ThetaTraits<TH>::narrow(th[x]);
+          }
+        }
       }
     }
-    if (n == VEC) {
-#pragma unroll
-      for (int h = 0; h < VEC / 4; ++h)
-        __stcs(reinterpret_cast<float4*>(accum + at) + h,
-               make_float4(a[4 * h], a[4 * h + 1], a[4 * h + 2], a[4 * h + 3]));
-      ThetaTraits<TH>::stg(theta + at, th);
-    } else {
-      for (int x = 0; x < n; ++x) {
-        accum[at + x] = a[x];
-        theta[at + x] = ThetaTraits<TH>::narrow(th[x]);
-      }
-    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    mbar_arrive(bars + 64 + 8 * slot);
   }
 }
 
@@ -2148,14 +2265,27 @@ gbmuf_status gbmuf_local_adagrad(gbmuf_ctx* ctx, const float* grad, float* accum
                                                        ctx->d_clip_scale);
     scale = ctx->d_clip_scale;
   }
+  // streaming update: chunks of 4096 elements (16 KB of gradient and accumulator each), 4 slots
+  AdagradParams A;
+  const int esz = (int)theta_size(ctx);
+  A.theta = ctx->theta; A.grad = grad; A.accum = accum; A.scale = scale; A.status = ctx->d_status;
+  A.N = ctx->cfg.N; A.ld = ctx->cfg.ld; A.K = K; A.T = 4096; A.ring = 4; A.groups = 2;
+  A.ring_off = 512; A.slot_stride = (uint32_t)((8 + esz) * A.T);
+  A.lr = lr; A.eps = eps; A.R = R;
+  const long long cpr = (ctx->cfg.N + A.T - 1) / A.T;
+  if (cpr * K > 0x7fffffffLL) return fail(ctx, GBMUF_ERR_UNSUPPORTED, "more than 2^31 - 1 chunks");
+  A.chunks_per_row = (int)cpr;
+  const uint32_t smem_bytes = A.ring_off + (uint32_t)A.ring * A.slot_stride;
+  const long long chunks = cpr * K;
+  const int grid = (int)(chunks < ctx->num_sms ? chunks : ctx->num_sms);
   if (ctx->cfg.theta_dtype == GBMUF_F32) {
-    const dim3 grid(row_grid(ctx, (ctx->cfg.N + 3) / 4, K), K);
-    adagrad_kernel<float><<<grid, 256, 0, st>>>((float*)ctx->theta, grad, accum, K, ctx->cfg.N,
-                                                ctx->cfg.ld, lr, eps, scale, R);
+    e = cudaFuncSetAttribute(adagrad_stream_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem);
+    if (e != cudaSuccess) return cuda_fail(ctx, "cudaFuncSetAttribute", e);
+    adagrad_stream_kernel<float><<<grid, 544, smem_bytes, st>>>(A);
   } else {
-    const dim3 grid(row_grid(ctx, (ctx->cfg.N + 7) / 8, K), K);
-    adagrad_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((__nv_bfloat16*)ctx->theta, grad, accum, K,
-                                                        ctx->cfg.N, ctx->cfg.ld, lr, eps, scale, R);
+    e = cudaFuncSetAttribute(adagrad_stream_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem);
+    if (e != cudaSuccess) return cuda_fail(ctx, "cudaFuncSetAttribute", e);
+    adagrad_stream_kernel<__nv_bfloat16><<<grid, 544, smem_bytes, st>>>(A);
   }
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, "launch of the Adagrad local-step kernels", e);

@@ -17,6 +17,8 @@ pytestmark = pytest.mark.gpu
     (3, (0, 7, 4099, 4100, 10000, 30001), [1, 0, 1, 0, 1]),   # three separate runs
     (2, (0, 50_000), [1]),                                    # everything clipped
     (5, (0, 64, 10_007), None),                               # no clipping
+    (8, (0, 100_000, 100_003, 333_333, 500_003), [0, 1, 1, 0]),   # every CTA goes round its ring of slots
+    (1, (0, 5), None),                                        # shorter than one 16-byte piece
 ])
 def test_adagrad_step_matches_oracle(dtype, K, offsets, mask):
     dev = torch.device("cuda:0")
