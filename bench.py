@@ -34,11 +34,11 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of the fused kernel per replica-parameter from an ncu capture (dram__bytes_read.sum
 # + dram__bytes_write.sum divided by the replica-parameters of the captured launch; key = theta
-# dtype: 0 fp32 from workload profile16 (tensor-memory kernel), 1 bf16 from profile16bf
-# (shared-memory kernel)), valid only
+# dtype: 0 fp32 from workload profile16, 1 bf16 from profile16bf, both the tensor-memory
+# kernel), valid only
 # for the kernel source it was taken from (source_sha() below).
-NCU_TRAFFIC = {"source_sha": "b3ec2c12f686", "bytes_per_replica_param": {0: 6.383429e9 / 268435536,
-                                                                   1: 5.309491e9 / 268435536}}
+NCU_TRAFFIC = {"source_sha": "e997b695ca4d", "bytes_per_replica_param": {0: 6.382833e9 / 268435536,
+                                                                   1: 5.309288e9 / 268435536}}
 
 
 def algorithmic_bytes_per_replica_param(dtype: int, mode: int = 0) -> int:
