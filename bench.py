@@ -103,14 +103,14 @@ class ClockSampler:
 
 
 def source_sha() -> str:
-    """Fingerprint of the fused kernel's source: the part of csrc/gbmuf.cu from the barrier /
-    bulk-copy primitives to the end of the fused round kernels (theta traits, filter, the
-    shared-memory-tile kernel and the tensor-memory-tile kernel)."""
-    with open(os.path.join(ROOT, "paper_1909_09010_b200", "csrc", "gbmuf.cu"), "rb") as f:
-        text = f.read()
-    a = text.index(b"// Shared-memory barrier and bulk-copy primitives")
-    b = text.index(b"// Self-test of the bounded wait")
-    return hashlib.sha256(text[a:b]).hexdigest()[:12]
+    """Fingerprint of the fused kernels' source: the files that hold the barrier / bulk-copy
+    primitives and theta traits, the shared-memory-tile kernel (with the averaging division and
+    the filter) and the tensor-memory-tile kernel."""
+    h = hashlib.sha256()
+    for name in ("primitives.cuh", "sync_fused.cuh", "sync_fused_tmem.cuh"):
+        with open(os.path.join(ROOT, "paper_1909_09010_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:12]
 
 
 # ------------------------------------------------------------------------------------------------

@@ -6,7 +6,8 @@ import subprocess
 
 PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
-SRC = os.path.join(PKG, "csrc", "gbmuf.cu")
+CSRC = os.path.join(PKG, "csrc")
+SRC = os.path.join(CSRC, "gbmuf.cu")          # the one translation unit; it includes csrc/*.cuh
 HDR = os.path.join(ROOT, "include", "gbmuf.h")
 LIB = os.path.join(PKG, "libgbmuf.so")
 
@@ -25,7 +26,8 @@ def is_stale() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    return any(os.path.getmtime(f) > t for f in (SRC, HDR))
+    sources = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cu", ".cuh"))]
+    return any(os.path.getmtime(f) > t for f in sources + [HDR])
 
 
 def build(force: bool = False, verbose: bool = False) -> str:

@@ -1,18 +1,24 @@
 // libgbmuf: the random-gossip BMUF synchronisation round (Algorithm 1 of "A Random Gossip BMUF
 // Process for Neural Language Modeling") for K parameter replicas resident in one GPU's memory.
-// CUDA for sm_100a.  The interface is include/gbmuf.h; this file holds the kernels and the
-// host-side C ABI.
+// CUDA for sm_100a.  The interface is include/gbmuf.h; this file holds the host side and the C
+// ABI, the kernels live in the headers it includes:
+//   philox.cuh           Philox4x32-10
+//   round_setup.cuh      round_setup_kernel: neighbour draws for every (worker, component) of a
+//                        round + the tile work-list prefix of the components that take part
+//   primitives.cuh       bounded barrier waits, bulk copies, theta storage types
+//   sync_fused.cuh       sync_fused_kernel: gather + average + block-momentum filter, one pass, in
+//                        place, theta tile in shared memory (also gossip-MA)
+//   sync_fused_tmem.cuh  sync_fused_tmem_kernel: the same with the theta tile in tensor memory and
+//                        bulk stores (the default in gossip-BMUF mode); device self-tests
+//   local_step.cuh       perturb_kernel (synthetic local steps), the Adagrad local step,
+//                        init_kernel (theta^k <- theta_0, omega^k <- theta_0, Delta^k <- 0),
+//                        final_average_kernel (theta = (1/K) sum_k theta^k)
+//   peer.cuh             one worker per GPU over peer-mapped buffers
 //
-// Kernels
-//   round_setup_kernel   neighbour draws for every (worker, component) of a round + the tile
-//                        work-list prefix of the components that take part
-//   sync_fused_kernel    gather + average + block-momentum filter, one pass, in place
-//   perturb_kernel       synthetic local steps (counter-based noise)
-//   init_kernel          theta^k <- theta_0, omega^k <- theta_0, Delta^k <- 0
-//   final_average_kernel theta = (1/K) sum_k theta^k
-//
-// Floating point: every operation is an explicit round-to-nearest intrinsic (__fadd_rn,
-// __fmul_rn, __fdiv_rn) so that nothing is contracted into a fused multiply-add.
+// Floating point: every operation of Algorithm 1 is an explicit round-to-nearest intrinsic
+// (__fadd_rn, __fmul_rn, ...) so that nothing is contracted into a fused multiply-add; the one
+// fused multiply-add in use sits inside the averaging division (sync_fused.cuh), whose result is
+// the correctly rounded quotient.
 
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -28,1656 +34,15 @@
 
 #include "gbmuf.h"
 
+#include "philox.cuh"
+#include "round_setup.cuh"
+#include "primitives.cuh"
+#include "sync_fused.cuh"
+#include "sync_fused_tmem.cuh"
+#include "local_step.cuh"
+#include "peer.cuh"
+
 namespace {
-
-// =================================================================================================
-// Philox4x32-10 (Salmon et al., SC'11), device side
-// =================================================================================================
-struct Philox4 { uint32_t x, y, z, w; };
-
-__device__ __forceinline__ Philox4 philox4x32_10(Philox4 c, uint32_t k0, uint32_t k1) {
-#pragma unroll
-  for (int r = 0; r < 10; ++r) {
-    const uint32_t hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
-    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
-    Philox4 n;
-    n.x = hi1 ^ c.y ^ k0;
-    n.y = lo1;
-    n.z = hi0 ^ c.w ^ k1;
-    n.w = lo0;
-    c = n;
-    k0 += 0x9E3779B9u;
-    k1 += 0xBB67AE85u;
-  }
-  return c;
-}
-
-constexpr uint32_t kTagSampler = 0x53414D50u;  // second key word of the neighbour-draw stream
-constexpr uint32_t kTagPerturb = 0x50455254u;  // second key word of the local-step noise stream
-constexpr int kMaxCand = 64;                   // largest candidate set min(2p, K-1)
-constexpr int kAlign = 8;                      // tiles start on multiples of 8 elements (>= 16 B)
-
-// =================================================================================================
-// Round set-up: neighbour draws (Algorithm 1, the neighbour-choice line: k_1..k_q) and the
-// work-list of this round.
-// =================================================================================================
-struct SetupParams {
-  int K, m, p, q, comp_base, T, use_mask, plan;
-  uint64_t seed, round;
-  const int64_t* off;      // [m+1]
-  const int32_t* periods;  // [m]
-  const uint8_t* mask;     // [m] when use_mask
-  int32_t* nbr;            // [m][K][q]
-  int32_t* tile_prefix;    // [m+1]
-};
-
-// Ring neighbours of worker k (Definition 1): (k-1)%K..(k-p)%K then (k+1)%K..(k+p)%K, leaving
-// out k itself and anything already listed.  Returns the count.
-__device__ int ring_candidates(int k, int K, int p, int32_t* a) {
-  int c = 0;
-  for (int side = 0; side < 2; ++side) {
-    for (int d = 1; d <= p && c < kMaxCand; ++d) {
-      const int step = d % K;
-      int node = side == 0 ? k - step : k + step;
-      if (node < 0) node += K;
-      if (node >= K) node -= K;
-      if (node == k) continue;
-      bool seen = false;
-      for (int j = 0; j < c; ++j) seen |= (a[j] == node);
-      if (!seen) a[c++] = node;
-    }
-  }
-  return c;
-}
-
-__device__ __forceinline__ int tiles_of_component(int64_t lo, int64_t hi, int T) {
-  if (hi <= lo) return 0;
-  const int64_t start = lo & ~(int64_t)(kAlign - 1);
-  return (int)((hi - start + T - 1) / T);
-}
-
-__global__ void __launch_bounds__(256) round_setup_kernel(SetupParams P) {
-  const int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (g < (int64_t)P.K * P.m && P.q > 0) {
-    const int i = (int)(g / P.K), k = (int)(g % P.K);
-    int32_t a[kMaxCand];
-    const int c = ring_candidates(k, P.K, P.p, a);
-    int32_t* out = P.nbr + g * P.q;
-    Philox4 r = {0, 0, 0, 0};
-    for (int j = 0; j < P.q && j < c; ++j) {
-      if ((j & 3) == 0) {
-        Philox4 ctr = {(uint32_t)P.round, (uint32_t)(P.round >> 32), (uint32_t)(P.comp_base + i),
-                       (uint32_t)k | ((uint32_t)(j >> 2) << 16)};
-        r = philox4x32_10(ctr, (uint32_t)P.seed, (uint32_t)(P.seed >> 32) ^ kTagSampler);
-      }
-      const uint32_t u = (j & 3) == 0 ? r.x : (j & 3) == 1 ? r.y : (j & 3) == 2 ? r.z : r.w;
-      const int t = j + (int)__umulhi(u, (uint32_t)(c - j));   // partial Fisher-Yates
-      const int32_t tmp = a[j];
-      a[j] = a[t];
-      a[t] = tmp;
-      out[j] = a[j];
-    }
-  }
-
-  // Block 0 also lays out the work-list: tile_prefix[i] = number of tiles of the participating
-  // components before i.  Block-wide exclusive scan, 256 components at a time.
-  if (blockIdx.x == 0 && P.plan) {
-    __shared__ int warp_tot[8];
-    __shared__ int carry_s;
-    if (threadIdx.x == 0) carry_s = 0;
-    __syncthreads();
-    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    for (int base = 0; base < P.m; base += 256) {
-      const int i = base + threadIdx.x;
-      int cnt = 0;
-      if (i < P.m) {
-        const bool due = P.use_mask ? (P.mask[i] != 0) : (P.round % (uint64_t)P.periods[i] == 0);
-        if (due) cnt = tiles_of_component(P.off[i], P.off[i + 1], P.T);
-      }
-      int inc = cnt;
-#pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
-        const int n = __shfl_up_sync(0xffffffffu, inc, d);
-        if (lane >= d) inc += n;
-      }
-      if (lane == 31) warp_tot[wid] = inc;
-      __syncthreads();
-      int before = 0;
-      for (int w2 = 0; w2 < wid; ++w2) before += warp_tot[w2];
-      const int carry = carry_s;
-      if (i < P.m) P.tile_prefix[i] = carry + before + inc - cnt;
-      __syncthreads();
-      if (threadIdx.x == 255) carry_s = carry + before + inc;
-      __syncthreads();
-    }
-    if (threadIdx.x == 0) P.tile_prefix[P.m] = carry_s;
-  }
-}
-
-// =================================================================================================
-// Shared-memory barrier and bulk-copy primitives (PTX).  Every wait is bounded.
-// =================================================================================================
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return (uint32_t)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
-               : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ unsigned long long global_timer_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // two seconds
-// Wait for the phase with the given parity to complete.  Bounded in wall-clock time: after
-// kWaitLimitNs it records GBMUF_ERR_TIMEOUT in the device status word and returns false; the
-// caller then leaves its loop.  (try_wait may itself suspend the thread for a while, so the bound
-// is on the timer, not on the number of tries.)
-__device__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, int32_t* status) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = global_timer_ns();
-  for (uint32_t spin = 0;; ++spin) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (spin > 32) __nanosleep(spin > 4096 ? 256 : 32);
-    if ((spin & 63) == 63 && global_timer_ns() - t0 > kWaitLimitNs) break;
-  }
-  atomicExch(status, (int32_t)GBMUF_ERR_TIMEOUT);
-  return false;
-}
-// Two-dimensional tiled TMA load: the box [rows 0..K) x [columns x, x + box width) of a row-major
-// [K][ld] array lands in shared memory as K consecutive rows of box-width elements.  One request
-// per box (no multicast); completion is counted in bytes on the mbarrier, out-of-range columns
-// are zero-filled and still counted.  x * element size must be a multiple of 16 bytes.
-__device__ __forceinline__ void tma_load_box(uint32_t dst_smem, const CUtensorMap* map, int x, int y,
-                                             uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], "
-      "[%1, {%2, %3}], [%4];" ::"r"(dst_smem),
-      "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
-      : "memory");
-}
-
-// One-dimensional bulk copy global -> shared through the copy engine (no multicast); completion
-// is counted in bytes on the mbarrier.  Addresses and size are multiples of 16 bytes.
-__device__ __forceinline__ void bulk_load_row(uint32_t dst_smem, const void* src, uint32_t bytes,
-                                              uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-          dst_smem),
-      "l"(src), "r"(bytes), "r"(bar)
-      : "memory");
-}
-
-// =================================================================================================
-// theta storage types
-// =================================================================================================
-template <typename TH> struct ThetaTraits;
-template <> struct ThetaTraits<float> {
-  static constexpr int VEC = 4;   // elements per 16-byte vector of theta
-  static __device__ __forceinline__ float widen(float v) { return v; }
-  static __device__ __forceinline__ float round_store(float v) { return v; }
-  static __device__ __forceinline__ float narrow(float v) { return v; }
-  static __device__ __forceinline__ void lds(const float* p, float (&x)[4]) {
-    const float4 t = *reinterpret_cast<const float4*>(p);
-    x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w;
-  }
-  static __device__ __forceinline__ void stg(float* p, const float (&x)[4]) {
-    __stcs(reinterpret_cast<float4*>(p), make_float4(x[0], x[1], x[2], x[3]));
-  }  // four consecutive elements (what one thread of the fused kernel handles per row)
-  static __device__ __forceinline__ void lds_quad(const float* p, float (&x)[4]) { lds(p, x); }
-  static __device__ __forceinline__ void stg_quad(float* p, const float (&x)[4]) { stg(p, x); }
-};
-template <> struct ThetaTraits<__nv_bfloat16> {
-  static constexpr int VEC = 8;
-  static __device__ __forceinline__ float widen(__nv_bfloat16 v) { return __bfloat162float(v); }
-  // value of v after a round trip through bf16 storage (round to nearest, ties to even)
-  static __device__ __forceinline__ float round_store(float v) {
-    return __bfloat162float(__float2bfloat16_rn(v));
-  }
-  static __device__ __forceinline__ __nv_bfloat16 narrow(float v) { return __float2bfloat16_rn(v); }
-  static __device__ __forceinline__ void lds(const __nv_bfloat16* p, float (&x)[8]) {
-    const uint4 t = *reinterpret_cast<const uint4*>(p);
-    x[0] = __uint_as_float(t.x << 16); x[1] = __uint_as_float(t.x & 0xFFFF0000u);
-    x[2] = __uint_as_float(t.y << 16); x[3] = __uint_as_float(t.y & 0xFFFF0000u);
-    x[4] = __uint_as_float(t.z << 16); x[5] = __uint_as_float(t.z & 0xFFFF0000u);
-    x[6] = __uint_as_float(t.w << 16); x[7] = __uint_as_float(t.w & 0xFFFF0000u);
-  }
-  static __device__ __forceinline__ void stg(__nv_bfloat16* p, const float (&x)[8]) {
-    uint4 t;
-    __nv_bfloat162 h;
-    h = __floats2bfloat162_rn(x[0], x[1]); t.x = *reinterpret_cast<uint32_t*>(&h);
-    h = __floats2bfloat162_rn(x[2], x[3]); t.y = *reinterpret_cast<uint32_t*>(&h);
-    h = __floats2bfloat162_rn(x[4], x[5]); t.z = *reinterpret_cast<uint32_t*>(&h);
-    h = __floats2bfloat162_rn(x[6], x[7]); t.w = *reinterpret_cast<uint32_t*>(&h);
-    __stcs(reinterpret_cast<uint4*>(p), t);
-  }
-  // four consecutive elements = 8 bytes
-  static __device__ __forceinline__ void lds_quad(const __nv_bfloat16* p, float (&x)[4]) {
-    const uint2 t = *reinterpret_cast<const uint2*>(p);
-    x[0] = __uint_as_float(t.x << 16); x[1] = __uint_as_float(t.x & 0xFFFF0000u);
-    x[2] = __uint_as_float(t.y << 16); x[3] = __uint_as_float(t.y & 0xFFFF0000u);
-  }
-  static __device__ __forceinline__ void stg_quad(__nv_bfloat16* p, const float (&x)[4]) {
-    uint2 t;
-    __nv_bfloat162 h;
-    h = __floats2bfloat162_rn(x[0], x[1]); t.x = *reinterpret_cast<uint32_t*>(&h);
-    h = __floats2bfloat162_rn(x[2], x[3]); t.y = *reinterpret_cast<uint32_t*>(&h);
-    __stcs(reinterpret_cast<uint2*>(p), t);
-  }
-};
-
-// =================================================================================================
-// The fused round: gather + average + block-momentum filter, in place, one pass.
-//
-// Work item = one tile: up to T consecutive elements of ONE component, for all K workers.  A
-// persistent CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...
-//
-// Shared memory holds (a) one or two theta stages, each the K replicas' slices of a tile -- every
-// worker's average may need any other worker's slice, so the whole K-row tile must be resident --
-// and (b) a small ring of row slots for omega and Delta, which are needed exactly once per
-// (worker, element) and therefore only pass through.  Keeping omega and Delta out of the tile
-// stage is what lets T, the contiguous run per row, be as long as 8 KB: measured DRAM efficiency
-// grows with that run length far more than with pipeline depth.
-//
-// Warp 0 is the producer.  Per tile it looks the tile up in the work-list, has the copy engine
-// fetch the theta stage (tiled TMA, one request per [K rows x 256 columns] box) and then, worker by
-// worker, one row of omega and one of Delta into the next free ring slot (bulk copies).  The other
-// warps are consumers: they wait for the theta stage, then for each worker k wait for its ring
-// slot; each thread takes 16-byte vectors of the row, sums worker k's own slice and its q
-// neighbours' slices out of shared memory (own first, then draw order), divides by q+1, applies the
-// filter and writes Delta, omega and the restart point theta straight to global memory, then
-// releases the slot.  All global reads are issued by the copy engine, so the bytes in flight do
-// not depend on how many threads are resident.  Because the CTA is the only reader and writer of
-// its tile in all K replicas and has staged the pre-round theta before writing any, every
-// neighbour read sees the replica as it was before the round.  Unique traffic per
-// replica-parameter: theta read once, omega and Delta read once, all three written once.
-//
-// Every wait is bounded; a wait that expires records GBMUF_ERR_TIMEOUT and the thread leaves.
-// =================================================================================================
-struct TileDesc {
-  long long e0;   // first element of the staged range (multiple of kAlign)
-  long long lo;   // first element this tile owns
-  long long hi;   // one past the last element this tile owns
-  int comp;
-  int pad;
-};
-
-constexpr int kMaxRing = 8;
-// barrier block at the start of shared memory (8 bytes each)
-constexpr uint32_t kBarThetaFull = 0, kBarThetaEmpty = 32, kBarRingFull = 64, kBarRingEmpty = 128;
-constexpr int kMaxThetaStages = 4;
-constexpr uint32_t kBarBytes = 256;
-
-struct SyncParams {
-  void* theta;
-  float* omega;
-  float* delta;
-  const int64_t* off;
-  const int32_t* tile_prefix;
-  const int32_t* nbr;   // [m][K][q]
-  int32_t* status;
-  long long ld;
-  int K, m, q, mode;
-  float eta, zeta, qp1, inv_qp1;
-  int inv_exact;        // q+1 is a power of two: multiplying by 1/(q+1) equals dividing
-  int T, BW, bw_shift, bw_mask;   // BW: columns per TMA box; column c of a tile is in box
-                                  // c >> bw_shift at c & bw_mask
-  int stages, ring, ncons;        // theta stages (1..4), ring slots, consumer threads
-  uint32_t stage_stride, nbr_off, desc_off;   // theta stage: [theta boxes | nbr | desc]
-  uint32_t ring_off, slot_stride;             // ring slot: [omega row T floats | Delta row T floats]
-};
-
-// The division of the gossip average, s / (q+1), for four elements.  The result is that of the
-// IEEE-754 division rounded to nearest even, bit for bit, for every input; only the route differs:
-//  - q+1 a power of two: multiplying by 1/(q+1) is exact;
-//  - otherwise, for the small integer divisor b = q+1 and y = RN(1/b): q0 = RN(s*y), the exact
-//    residual r = fma(-b, q0, s), then RN(q0 + r*y) (Markstein's correction step).  It is taken
-//    only when the exponent of s is in the middle range, where no intermediate can overflow,
-//    underflow or be subnormal; zeros, subnormals, huge values, infinities and NaNs go through the
-//    division instruction sequence.  gbmuf_selftest_divide compares this routine with the plain
-//    division over all 2^32 bit patterns for a given divisor.
-// Costs 3 arithmetic instructions per element instead of about 10; gossip-MA with q+1 = 3 was
-// limited by the divide.
-// Exponent test: the result has one of its two top bits set iff the biased exponent of s is
-// outside [64, 191], i.e. unless 2^-63 <= |s| < 2^65; results of several values may be OR-ed.
-__device__ __forceinline__ uint32_t outside_mid_range(float s) {
-  return (__float_as_uint(s) & 0x7F800000u) - 0x20000000u;
-}
-__device__ __forceinline__ float divide_corrected(float s, float b, float y) {
-  const float q0 = __fmul_rn(s, y);
-  const float r = __fmaf_rn(-b, q0, s);
-  return __fmaf_rn(r, y, q0);
-}
-__device__ __forceinline__ void average_divide(float (&a)[4], float b, float y, int y_exact) {
-  if (y_exact) {
-#pragma unroll
-    for (int x = 0; x < 4; ++x) a[x] = __fmul_rn(a[x], y);
-  } else if (!((outside_mid_range(a[0]) | outside_mid_range(a[1]) | outside_mid_range(a[2]) |
-                outside_mid_range(a[3])) & 0xC0000000u)) {
-#pragma unroll
-    for (int x = 0; x < 4; ++x) a[x] = divide_corrected(a[x], b, y);
-  } else {
-#pragma unroll
-    for (int x = 0; x < 4; ++x) a[x] = __fdiv_rn(a[x], b);
-  }
-}
-
-// Block-momentum filter for one element (Algorithm 1: G, Delta, omega, theta lines).  The
-// block-start value is recomputed from the pre-round omega and Delta.
-template <typename TH>
-__device__ __forceinline__ void bmuf_filter(float avg, float& w, float& d, float& t, float eta,
-                                            float zeta) {
-  const float etad = __fmul_rn(eta, d);
-  const float r = ThetaTraits<TH>::round_store(__fadd_rn(w, etad));
-  const float g = __fsub_rn(avg, r);
-  d = __fadd_rn(etad, __fmul_rn(zeta, g));
-  w = __fadd_rn(w, d);
-  t = __fadd_rn(w, __fmul_rn(eta, d));
-}
-
-template <typename TH>
-__global__ void __launch_bounds__(1024, 1)
-sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_theta) {
-  constexpr int VEC = 4;   // elements per thread and row: 16 bytes of omega / Delta, 16 or 8 of theta
-  extern __shared__ __align__(128) unsigned char smem[];
-  const uint32_t bars = smem_u32(smem);
-  unsigned char* stage0 = smem + kBarBytes;
-  unsigned char* ring0 = smem + P.ring_off;
-  const int total = P.tile_prefix[P.m];
-  const int S = P.stages, R = P.ring;
-  const bool bmuf = P.mode == GBMUF_MODE_BMUF;
-  const int my_tiles = (int)blockIdx.x < total ? (total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < S; ++s) {
-      mbar_init(bars + kBarThetaFull + 8 * s, 1);          // the producer's arrival + bytes
-      mbar_init(bars + kBarThetaEmpty + 8 * s, P.ncons);   // every consumer thread arrives
-      reinterpret_cast<TileDesc*>(stage0 + (size_t)s * P.stage_stride + P.desc_off)->comp = -1;
-    }
-    for (int r = 0; r < R; ++r) {
-      mbar_init(bars + kBarRingFull + 8 * r, 1);
-      mbar_init(bars + kBarRingEmpty + 8 * r, P.ncons);
-    }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  }
-  __syncthreads();
-
-  if (threadIdx.x < 32) {
-    // ------------------------------------------------------------------ producer warp
-    const int lane = threadIdx.x;
-    bool ok = true;
-    // The tiles of this CTA come in increasing order, so the component only ever moves forward:
-    // find the first one by bisection, then advance.  In the steady state the loop below touches
-    // no global memory except through the copies it issues.
-    int comp = 0, pfx_lo = 0, pfx_hi = 0;
-    long long cb = 0, ce = 0;
-    if (my_tiles > 0) {
-      int lo_i = 0, hi_i = P.m;
-      while (hi_i - lo_i > 1) {
-        const int mid = (lo_i + hi_i) >> 1;
-        if (__ldg(P.tile_prefix + mid) <= (int)blockIdx.x) lo_i = mid; else hi_i = mid;
-      }
-      comp = lo_i;
-      pfx_lo = __ldg(P.tile_prefix + comp);
-      pfx_hi = __ldg(P.tile_prefix + comp + 1);
-      cb = __ldg(P.off + comp);
-      ce = __ldg(P.off + comp + 1);
-    }
-    int theta_issued = 0;    // tiles whose theta stage has been requested
-    int ring_issued = 0;     // ring slots requested so far (over all tiles)
-
-    // request the theta stage of this CTA's j-th tile (j = theta_issued)
-    auto issue_theta = [&]() -> bool {
-      const int j = theta_issued;
-      const int w = (int)blockIdx.x + j * (int)gridDim.x;
-      const int s = j % S;
-      if (j >= S) {
-        bool fine = mbar_wait_bounded(bars + kBarThetaEmpty + 8 * s, ((j / S) - 1) & 1, P.status);
-        if (!__all_sync(0xffffffffu, fine)) return false;
-      }
-      if (w >= pfx_hi) {
-        while (w >= pfx_hi) {      // w < total = tile_prefix[m], so comp stays below m
-          ++comp;
-          pfx_lo = pfx_hi;
-          pfx_hi = __ldg(P.tile_prefix + comp + 1);
-        }
-        cb = __ldg(P.off + comp);
-        ce = __ldg(P.off + comp + 1);
-      }
-      const long long e0 = (cb & ~(long long)(kAlign - 1)) + (long long)(w - pfx_lo) * P.T;
-      unsigned char* st = stage0 + (size_t)s * P.stage_stride;
-      TileDesc* d = reinterpret_cast<TileDesc*>(st + P.desc_off);
-      if (d->comp != comp) {       // the stage still holds the table of the component it last served
-        int* snb = reinterpret_cast<int*>(st + P.nbr_off);
-        const int32_t* gnb = P.nbr + (size_t)comp * P.K * P.q;
-        for (int x = lane; x < P.K * P.q; x += 32) snb[x] = __ldg(gnb + x);
-      }
-      __syncwarp();
-      if (lane == 0) {
-        d->e0 = e0;
-        d->lo = cb > e0 ? cb : e0;
-        d->hi = ce < e0 + P.T ? ce : e0 + P.T;
-        d->comp = comp;
-      }
-      __syncwarp();
-      const uint32_t full = bars + kBarThetaFull + 8 * s;
-      const uint32_t sbase = smem_u32(st);
-      if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)P.K * (uint32_t)P.T * (uint32_t)sizeof(TH));
-      __syncwarp();
-      const uint32_t box_bytes = (uint32_t)P.K * (uint32_t)P.BW * (uint32_t)sizeof(TH);
-      for (int b = lane; b < P.T / P.BW; b += 32)
-        tma_load_box(sbase + (uint32_t)b * box_bytes, &map_theta, (int)e0 + b * P.BW, 0, full);
-      ++theta_issued;
-      return true;
-    };
-
-    for (int j = 0; j < S - 1 && j < my_tiles && ok; ++j) ok = issue_theta();
-    for (int it = 0; it < my_tiles && ok; ++it) {
-      if (it + S - 1 < my_tiles) ok = issue_theta();   // keeps S-1 tiles of theta ahead (S=1: this tile)
-      if (!ok) break;
-      if (bmuf) {
-        const TileDesc* d = reinterpret_cast<const TileDesc*>(stage0 + (size_t)(it % S) * P.stage_stride + P.desc_off);
-        const long long e0 = d->e0;
-        long long run = P.ld - e0;                       // a row ends at ld: never read past it
-        if (run > P.T) run = P.T;
-        const uint32_t bytes = (uint32_t)run * 4u;
-        for (int k = 0; k < P.K; ++k) {
-          const int slot = ring_issued % R;
-          if (ring_issued >= R) {
-            bool fine = mbar_wait_bounded(bars + kBarRingEmpty + 8 * slot, ((ring_issued / R) - 1) & 1, P.status);
-            ok = __all_sync(0xffffffffu, fine);
-            if (!ok) break;
-          }
-          if (lane == 0) {
-            const uint32_t full = bars + kBarRingFull + 8 * slot;
-            const uint32_t dst = smem_u32(ring0 + (size_t)slot * P.slot_stride);
-            const long long at = (long long)k * P.ld + e0;
-            mbar_arrive_expect_tx(full, 2u * bytes);
-            bulk_load_row(dst, P.omega + at, bytes, full);
-            bulk_load_row(dst + (uint32_t)P.T * 4u, P.delta + at, bytes, full);
-          }
-          ++ring_issued;
-        }
-      }
-    }
-    if (!ok) {
-      // leave only after the copies already requested into this CTA's shared memory have landed
-      for (int j = theta_issued > S ? theta_issued - S : 0; j < theta_issued; ++j)
-        mbar_wait_bounded(bars + kBarThetaFull + 8 * (j % S), (j / S) & 1, P.status);
-      for (int j = ring_issued > R ? ring_issued - R : 0; j < ring_issued; ++j)
-        mbar_wait_bounded(bars + kBarRingFull + 8 * (j % R), (j / R) & 1, P.status);
-    }
-    return;
-  }
-
-  // -------------------------------------------------------------------- consumer warps
-  const int c = threadIdx.x - 32;
-  const int nv = P.T / VEC;            // vectors per row of a tile
-  const int q = P.q, BW = P.BW, box_elems = P.K * P.BW;
-  TH* theta = static_cast<TH*>(P.theta);
-  int ring_taken = 0;
-  for (int it = 0; it < my_tiles; ++it) {
-    const int s = it % S;
-    if (!mbar_wait_bounded(bars + kBarThetaFull + 8 * s, (it / S) & 1, P.status)) return;
-    unsigned char* st = stage0 + (size_t)s * P.stage_stride;
-    const TH* sth = reinterpret_cast<const TH*>(st);
-    const int* snb = reinterpret_cast<const int*>(st + P.nbr_off);
-    const TileDesc* d = reinterpret_cast<const TileDesc*>(st + P.desc_off);
-    const long long e0 = d->e0, lo = d->lo, hi = d->hi;
-    if (!bmuf) {
-      // gossip-MA: theta <- average.  No omega / Delta stream paces the workers, so each thread
-      // walks all workers for its group of elements; unrolled so that the shared-memory loads
-      // and the arithmetic of several workers overlap.
-      // With more threads than element groups the workers are split between thread groups:
-      // thread c takes group c % nv for workers c / nv, c / nv + kg, ...
-      // The division (see average_divide) is kept free of branches inside the loop, which is
-      // what lets the unrolled workers overlap: a pass either multiplies by an exact reciprocal
-      // (DIV 0), or takes the corrected-product route for every element while OR-ing the exponent
-      // tests (DIV 1), or divides plainly (DIV 2).  If a DIV 1 pass met a sum outside the middle
-      // range, the thread repeats its share of the tile with DIV 2 from the still-staged theta,
-      // overwriting what it stored.
-      // Each thread takes 16 bytes of theta per row here: 4 fp32 or 8 bf16 elements.
-      constexpr int MV = ThetaTraits<TH>::VEC;
-      const int nvm = P.T / MV;
-      const int kg = P.ncons > nvm ? P.ncons / nvm : 1;
-      const int k_first = P.ncons > nvm ? c / nvm : 0;
-      auto ma_pass = [&](auto div_tag) -> bool {
-        constexpr int DIV = decltype(div_tag)::value;
-        uint32_t oor = 0;
-        for (int v = P.ncons > nvm ? c - k_first * nvm : c; v < nvm && k_first < kg; v += P.ncons) {
-          const int col = v * MV;
-          const long long e = e0 + col;
-          if (e >= hi || e + MV <= lo) continue;
-          const int b = col >> P.bw_shift, cin = col & P.bw_mask;
-          const int boxbase = b * box_elems + cin;
-          const bool whole = e >= lo && e + MV <= hi;
-#pragma unroll 4
-          for (int k = k_first; k < P.K; k += kg) {
-            float a[MV], t[MV];
-            ThetaTraits<TH>::lds(sth + boxbase + k * BW, a);
-            for (int j = 0; j < q; ++j) {
-              ThetaTraits<TH>::lds(sth + boxbase + snb[k * q + j] * BW, t);
-#pragma unroll
-              for (int x = 0; x < MV; ++x) a[x] = __fadd_rn(a[x], t[x]);
-            }
-#pragma unroll
-            for (int x = 0; x < MV; ++x) {
-              if (DIV == 0) {
-                a[x] = __fmul_rn(a[x], P.inv_qp1);
-              } else if (DIV == 1) {
-                oor |= outside_mid_range(a[x]);
-                a[x] = divide_corrected(a[x], P.qp1, P.inv_qp1);
-              } else {
-                a[x] = __fdiv_rn(a[x], P.qp1);
-              }
-            }
-            const long long at = (long long)k * P.ld + e;
-            if (whole) {
-              ThetaTraits<TH>::stg(theta + at, a);
-            } else {
-              for (int x = 0; x < MV; ++x)
-                if (e + x >= lo && e + x < hi) theta[at + x] = ThetaTraits<TH>::narrow(a[x]);
-            }
-          }
-        }
-        return (oor & 0xC0000000u) != 0;
-      };
-      if (P.inv_exact) {
-        ma_pass(std::integral_constant<int, 0>{});
-      } else if (ma_pass(std::integral_constant<int, 1>{})) {
-        ma_pass(std::integral_constant<int, 2>{});
-      }
-      mbar_arrive(bars + kBarThetaEmpty + 8 * s);
-      continue;
-    }
-    for (int k = 0; k < P.K; ++k) {
-      const float* som = nullptr;
-      const float* sde = nullptr;
-      int slot = 0;
-      if (bmuf) {
-        slot = ring_taken % R;
-        if (!mbar_wait_bounded(bars + kBarRingFull + 8 * slot, (ring_taken / R) & 1, P.status)) return;
-        som = reinterpret_cast<const float*>(ring0 + (size_t)slot * P.slot_stride);
-        sde = som + P.T;
-      }
-      for (int v = c; v < nv; v += P.ncons) {
-        const int col = v * VEC;
-        const long long e = e0 + col;
-        if (e >= hi || e + VEC <= lo) continue;
-        // staged layout of theta: box b = col / BW holds K rows of BW columns
-        const int b = col >> P.bw_shift, cin = col & P.bw_mask;
-        const int boxbase = b * box_elems + cin;
-        // gossip average: own slice first, then the neighbours in draw order
-        float a[VEC], t[VEC];
-        ThetaTraits<TH>::lds_quad(sth + boxbase + k * BW, a);
-        for (int j = 0; j < q; ++j) {
-          ThetaTraits<TH>::lds_quad(sth + boxbase + snb[k * q + j] * BW, t);
-#pragma unroll
-          for (int x = 0; x < VEC; ++x) a[x] = __fadd_rn(a[x], t[x]);
-        }
-        average_divide(a, P.qp1, P.inv_qp1, P.inv_exact);
-        const long long at = (long long)k * P.ld + e;
-        const bool whole = e >= lo && e + VEC <= hi;
-        if (!bmuf) {                                       // gossip-MA: theta <- average
-          if (whole) {
-            ThetaTraits<TH>::stg_quad(theta + at, a);
-          } else {
-            for (int x = 0; x < VEC; ++x)
-              if (e + x >= lo && e + x < hi) theta[at + x] = ThetaTraits<TH>::narrow(a[x]);
-          }
-          continue;
-        }
-        const float4 W = *reinterpret_cast<const float4*>(som + col);
-        const float4 D = *reinterpret_cast<const float4*>(sde + col);
-        float wv[VEC] = {W.x, W.y, W.z, W.w}, dv[VEC] = {D.x, D.y, D.z, D.w};
-#pragma unroll
-        for (int x = 0; x < VEC; ++x) bmuf_filter<TH>(a[x], wv[x], dv[x], t[x], P.eta, P.zeta);
-        if (whole) {
-          __stcs(reinterpret_cast<float4*>(P.delta + at), make_float4(dv[0], dv[1], dv[2], dv[3]));
-          __stcs(reinterpret_cast<float4*>(P.omega + at), make_float4(wv[0], wv[1], wv[2], wv[3]));
-          ThetaTraits<TH>::stg_quad(theta + at, t);
-        } else {
-          // a vector that straddles the edge of the component: only the elements this tile owns
-          for (int x = 0; x < VEC; ++x) {
-            if (e + x >= lo && e + x < hi) {
-              P.delta[at + x] = dv[x];
-              P.omega[at + x] = wv[x];
-              theta[at + x] = ThetaTraits<TH>::narrow(t[x]);
-            }
-          }
-        }
-      }
-      if (bmuf) {
-        mbar_arrive(bars + kBarRingEmpty + 8 * slot);    // this thread is done with the slot
-        ++ring_taken;
-      }
-    }
-    mbar_arrive(bars + kBarThetaEmpty + 8 * s);          // this thread is done with the theta stage
-  }
-}
-
-// =================================================================================================
-// Variant of the fused round that keeps the theta tile in tensor memory (TMEM) instead of shared
-// memory.  A K x T fp32 tile of up to 256 KB does not fit shared memory next to anything else,
-// but it is exactly what the 512 columns x 128 lanes of an SM's tensor memory hold.  Every row of
-// theta, omega and Delta streams through one ring of shared-memory slots: first the K theta rows
-// of a tile (several per slot), which each consumer thread moves from the slot into its own TMEM
-// cells (tcgen05.st), then the output items, for which the thread reads its own and the drawn
-// neighbours' theta back from those cells (tcgen05.ld).  A thread only ever reads cells it wrote
-// itself, so TMEM needs no synchronisation between threads, and the run per row can be about
-// twice as long as with a shared-memory tile.
-//
-// (gossip-BMUF mode only.  The same schedule was tried for gossip-MA, whose output items carry
-// only averages: its consumers, 16 warps of serial TMEM round trips, could not keep up with 8
-// bytes per element and it ran at 60 % of the shared-memory schedule's speed.)
-//
-// TMEM addressing: a warp reaches the 32 lanes 32 * (warp id % 4) ..; with the .32x32b.xN shape
-// each thread moves the N consecutive 32-bit columns of its lane that start at the given column.
-// Four consecutive elements of a row are one cell: 4 columns for fp32, 2 for bf16 (kept packed).
-// Element group g (4 elements) of a tile lives in lane g % 128, columns ((g / 128) * K + row) *
-// cell width.  The allocation is released by the warp that made it after every thread has
-// reached the end of the kernel; no path returns early.
-// =================================================================================================
-struct TmemParams {
-  const void* theta_in;    // same array as theta (read side)
-  void* theta;
-  float* omega;
-  float* delta;
-  const int64_t* off;
-  const int32_t* tile_prefix;
-  const int32_t* nbr;      // [m][K][q]
-  int32_t* status;
-  long long ld;
-  int K, m, q;
-  float eta, zeta, qp1, inv_qp1;
-  int inv_exact;
-  int T, ring, ncols;      // T multiple of 512; ring slots; TMEM columns (power of 2)
-  uint32_t ring_off, meta_off, meta_stride;   // meta ring (4 entries): [TileDesc | nbr K*q ints]
-  uint32_t slot_stride;    // bytes per ring slot
-};
-
-// Four consecutive theta elements of one row <-> this thread's TMEM cell.  Load and wait sit in
-// ONE asm statement because the registers are only valid after the wait and nothing may be
-// scheduled between the two.  (Several loads per wait were measured slower, not faster.)
-template <typename TH> struct TmemCell;
-template <> struct TmemCell<float> {
-  static constexpr int COLS = 4;
-  static __device__ __forceinline__ void deposit(uint32_t taddr, const float* src) {
-    const float4 v = *reinterpret_cast<const float4*>(src);
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};" ::"r"(taddr),
-                 "r"(__float_as_uint(v.x)), "r"(__float_as_uint(v.y)), "r"(__float_as_uint(v.z)),
-                 "r"(__float_as_uint(v.w))
-                 : "memory");
-  }
-  static __device__ __forceinline__ void fetch(uint32_t taddr, float (&x)[4]) {
-    uint32_t a, b, c, d;
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];\n\t"
-        "tcgen05.wait::ld.sync.aligned;"
-        : "=r"(a), "=r"(b), "=r"(c), "=r"(d)
-        : "r"(taddr)
-        : "memory");
-    x[0] = __uint_as_float(a); x[1] = __uint_as_float(b); x[2] = __uint_as_float(c); x[3] = __uint_as_float(d);
-  }
-  static __device__ __forceinline__ void sts_quad(float* dst, const float (&x)[4]) {
-    *reinterpret_cast<float4*>(dst) = make_float4(x[0], x[1], x[2], x[3]);
-  }
-};
-template <> struct TmemCell<__nv_bfloat16> {
-  static constexpr int COLS = 2;
-  static __device__ __forceinline__ void deposit(uint32_t taddr, const __nv_bfloat16* src) {
-    const uint2 v = *reinterpret_cast<const uint2*>(src);
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x2.b32 [%0], {%1, %2};" ::"r"(taddr), "r"(v.x), "r"(v.y)
-                 : "memory");
-  }
-  static __device__ __forceinline__ void fetch(uint32_t taddr, float (&x)[4]) {
-    uint32_t a, b;
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x2.b32 {%0, %1}, [%2];\n\t"
-        "tcgen05.wait::ld.sync.aligned;"
-        : "=r"(a), "=r"(b)
-        : "r"(taddr)
-        : "memory");
-    x[0] = __uint_as_float(a << 16); x[1] = __uint_as_float(a & 0xFFFF0000u);
-    x[2] = __uint_as_float(b << 16); x[3] = __uint_as_float(b & 0xFFFF0000u);
-  }
-  static __device__ __forceinline__ void sts_quad(__nv_bfloat16* dst, const float (&x)[4]) {
-    uint2 t;
-    __nv_bfloat162 h;
-    h = __floats2bfloat162_rn(x[0], x[1]); t.x = *reinterpret_cast<uint32_t*>(&h);
-    h = __floats2bfloat162_rn(x[2], x[3]); t.y = *reinterpret_cast<uint32_t*>(&h);
-    *reinterpret_cast<uint2*>(dst) = t;
-  }
-};
-
-// Sum of worker k's own cell and its q drawn neighbours' cells of element group `cell0` (the
-// TMEM address of row 0's cell), own first, then draw order, each addition rounded.
-template <typename TH>
-__device__ __forceinline__ void tmem_gather(uint32_t cell0, int k, const int* nb, int q, float (&a)[4]) {
-  constexpr int CW = TmemCell<TH>::COLS;
-  TmemCell<TH>::fetch(cell0 + (uint32_t)(k * CW), a);
-  for (int j = 0; j < q; ++j) {
-    float t[4];
-    TmemCell<TH>::fetch(cell0 + (uint32_t)(nb[j] * CW), t);
-#pragma unroll
-    for (int x = 0; x < 4; ++x) a[x] = __fadd_rn(a[x], t[x]);
-  }
-}
-
-// What the producer must know to send a finished slot out: the staged range starts at e0, whole
-// 16-byte pieces of the rows cover [sb, se); k < 0: a load item, nothing to send.
-struct SlotInfo { long long e0, sb, se; int k; int pad; };
-
-// Slot layout.  Load item: IN_ROWS rows of T theta elements.  Output item (one per worker):
-// [omega T floats | Delta T floats | (BULK) new theta T elements].
-// BULK: the outputs leave through bulk stores from the ring slot instead of st.global from
-// registers.
-template <typename TH, bool BULK>
-__global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParams P) {
-  constexpr int EB = (int)sizeof(TH);
-  constexpr int CW = TmemCell<TH>::COLS;
-  constexpr int IN_ROWS = 8 / EB;                    // theta rows per load item
-  constexpr long long ALN = 16 / EB;                 // elements per 16 bytes of theta
-  extern __shared__ __align__(128) unsigned char smem[];
-  // [0,64) ring full, [64,128) ring empty (consumers done), [128,132) TMEM base address,
-  // [192,448) per-slot retire information (BULK)
-  const uint32_t bars = smem_u32(smem);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 128);
-  SlotInfo* sinfo = reinterpret_cast<SlotInfo*>(smem + 192);
-  unsigned char* ring0 = smem + P.ring_off;
-  unsigned char* meta0 = smem + P.meta_off;
-  TH* const theta = reinterpret_cast<TH*>(P.theta);
-  const TH* const theta_in = reinterpret_cast<const TH*>(P.theta_in);
-  const int total = P.tile_prefix[P.m];
-  const int R = P.ring, K = P.K, q = P.q, T = P.T;
-  const int my_tiles = (int)blockIdx.x < total ? (total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
-  const int ntheta = (K + IN_ROWS - 1) / IN_ROWS;                  // load items per tile
-  const int nout = K;                                              // output items per tile
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-  if (threadIdx.x == 0) {
-    for (int r = 0; r < R; ++r) {
-      mbar_init(bars + 8 * r, 1);
-      mbar_init(bars + 64 + 8 * r, 512);                 // every consumer thread arrives
-    }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  }
-  if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                 "r"((uint32_t)P.ncols)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
-  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-  const uint32_t tmem_base = *tmem_slot;
-
-  if (warp == 0) {
-    // ------------------------------------------------------------------ producer warp
-    int comp = 0, pfx_lo = 0, pfx_hi = 0;
-    long long cb = 0, ce = 0;
-    if (my_tiles > 0) {
-      int lo_i = 0, hi_i = P.m;
-      while (hi_i - lo_i > 1) {
-        const int mid = (lo_i + hi_i) >> 1;
-        if (__ldg(P.tile_prefix + mid) <= (int)blockIdx.x) lo_i = mid; else hi_i = mid;
-      }
-      comp = lo_i;
-      pfx_lo = __ldg(P.tile_prefix + comp);
-      pfx_hi = __ldg(P.tile_prefix + comp + 1);
-      cb = __ldg(P.off + comp);
-      ce = __ldg(P.off + comp + 1);
-    }
-    int gi = 0;              // ring items requested so far
-    bool ok = true;
-    // BULK: item j is finished by the consumers -> send its results out of the slot.  One bulk
-    // group per item (an empty one for load items) so that "all but the newest group have been
-    // read" means exactly "the slot about to be refilled is free".
-    auto retire = [&](int j) -> bool {
-      const int slot = j % R;
-      bool fine = mbar_wait_bounded(bars + 64 + 8 * slot, (j / R) & 1, P.status);
-      if (!__all_sync(0xffffffffu, fine)) return false;
-      if (lane == 0) {
-        const SlotInfo si = sinfo[slot];
-        if (si.k >= 0 && si.se > si.sb) {
-          const uint32_t base = smem_u32(ring0 + (size_t)slot * P.slot_stride);
-          const uint32_t skip = (uint32_t)(si.sb - si.e0), n = (uint32_t)(si.se - si.sb);
-          const long long at = (long long)si.k * P.ld + si.sb;
-          asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(P.omega + at), "r"(base + skip * 4u), "r"(n * 4u) : "memory");
-          asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(P.delta + at), "r"(base + (uint32_t)T * 4u + skip * 4u), "r"(n * 4u) : "memory");
-          asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(theta + at), "r"(base + (uint32_t)T * 8u + skip * EB), "r"(n * EB) : "memory");
-        }
-        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-      }
-      __syncwarp();
-      return true;
-    };
-    for (int it = 0; it < my_tiles && ok; ++it) {
-      const int w = (int)blockIdx.x + it * (int)gridDim.x;
-      if (w >= pfx_hi) {
-        while (w >= pfx_hi) {
-          ++comp;
-          pfx_lo = pfx_hi;
-          pfx_hi = __ldg(P.tile_prefix + comp + 1);
-        }
-        cb = __ldg(P.off + comp);
-        ce = __ldg(P.off + comp + 1);
-      }
-      const long long e0 = (cb & ~(long long)(kAlign - 1)) + (long long)(w - pfx_lo) * T;
-      long long run = P.ld - e0;
-      if (run > T) run = T;
-      const long long lo = cb > e0 ? cb : e0, hi = ce < e0 + T ? ce : e0 + T;
-      // tile descriptor + neighbour table into the meta ring (4 entries: the consumers are never
-      // more than a ring of items, i.e. at most three tiles, behind)
-      unsigned char* meta = meta0 + (size_t)(it & 3) * P.meta_stride;
-      TileDesc* d = reinterpret_cast<TileDesc*>(meta);
-      int* snb = reinterpret_cast<int*>(meta + sizeof(TileDesc));
-      if (d->comp != comp || it < 4) {
-        const int32_t* gnb = P.nbr + (size_t)comp * K * q;
-        for (int x = lane; x < K * q; x += 32) snb[x] = __ldg(gnb + x);
-      }
-      __syncwarp();
-      if (lane == 0) {
-        d->e0 = e0;
-        d->lo = lo;
-        d->hi = hi;
-        d->comp = comp;
-      }
-      __syncwarp();
-      for (int item = 0; item < ntheta + nout && ok; ++item, ++gi) {
-        const int slot = gi % R;
-        if (BULK) {
-          if (gi >= R - 1) ok = retire(gi - (R - 1));       // consumers done with it; its stores go out
-          if (!ok) break;
-          if (gi >= R && lane == 0)                          // the slot's own stores have read it
-            asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-          __syncwarp();
-        } else if (gi >= R) {
-          bool fine = mbar_wait_bounded(bars + 64 + 8 * slot, ((gi / R) - 1) & 1, P.status);
-          ok = __all_sync(0xffffffffu, fine);
-          if (!ok) break;
-        }
-        if (lane == 0) {
-          const uint32_t full = bars + 8 * slot;
-          const uint32_t dst = smem_u32(ring0 + (size_t)slot * P.slot_stride);
-          if (BULK) {
-            SlotInfo si;
-            si.e0 = e0;
-            si.sb = (lo + ALN - 1) & ~(ALN - 1);
-            si.se = hi & ~(ALN - 1);
-            si.k = item < ntheta ? -1 : item - ntheta;
-            si.pad = 0;
-            sinfo[slot] = si;
-          }
-          if (item < ntheta) {
-            const int r0 = IN_ROWS * item;
-            const int rows = K - r0 < IN_ROWS ? K - r0 : IN_ROWS;
-            const uint32_t bytes = (uint32_t)run * EB;
-            mbar_arrive_expect_tx(full, (uint32_t)rows * bytes);
-            for (int r = 0; r < rows; ++r)
-              bulk_load_row(dst + (uint32_t)r * (uint32_t)T * EB, theta_in + (long long)(r0 + r) * P.ld + e0, bytes, full);
-          } else {
-            const long long at = (long long)(item - ntheta) * P.ld + e0;
-            const uint32_t bytes = (uint32_t)run * 4u;
-            mbar_arrive_expect_tx(full, 2u * bytes);
-            bulk_load_row(dst, P.omega + at, bytes, full);
-            bulk_load_row(dst + (uint32_t)T * 4u, P.delta + at, bytes, full);
-          }
-        }
-      }
-    }
-    if (BULK) {
-      for (int j = gi > R - 1 ? gi - (R - 1) : 0; j < gi && ok; ++j) ok = retire(j);
-      if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-      __syncwarp();
-    }
-    if (!ok) {
-      for (int j = gi > R ? gi - R : 0; j < gi; ++j)
-        mbar_wait_bounded(bars + 8 * (j % R), (j / R) & 1, P.status);
-    }
-  } else {
-    // -------------------------------------------------------------------- consumer warps (16)
-    // lanes this warp reaches, and which of the four warps of that lane quarter it is
-    // (24 consumer warps were measured slower than 16)
-    const int quarter = warp & 3, sub = (warp - 1) >> 2;
-    const uint32_t tlane = tmem_base + ((uint32_t)(quarter * 32) << 16);
-    const int ngroups = T / 512;                  // element groups of 128 x 4 per row
-    int gi = 0;
-    bool ok = true;
-    for (int it = 0; it < my_tiles && ok; ++it) {
-      const unsigned char* meta = meta0 + (size_t)(it & 3) * P.meta_stride;
-      const TileDesc* d = reinterpret_cast<const TileDesc*>(meta);
-      const int* snb = reinterpret_cast<const int*>(meta + sizeof(TileDesc));
-      long long e0 = 0, lo = 0, hi = 0, sb = 0, se = 0;
-      for (int item = 0; item < ntheta + nout && ok; ++item, ++gi) {
-        const int slot = gi % R;
-        bool fine = mbar_wait_bounded(bars + 8 * slot, (gi / R) & 1, P.status);
-        ok = __all_sync(0xffffffffu, fine);
-        if (!ok) break;
-        if (item == 0) {
-          e0 = d->e0; lo = d->lo; hi = d->hi;
-          sb = (lo + ALN - 1) & ~(ALN - 1);       // whole 16-byte pieces of theta inside the tile
-          se = hi & ~(ALN - 1);
-        }
-        unsigned char* const sbase = ring0 + (size_t)slot * P.slot_stride;
-        if (item < ntheta) {
-          // deposit the theta rows of this item into this thread's TMEM cells
-          const int r0 = IN_ROWS * item;
-          const TH* rows_in = reinterpret_cast<const TH*>(sbase);
-          for (int g = sub; g < ngroups; g += 4) {
-            const int col = (g * 128 + quarter * 32 + lane) * 4;
-#pragma unroll
-            for (int r = 0; r < IN_ROWS; ++r)
-              if (r0 + r < K)
-                TmemCell<TH>::deposit(tlane + (uint32_t)((g * K + r0 + r) * CW), rows_in + (size_t)r * T + col);
-          }
-          asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-        } else {
-          const int k = item - ntheta;
-          float* row0 = reinterpret_cast<float*>(sbase);
-          float* row1 = row0 + T;
-          TH* row2 = reinterpret_cast<TH*>(row1 + T);      // BULK: the new theta
-          for (int g = sub; g < ngroups; g += 4) {
-            const int col = (g * 128 + quarter * 32 + lane) * 4;
-            const long long e = e0 + col;
-            float a[4], t[4];
-            __syncwarp();                          // lanes that left the last group early rejoin
-            tmem_gather<TH>(tlane + (uint32_t)(g * K * CW), k, snb + k * q, q, a);
-            if (e >= hi || e + 4 <= lo) continue;
-            average_divide(a, P.qp1, P.inv_qp1, P.inv_exact);
-            const float4 W = *reinterpret_cast<const float4*>(row0 + col);
-            const float4 D = *reinterpret_cast<const float4*>(row1 + col);
-            float wv[4] = {W.x, W.y, W.z, W.w}, dv[4] = {D.x, D.y, D.z, D.w};
-#pragma unroll
-            for (int x = 0; x < 4; ++x) bmuf_filter<TH>(a[x], wv[x], dv[x], t[x], P.eta, P.zeta);
-            const long long at = (long long)k * P.ld + e;
-            if (BULK && e >= sb && e + 4 <= se) {
-              *reinterpret_cast<float4*>(row0 + col) = make_float4(wv[0], wv[1], wv[2], wv[3]);
-              *reinterpret_cast<float4*>(row1 + col) = make_float4(dv[0], dv[1], dv[2], dv[3]);
-              TmemCell<TH>::sts_quad(row2 + col, t);
-            } else if (!BULK && e >= lo && e + 4 <= hi) {
-              __stcs(reinterpret_cast<float4*>(P.delta + at), make_float4(dv[0], dv[1], dv[2], dv[3]));
-              __stcs(reinterpret_cast<float4*>(P.omega + at), make_float4(wv[0], wv[1], wv[2], wv[3]));
-              ThetaTraits<TH>::stg_quad(theta + at, t);
-            } else {
-              for (int x = 0; x < 4; ++x) {
-                if (e + x >= lo && e + x < hi) {
-                  P.delta[at + x] = dv[x];
-                  P.omega[at + x] = wv[x];
-                  theta[at + x] = ThetaTraits<TH>::narrow(t[x]);
-                }
-              }
-            }
-          }
-        }
-        if (BULK && item >= ntheta) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        mbar_arrive(bars + 64 + 8 * slot);
-      }
-    }
-  }
-  // every thread arrives here; only then is the tensor memory given back
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
-  if (warp == 0) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)P.ncols) : "memory");
-  }
-}
-
-// Self-test of average_divide: runs its correction route (never the power-of-two shortcut) and
-// the plain division over all 2^32 bit patterns of the dividend, four consecutive patterns per
-// call as in the round kernels, and counts the patterns whose results differ in any bit.
-__global__ void __launch_bounds__(256) divide_selftest_kernel(float b, float y, unsigned long long* mismatches,
-                                                              unsigned int* first_bad) {
-  const unsigned long long nquads = 1ull << 30;
-  unsigned int bad = 0, first = 0xFFFFFFFFu;
-  for (unsigned long long qd = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; qd < nquads;
-       qd += (unsigned long long)gridDim.x * blockDim.x) {
-    float a[4], ref[4];
-#pragma unroll
-    for (int x = 0; x < 4; ++x) {
-      a[x] = __uint_as_float((unsigned int)(qd * 4 + x));
-      ref[x] = __fdiv_rn(a[x], b);
-    }
-    average_divide(a, b, y, 0);
-#pragma unroll
-    for (int x = 0; x < 4; ++x) {
-      if (__float_as_uint(a[x]) != __float_as_uint(ref[x])) {
-        ++bad;
-        const unsigned int pat = (unsigned int)(qd * 4 + x);
-        if (pat < first) first = pat;
-      }
-    }
-  }
-  if (bad) {
-    atomicAdd(mismatches, (unsigned long long)bad);
-    atomicMin(first_bad, first);
-  }
-}
-
-// Self-test of the bounded wait: one warp waits on a barrier that nothing will ever signal.  The
-// wait must expire, set the status word and return; nothing here can hang or trap.
-__global__ void wait_timeout_selftest_kernel(int32_t* status, int32_t* returned) {
-  __shared__ __align__(8) unsigned long long bar_storage;
-  const uint32_t bar = smem_u32(&bar_storage);
-  if (threadIdx.x == 0) {
-    mbar_init(bar, 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  __syncwarp();
-  const bool ok = mbar_wait_bounded(bar, 0, status);
-  if (threadIdx.x == 0) *returned = ok ? 1 : 2;
-}
-
-// =================================================================================================
-// Synthetic local step: theta <- store(theta - lr * (sigma * z)), z from the four 16-bit halves
-// of two Philox words (Irwin-Hall, n = 4), keyed by (seed, step, worker, global element pair).
-// =================================================================================================
-__device__ __forceinline__ float noise_from_words(uint32_t a, uint32_t b) {
-  const int sum = (int)((a & 0xFFFFu) + (a >> 16) + (b & 0xFFFFu) + (b >> 16));
-  return __fmul_rn((float)(sum - 131070), 0x1.bb67aep-16f);   // 1 / sqrt((2^32 - 1) / 3)
-}
-
-template <typename TH>
-__global__ void __launch_bounds__(256) perturb_kernel(TH* theta, int K, long long N, long long ld,
-                                                      uint32_t key0, uint32_t key1, uint32_t step0,
-                                                      int nsteps, float lr, float sigma,
-                                                      long long elem_base) {
-  constexpr int VEC = ThetaTraits<TH>::VEC;
-  const long long nvec = (N + VEC - 1) / VEC;
-  const int k = blockIdx.y;                 // one grid row per worker
-  for (long long iv = (long long)blockIdx.x * blockDim.x + threadIdx.x; iv < nvec;
-       iv += (long long)gridDim.x * blockDim.x) {
-    const long long e = iv * VEC;
-    TH* row = theta + (long long)k * ld + e;
-    const int n = N - e < VEC ? (int)(N - e) : VEC;
-    float v[VEC];
-    if (n == VEC) {
-      ThetaTraits<TH>::lds(row, v);   // a 16-byte load (rows and vectors are 16-byte aligned)
-    } else {
-      for (int x = 0; x < n; ++x) v[x] = ThetaTraits<TH>::widen(row[x]);
-    }
-    for (int s = 0; s < nsteps; ++s) {
-      unsigned long long have = ~0ull;
-      Philox4 r = {0, 0, 0, 0};
-#pragma unroll
-      for (int x = 0; x < VEC; ++x) {
-        if (x < n) {
-          const unsigned long long ge = (unsigned long long)(elem_base + e + x);
-          const unsigned long long pair = ge >> 1;
-          if (pair != have) {
-            Philox4 ctr = {(uint32_t)pair, (uint32_t)(pair >> 32), (uint32_t)k, step0 + (uint32_t)s};
-            r = philox4x32_10(ctr, key0, key1);
-            have = pair;
-          }
-          const float z = (ge & 1) ? noise_from_words(r.z, r.w) : noise_from_words(r.x, r.y);
-          const float upd = __fmul_rn(lr, __fmul_rn(sigma, z));
-          v[x] = ThetaTraits<TH>::round_store(__fsub_rn(v[x], upd));
-        }
-      }
-    }
-    if (n == VEC) {
-      ThetaTraits<TH>::stg(row, v);
-    } else {
-      for (int x = 0; x < n; ++x) row[x] = ThetaTraits<TH>::narrow(v[x]);
-    }
-  }
-}
-
-// =================================================================================================
-// Local step with the optimiser of the paper's experiments (Section 3.2): Adagrad with the
-// gradient norm of a group of components clipped.  Three kernels: per-(worker, block) partial sums
-// of squares in double over the clip ranges, a fixed-order final sum that turns them into one
-// scale factor per worker (deterministic: no atomics), and the element-wise update.
-// =================================================================================================
-constexpr int kMaxClipRanges = 16;
-constexpr int kNormBlocks = 128;    // partial sums per worker
-
-struct ClipRanges {
-  int n;
-  long long begin[kMaxClipRanges], end[kMaxClipRanges];
-};
-
-__global__ void __launch_bounds__(256) sumsq_partial_kernel(const float* grad, long long ld,
-                                                            ClipRanges R, double* partial) {
-  const int k = blockIdx.y;
-  const float* row = grad + (long long)k * ld;
-  // four independent partial sums per thread keep four loads in flight; the order of the
-  // additions is fixed by the launch shape, so the result is reproducible
-  double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
-  const long long stride = (long long)gridDim.x * blockDim.x;
-  for (int r = 0; r < R.n; ++r) {
-    long long e = R.begin[r] + (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    for (; e + 3 * stride < R.end[r]; e += 4 * stride) {
-      const double g0 = (double)row[e], g1 = (double)row[e + stride];
-      const double g2 = (double)row[e + 2 * stride], g3 = (double)row[e + 3 * stride];
-      a0 += g0 * g0; a1 += g1 * g1; a2 += g2 * g2; a3 += g3 * g3;
-    }
-    for (; e < R.end[r]; e += stride) {
-      const double g = (double)row[e];
-      a0 += g * g;
-    }
-  }
-  double acc = (a0 + a1) + (a2 + a3);
-  __shared__ double warp_sum[8];
-  for (int d = 16; d > 0; d >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, d);
-  if ((threadIdx.x & 31) == 0) warp_sum[threadIdx.x >> 5] = acc;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    double s = 0.0;
-    for (int w = 0; w < 8; ++w) s += warp_sum[w];
-    partial[(size_t)k * gridDim.x + blockIdx.x] = s;
-  }
-}
-
-__global__ void clip_scale_kernel(const double* partial, int K, int nblk, float clip_norm,
-                                  float* scale) {
-  const int k = blockIdx.x * blockDim.x + threadIdx.x;
-  if (k >= K) return;
-  double s = 0.0;
-  for (int b = 0; b < nblk; ++b) s += partial[(size_t)k * nblk + b];
-  const float norm = (float)sqrt(s);
-  scale[k] = __fdiv_rn(clip_norm, norm > clip_norm ? norm : clip_norm);
-}
-
-// The element-wise Adagrad update as a streaming kernel: 20 bytes per replica-parameter (fp32
-// theta) and nothing else, so it is built like the fused round: persistent CTAs, a producer warp
-// that has the copy engine fetch [gradient | accumulator | theta] chunks of one worker's row into a
-// ring of shared-memory slots, 16 consumer warps that update accumulator and theta inside the slot,
-// and bulk stores that send the two rows back.  Chunks are T consecutive elements of one row;
-// consecutive CTAs take consecutive chunks.  Rows are read up to the padded stride (a multiple of
-// 16 bytes); stores cover whole 16-byte pieces below N, the few elements after the last whole
-// piece are stored by the thread that computed them, and the padding is never written.
-struct AdagradParams {
-  void* theta;
-  const float* grad;
-  float* accum;
-  const float* scale;      // [K] clip factor per worker, or NULL
-  int32_t* status;
-  long long N, ld;
-  int K, T, ring, chunks_per_row, groups;   // groups: consumer thread groups (1, 2 or 4)
-  uint32_t ring_off, slot_stride;
-  float lr, eps;
-  ClipRanges R;
-};
-
-// What producer and consumers share about the chunk in a slot: it starts at element e0 of worker
-// k's row and ends before hi (<= N); whole 16-byte pieces end at se; `where` places it relative
-// to the clip ranges (0 outside all, 1 inside one, 2 mixed) and sc is the worker's clip factor.
-struct AdagradSlot { long long e0, hi, se; int k; int where; float sc; int pad; };
-
-template <typename TH>
-__global__ void __launch_bounds__(544, 1) adagrad_stream_kernel(const AdagradParams P) {
-  constexpr int EB = (int)sizeof(TH);
-  constexpr long long ALN = 16 / EB;                 // elements per 16 bytes of theta
-  extern __shared__ __align__(128) unsigned char smem[];
-  // [0,64) slot full, [64,128) slot done (consumers), [128,512) per-slot chunk descriptors
-  const uint32_t bars = smem_u32(smem);
-  AdagradSlot* sinfo = reinterpret_cast<AdagradSlot*>(smem + 128);
-  unsigned char* ring0 = smem + P.ring_off;
-  TH* const theta = reinterpret_cast<TH*>(P.theta);
-  const int R = P.ring, T = P.T;
-  const long long total = (long long)P.chunks_per_row * P.K;
-  const int my_chunks = (long long)blockIdx.x < total
-                            ? (int)((total - (long long)blockIdx.x + (long long)gridDim.x - 1) / (long long)gridDim.x)
-                            : 0;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-  if (threadIdx.x == 0) {
-    for (int r = 0; r < R; ++r) {
-      mbar_init(bars + 8 * r, 1);
-      mbar_init(bars + 64 + 8 * r, 512 / P.groups);      // every thread of one consumer group arrives
-    }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  }
-  __syncthreads();
-
-  if (warp == 0) {
-    // ------------------------------------------------------------------ producer warp
-    bool ok = true;
-    // chunk j is finished by the consumers -> send accumulator and theta out of the slot.  One
-    // bulk group per chunk, so that "all but the newest group have been read" means exactly
-    // "the slot about to be refilled is free".
-    auto retire = [&](int j) -> bool {
-      const int slot = j % R;
-      bool fine = mbar_wait_bounded(bars + 64 + 8 * slot, (j / R) & 1, P.status);
-      if (!__all_sync(0xffffffffu, fine)) return false;
-      if (lane == 0) {
-        const AdagradSlot si = sinfo[slot];
-        if (si.se > si.e0) {
-          const uint32_t base = smem_u32(ring0 + (size_t)slot * P.slot_stride);
-          const uint32_t n = (uint32_t)(si.se - si.e0);
-          const long long at = (long long)si.k * P.ld + si.e0;
-          asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(P.accum + at), "r"(base + (uint32_t)T * 4u), "r"(n * 4u) : "memory");
-          asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(theta + at), "r"(base + (uint32_t)T * 8u), "r"(n * EB) : "memory");
-        }
-        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-      }
-      __syncwarp();
-      return true;
-    };
-    // this CTA's chunks are w = blockIdx.x + it * gridDim.x: keep (row, chunk in row) incrementally
-    int k = (int)(blockIdx.x / (unsigned)P.chunks_per_row);
-    int cin = (int)(blockIdx.x % (unsigned)P.chunks_per_row);
-    const int dk = (int)(gridDim.x / (unsigned)P.chunks_per_row), dc = (int)(gridDim.x % (unsigned)P.chunks_per_row);
-    float sc = (P.scale && lane == 0 && my_chunks > 0) ? __ldg(P.scale + k) : 1.0f;
-    int it = 0;
-    for (; it < my_chunks && ok; ++it) {
-      const long long e0 = (long long)cin * T;
-      long long run = P.ld - e0;                         // a row ends at ld: never read past it
-      if (run > T) run = T;
-      const long long hi = e0 + T < P.N ? e0 + T : P.N;
-      const int slot = it % R;
-      if (it >= R - 1) ok = retire(it - (R - 1));        // consumers done with it; its stores go out
-      if (!ok) break;
-      if (it >= R && lane == 0)                          // the slot's own stores have read it
-        asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-      __syncwarp();
-      if (lane == 0) {
-        AdagradSlot si;
-        si.e0 = e0; si.hi = hi; si.se = hi & ~(ALN - 1); si.k = k; si.where = 0; si.sc = sc; si.pad = 0;
-        if (P.scale) {
-          for (int r = 0; r < P.R.n; ++r) {
-            if (e0 >= P.R.begin[r] && hi <= P.R.end[r]) si.where = 1;
-            else if (e0 < P.R.end[r] && hi > P.R.begin[r] && si.where == 0) si.where = 2;
-          }
-        }
-        sinfo[slot] = si;
-        const uint32_t full = bars + 8 * slot;
-        const uint32_t dst = smem_u32(ring0 + (size_t)slot * P.slot_stride);
-        const long long at = (long long)k * P.ld + e0;
-        mbar_arrive_expect_tx(full, (uint32_t)run * (8u + EB));
-        bulk_load_row(dst, P.grad + at, (uint32_t)run * 4u, full);
-        bulk_load_row(dst + (uint32_t)T * 4u, P.accum + at, (uint32_t)run * 4u, full);
-        bulk_load_row(dst + (uint32_t)T * 8u, theta + at, (uint32_t)run * EB, full);
-      }
-      // next chunk of this CTA
-      const int k_before = k;
-      k += dk; cin += dc;
-      if (cin >= P.chunks_per_row) { cin -= P.chunks_per_row; ++k; }
-      if (P.scale && lane == 0 && k != k_before && it + 1 < my_chunks) sc = __ldg(P.scale + k);
-    }
-    for (int j = it > R - 1 ? it - (R - 1) : 0; j < it && ok; ++j) ok = retire(j);
-    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-    __syncwarp();
-    if (!ok) {
-      // leave only after the copies already requested into this CTA's shared memory have landed
-      for (int j = it > R ? it - R : 0; j < it; ++j)
-        mbar_wait_bounded(bars + 8 * (j % R), (j / R) & 1, P.status);
-    }
-    return;
-  }
-
-  // -------------------------------------------------------------------- consumer warps (16)
-  // The consumer threads form `groups` groups that take chunks in turn, so that several chunks
-  // are being updated at once: one chunk's chain of loads, square root, divide and stores is
-  // long, and a single group would make the ring wait for it.
-  const int gsize = 512 / P.groups;
-  const int grp = (threadIdx.x - 32) / gsize, c = (threadIdx.x - 32) - grp * gsize;
-  for (int it = grp; it < my_chunks; it += P.groups) {
-    const int slot = it % R;
-    if (!mbar_wait_bounded(bars + 8 * slot, (it / R) & 1, P.status)) return;
-    const AdagradSlot si = sinfo[slot];
-    const long long e0 = si.e0, hi = si.hi, se = si.se;
-    const int where = si.where;
-    const float sc = si.sc;
-    float* sg = reinterpret_cast<float*>(ring0 + (size_t)slot * P.slot_stride);
-    float* sa = sg + T;
-    TH* sth = reinterpret_cast<TH*>(sa + T);
-#pragma unroll 2
-    for (int col = c * 4; col < T; col += gsize * 4) {
-      const long long e = e0 + col;
-      if (e >= hi) break;
-      const float4 gv = *reinterpret_cast<const float4*>(sg + col);
-      const float4 av = *reinterpret_cast<const float4*>(sa + col);
-      float g[4] = {gv.x, gv.y, gv.z, gv.w}, a[4] = {av.x, av.y, av.z, av.w}, th[4];
-      ThetaTraits<TH>::lds_quad(sth + col, th);
-#pragma unroll
-      for (int x = 0; x < 4; ++x) {
-        bool inside = where == 1;
-        if (where == 2)
-          for (int r = 0; r < P.R.n; ++r) inside = inside || (e + x >= P.R.begin[r] && e + x < P.R.end[r]);
-        float gx = g[x];
-        if (inside) gx = __fmul_rn(gx, sc);
-        a[x] = __fadd_rn(a[x], __fmul_rn(gx, gx));
-        const float denom = __fadd_rn(__fsqrt_rn(a[x]), P.eps);
-        th[x] = __fsub_rn(th[x], __fdiv_rn(__fmul_rn(P.lr, gx), denom));
-      }
-      if (e + 4 <= se) {
-        *reinterpret_cast<float4*>(sa + col) = make_float4(a[0], a[1], a[2], a[3]);
-        TmemCell<TH>::sts_quad(sth + col, th);
-      } else {
-        // after the last whole 16-byte piece of the row: only the elements below N
-        const long long at = (long long)si.k * P.ld + e;
-        for (int x = 0; x < 4; ++x) {
-          if (e + x < hi) {
-            P.accum[at + x] = a[x];
-            theta[at + x] = ThetaTraits<TH>::narrow(th[x]);
-          }
-        }
-      }
-    }
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    mbar_arrive(bars + 64 + 8 * slot);
-  }
-}
-
-// =================================================================================================
-// Initialisation line of Algorithm 1 and its return line.
-// =================================================================================================
-template <typename TH>
-__global__ void __launch_bounds__(256) init_kernel(const TH* theta0, TH* theta, float* omega,
-                                                   float* delta, int K, long long N, long long ld) {
-  constexpr int VEC = ThetaTraits<TH>::VEC;
-  const long long nvec = (N + VEC - 1) / VEC;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec;
-       i += (long long)gridDim.x * blockDim.x) {
-    const long long e = i * VEC;
-    if (e + VEC <= N) {
-      const uint4 raw = *reinterpret_cast<const uint4*>(theta0 + e);   // 16 bytes of theta_0
-      float f[VEC];
-      ThetaTraits<TH>::lds(theta0 + e, f);
-      const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int k = 0; k < K; ++k) {
-        const long long at = (long long)k * ld + e;
-        __stcs(reinterpret_cast<uint4*>(theta + at), raw);
-#pragma unroll
-        for (int h = 0; h < VEC / 4; ++h) {
-          __stcs(reinterpret_cast<float4*>(omega + at) + h,
-                 make_float4(f[4 * h], f[4 * h + 1], f[4 * h + 2], f[4 * h + 3]));
-          __stcs(reinterpret_cast<float4*>(delta + at) + h, zero);
-        }
-      }
-    } else {
-      for (long long x = e; x < N; ++x) {
-        const TH v = theta0[x];
-        for (int k = 0; k < K; ++k) {
-          const long long at = (long long)k * ld + x;
-          theta[at] = v;
-          omega[at] = ThetaTraits<TH>::widen(v);
-          delta[at] = 0.0f;
-        }
-      }
-    }
-  }
-}
-
-template <typename TH>
-__global__ void __launch_bounds__(256) final_average_kernel(const TH* theta, TH* out, int K,
-                                                            long long N, long long ld) {
-  constexpr int VEC = ThetaTraits<TH>::VEC;
-  const float fk = (float)K;
-  const long long nvec = (N + VEC - 1) / VEC;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec;
-       i += (long long)gridDim.x * blockDim.x) {
-    const long long e = i * VEC;
-    if (e + VEC <= N) {
-      float s[VEC], t[VEC];
-      ThetaTraits<TH>::lds(theta + e, s);
-      for (int k = 1; k < K; ++k) {                  // k = 0, 1, ..., K-1 in that order
-        ThetaTraits<TH>::lds(theta + (long long)k * ld + e, t);
-#pragma unroll
-        for (int x = 0; x < VEC; ++x) s[x] = __fadd_rn(s[x], t[x]);
-      }
-#pragma unroll
-      for (int x = 0; x < VEC; ++x) s[x] = __fdiv_rn(s[x], fk);
-      ThetaTraits<TH>::stg(out + e, s);
-    } else {
-      for (long long x = e; x < N; ++x) {
-        float s = ThetaTraits<TH>::widen(theta[x]);
-        for (int k = 1; k < K; ++k)
-          s = __fadd_rn(s, ThetaTraits<TH>::widen(theta[(long long)k * ld + x]));
-        out[x] = ThetaTraits<TH>::narrow(__fdiv_rn(s, fk));
-      }
-    }
-  }
-}
-
-// =================================================================================================
-// One worker per GPU ("peer" form): this GPU holds worker `rank`'s theta (two buffers, read one /
-// write the other), omega and Delta; the other workers' theta buffers are peer-mapped pointers.
-// For every participating component the worker's q neighbours are drawn exactly as in the
-// resident form, and the fused kernel pulls their slices straight from peer memory with
-// non-multicast bulk copies into the same shared-memory stage as its own theta, omega and Delta
-// slices, averages (own first, then draw order), filters, and writes omega and Delta in place and
-// the new theta into the OTHER buffer: peers that are still reading this worker's current buffer
-// never see a half-updated replica.  Components that do not take part are copied through to the
-// other buffer.  Every row of a stage passes through once, so stages are simply pipelined.
-// =================================================================================================
-struct PeerPlanParams {
-  int K, m, p, q, comp_base, rank, use_mask;
-  uint64_t seed, round;
-  const int32_t* periods;
-  const uint8_t* mask;
-  int32_t* nbr;    // [m][q] neighbours of worker `rank`
-  uint8_t* due;    // [m]
-};
-
-__global__ void __launch_bounds__(256) peer_plan_kernel(PeerPlanParams P) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= P.m) return;
-  P.due[i] = P.use_mask ? (P.mask[i] != 0) : (P.round % (uint64_t)P.periods[i] == 0);
-  if (P.q == 0) return;
-  int32_t a[kMaxCand];
-  const int c = ring_candidates(P.rank, P.K, P.p, a);
-  Philox4 r = {0, 0, 0, 0};
-  for (int j = 0; j < P.q && j < c; ++j) {
-    if ((j & 3) == 0) {
-      Philox4 ctr = {(uint32_t)P.round, (uint32_t)(P.round >> 32), (uint32_t)(P.comp_base + i),
-                     (uint32_t)P.rank | ((uint32_t)(j >> 2) << 16)};
-      r = philox4x32_10(ctr, (uint32_t)P.seed, (uint32_t)(P.seed >> 32) ^ kTagSampler);
-    }
-    const uint32_t u = (j & 3) == 0 ? r.x : (j & 3) == 1 ? r.y : (j & 3) == 2 ? r.z : r.w;
-    const int t = j + (int)__umulhi(u, (uint32_t)(c - j));
-    const int32_t tmp = a[j];
-    a[j] = a[t];
-    a[t] = tmp;
-    P.nbr[(size_t)i * P.q + j] = a[j];
-  }
-}
-
-struct PeerParams {
-  const void* const* theta_in;   // device array [K]: worker j's current theta buffer (peers included)
-  void* theta_out;               // this worker's other buffer
-  float* omega;                  // this worker's, [N]
-  float* delta;
-  const int64_t* off;            // [m+1]
-  const int32_t* tile_prefix;    // [m+1], over ALL components
-  const int32_t* nbr;            // [m][q]
-  const uint8_t* due;            // [m]
-  int32_t* status;
-  long long N;                   // columns; rows are read up to N rounded up to 8 (<= ld)
-  int rank, m, q, mode;
-  float eta, zeta, qp1, inv_qp1;
-  int inv_exact;
-  int T, stages, ncons;
-  uint32_t stage_stride, omega_off, delta_off, desc_off;   // stage: [q+1 theta rows | omega | Delta | desc]
-};
-
-template <typename TH>
-__global__ void __launch_bounds__(1024, 1) peer_round_kernel(const PeerParams P) {
-  constexpr int VEC = 4;
-  extern __shared__ __align__(128) unsigned char smem[];
-  const uint32_t bars = smem_u32(smem);            // [0,64) full, [64,128) empty
-  unsigned char* stage0 = smem + 128;
-  const int total = P.tile_prefix[P.m];
-  const int S = P.stages;
-  const bool bmuf = P.mode == GBMUF_MODE_BMUF;
-  const int my_tiles = (int)blockIdx.x < total ? (total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < S; ++s) {
-      mbar_init(bars + 8 * s, 1);
-      mbar_init(bars + 64 + 8 * s, P.ncons);
-    }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  }
-  __syncthreads();
-
-  if (threadIdx.x < 32) {
-    // ------------------------------------------------------------------ producer warp
-    const int lane = threadIdx.x;
-    int comp = 0, pfx_lo = 0, pfx_hi = 0;
-    long long cb = 0, ce = 0;
-    if (my_tiles > 0) {
-      int lo_i = 0, hi_i = P.m;
-      while (hi_i - lo_i > 1) {
-        const int mid = (lo_i + hi_i) >> 1;
-        if (__ldg(P.tile_prefix + mid) <= (int)blockIdx.x) lo_i = mid; else hi_i = mid;
-      }
-      comp = lo_i;
-      pfx_lo = __ldg(P.tile_prefix + comp);
-      pfx_hi = __ldg(P.tile_prefix + comp + 1);
-      cb = __ldg(P.off + comp);
-      ce = __ldg(P.off + comp + 1);
-    }
-    int issued = 0;
-    bool ok = true;
-    const long long row_end = (P.N + kAlign - 1) & ~(long long)(kAlign - 1);
-    for (int it = 0; it < my_tiles; ++it) {
-      const int w = (int)blockIdx.x + it * (int)gridDim.x;
-      const int s = it % S;
-      if (it >= S) {
-        ok = mbar_wait_bounded(bars + 64 + 8 * s, ((it / S) - 1) & 1, P.status);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-      }
-      if (w >= pfx_hi) {
-        while (w >= pfx_hi) {
-          ++comp;
-          pfx_lo = pfx_hi;
-          pfx_hi = __ldg(P.tile_prefix + comp + 1);
-        }
-        cb = __ldg(P.off + comp);
-        ce = __ldg(P.off + comp + 1);
-      }
-      const long long e0 = (cb & ~(long long)(kAlign - 1)) + (long long)(w - pfx_lo) * P.T;
-      long long load_end = (ce + kAlign - 1) & ~(long long)(kAlign - 1);
-      if (load_end > e0 + P.T) load_end = e0 + P.T;
-      if (load_end > row_end) load_end = row_end;
-      const uint32_t nelem = (uint32_t)(load_end - e0);
-      const uint32_t bytes_th = nelem * (uint32_t)sizeof(TH), bytes_f = nelem * 4u;
-      const bool due = __ldg(P.due + comp) != 0;
-      unsigned char* st = stage0 + (size_t)s * P.stage_stride;
-      if (lane == 0) {
-        TileDesc* d = reinterpret_cast<TileDesc*>(st + P.desc_off);
-        d->e0 = e0;
-        d->lo = cb > e0 ? cb : e0;
-        d->hi = ce < e0 + P.T ? ce : e0 + P.T;
-        d->comp = due ? comp : -1 - comp;            // negative: copy the component through
-      }
-      const uint32_t full = bars + 8 * s;
-      const int nrows = due ? P.q + 1 : 1;
-      if (lane == 0)
-        mbar_arrive_expect_tx(full, (uint32_t)nrows * bytes_th + ((due && bmuf) ? 2u * bytes_f : 0u));
-      __syncwarp();
-      const uint32_t sbase = smem_u32(st);
-      for (int r = lane; r < nrows; r += 32) {
-        const int src_worker = r == 0 ? P.rank : __ldg(P.nbr + (size_t)comp * P.q + (r - 1));
-        const TH* row = static_cast<const TH*>(P.theta_in[src_worker]);   // own or a peer's memory
-        bulk_load_row(sbase + (uint32_t)r * (uint32_t)P.T * (uint32_t)sizeof(TH), row + e0, bytes_th, full);
-      }
-      if (due && bmuf && lane == 0) {
-        bulk_load_row(sbase + P.omega_off, P.omega + e0, bytes_f, full);
-        bulk_load_row(sbase + P.delta_off, P.delta + e0, bytes_f, full);
-      }
-      issued = it + 1;
-    }
-    if (!ok) {
-      for (int it = issued > S ? issued - S : 0; it < issued; ++it)
-        mbar_wait_bounded(bars + 8 * (it % S), (it / S) & 1, P.status);
-    }
-    return;
-  }
-
-  // -------------------------------------------------------------------- consumer warps
-  const int c = threadIdx.x - 32;
-  const int nv = P.T / VEC, q = P.q, T = P.T;
-  TH* out = static_cast<TH*>(P.theta_out);
-  for (int it = 0; it < my_tiles; ++it) {
-    const int s = it % S;
-    if (!mbar_wait_bounded(bars + 8 * s, (it / S) & 1, P.status)) return;
-    unsigned char* st = stage0 + (size_t)s * P.stage_stride;
-    const TH* sth = reinterpret_cast<const TH*>(st);
-    const float* som = reinterpret_cast<const float*>(st + P.omega_off);
-    const float* sde = reinterpret_cast<const float*>(st + P.delta_off);
-    const TileDesc* d = reinterpret_cast<const TileDesc*>(st + P.desc_off);
-    const long long e0 = d->e0, lo = d->lo, hi = d->hi;
-    const bool due = d->comp >= 0;
-    for (int v = c; v < nv; v += P.ncons) {
-      const int col = v * VEC;
-      const long long e = e0 + col;
-      if (e >= hi || e + VEC <= lo) continue;
-      const bool whole = e >= lo && e + VEC <= hi;
-      float a[VEC], t[VEC];
-      ThetaTraits<TH>::lds_quad(sth + col, a);
-      if (!due) {                                         // not this round: carry theta over
-        if (whole) {
-          ThetaTraits<TH>::stg_quad(out + e, a);
-        } else {
-          for (int x = 0; x < VEC; ++x)
-            if (e + x >= lo && e + x < hi) out[e + x] = ThetaTraits<TH>::narrow(a[x]);
-        }
-        continue;
-      }
-      for (int j = 1; j <= q; ++j) {                      // neighbours in draw order
-        ThetaTraits<TH>::lds_quad(sth + (size_t)j * T + col, t);
-#pragma unroll
-        for (int x = 0; x < VEC; ++x) a[x] = __fadd_rn(a[x], t[x]);
-      }
-      average_divide(a, P.qp1, P.inv_qp1, P.inv_exact);
-      if (!bmuf) {
-        if (whole) {
-          ThetaTraits<TH>::stg_quad(out + e, a);
-        } else {
-          for (int x = 0; x < VEC; ++x)
-            if (e + x >= lo && e + x < hi) out[e + x] = ThetaTraits<TH>::narrow(a[x]);
-        }
-        continue;
-      }
-      const float4 W = *reinterpret_cast<const float4*>(som + col);
-      const float4 D = *reinterpret_cast<const float4*>(sde + col);
-      float wv[VEC] = {W.x, W.y, W.z, W.w}, dv[VEC] = {D.x, D.y, D.z, D.w};
-#pragma unroll
-      for (int x = 0; x < VEC; ++x) bmuf_filter<TH>(a[x], wv[x], dv[x], t[x], P.eta, P.zeta);
-      if (whole) {
-        __stcs(reinterpret_cast<float4*>(P.delta + e), make_float4(dv[0], dv[1], dv[2], dv[3]));
-        __stcs(reinterpret_cast<float4*>(P.omega + e), make_float4(wv[0], wv[1], wv[2], wv[3]));
-        ThetaTraits<TH>::stg_quad(out + e, t);
-      } else {
-        for (int x = 0; x < VEC; ++x) {
-          if (e + x >= lo && e + x < hi) {
-            P.delta[e + x] = dv[x];
-            P.omega[e + x] = wv[x];
-            out[e + x] = ThetaTraits<TH>::narrow(t[x]);
-          }
-        }
-      }
-    }
-    mbar_arrive(bars + 64 + 8 * s);
-  }
-}
 
 // =================================================================================================
 // Host side
