@@ -260,6 +260,31 @@ def run_gpu(args, w):
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
     total_sync_s = float(tt.item())
 
+    # ---- the same rounds back to back, replayed from one CUDA graph (set-up + fused kernel per
+    # round, no local step in between): what a launch-bound small model gains from a graph
+    graph_ms = None
+    if not args.no_graph:
+        gs = torch.cuda.Stream(device=dev)
+        gs.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(gs):
+            g.sync_round(rnd)
+            rnd += 1
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=gs):
+                for i in range(args.steps):
+                    g.sync_round(rnd + i)
+            rnd += args.steps
+            ga, gb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            graph.replay()                      # warm-up replay
+            ga.record(gs)
+            graph.replay()
+            gb.record(gs)
+        gs.synchronize()
+        torch.cuda.current_stream().wait_stream(gs)
+        graph_ms = ga.elapsed_time(gb) / args.steps
+        del graph
+        status = status or g.device_status()
+
     # ---- end to end: the same round through the host-buffer entry point (replicas in page-locked
     # host memory; host->device and device->host copies of theta, omega and Delta inside the timed
     # call), on a bounded column sample so that all ranks together pin at most ~26 GB of host RAM
@@ -321,7 +346,7 @@ def run_gpu(args, w):
                            "local_step_ms": sum(pert_ms) / len(pert_ms),
                            "round_plus_local_step_ms": (sum(pert_ms) + sum(sync_ms)) / len(sync_ms),
                            "sync_ms_min": min(sync_ms), "sync_ms_max": max(sync_ms),
-                           "device_status": status},
+                           "sync_ms_in_cuda_graph": graph_ms, "device_status": status},
                 "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                              "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                              "frac_of_nominal_8TBs": achieved / 8000.0,
@@ -358,6 +383,8 @@ def main():
                     help="what moves the replicas between rounds (launched outside the timed interval)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-graph", action="store_true",
+                    help="skip the extra timing of the rounds replayed from one CUDA graph")
     ap.add_argument("--e2e-cols", type=int, default=1 << 27,
                     help="columns (summed over ranks) of the end-to-end host-buffer sample")
     ap.add_argument("--e2e-steps", type=int, default=3)

@@ -11,7 +11,7 @@
 //   sync_fused_tmem.cuh  sync_fused_tmem_kernel: the same with the theta tile in tensor memory and
 //                        bulk stores (the default in gossip-BMUF mode); device self-tests
 //   local_step.cuh       perturb_kernel (synthetic local steps), the Adagrad local step,
-//                        init_kernel (theta^k <- theta_0, omega^k <- theta_0, Delta^k <- 0),
+//                        init_stream_kernel (theta^k <- theta_0, omega^k <- theta_0, Delta^k <- 0),
 //                        final_average_kernel (theta = (1/K) sum_k theta^k)
 //   peer.cuh             one worker per GPU over peer-mapped buffers
 //
@@ -548,16 +548,28 @@ gbmuf_status gbmuf_init(gbmuf_ctx* ctx, const void* theta0, void* stream) {
     return fail(ctx, GBMUF_ERR_INVALID_ARG, "theta0 must be a 16-byte aligned device pointer");
   DeviceGuard guard(ctx->cfg.device);
   if (!guard.ok) return fail(ctx, GBMUF_ERR_CUDA, "cudaSetDevice failed");
-  const int grid = elementwise_grid(ctx, (ctx->cfg.N + 3) / 4);
   cudaStream_t st = (cudaStream_t)stream;
-  if (ctx->cfg.theta_dtype == GBMUF_F32)
-    init_kernel<float><<<grid, 256, 0, st>>>((const float*)theta0, (float*)ctx->theta, ctx->omega,
-                                             ctx->delta, ctx->cfg.K, ctx->cfg.N, ctx->cfg.ld);
-  else
-    init_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)theta0,
-                                                     (__nv_bfloat16*)ctx->theta, ctx->omega,
-                                                     ctx->delta, ctx->cfg.K, ctx->cfg.N, ctx->cfg.ld);
-  cudaError_t e = cudaGetLastError();
+  const long long nchunks = (ctx->cfg.N + kInitChunk - 1) / kInitChunk;
+  const int grid = (int)(nchunks < ctx->num_sms ? nchunks : ctx->num_sms);   // persistent CTAs
+  const int esz = (int)theta_size(ctx);
+  const size_t smem = 128 + (size_t)kInitChunk * 4 +
+                      (size_t)kInitSlots * ((size_t)kInitChunk * esz + (esz != 4 ? (size_t)kInitChunk * 4 : 0));
+  cudaError_t e;
+  if (ctx->cfg.theta_dtype == GBMUF_F32) {
+    e = cudaFuncSetAttribute(init_stream_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem);
+    if (e != cudaSuccess) return cuda_fail(ctx, "cudaFuncSetAttribute", e);
+    init_stream_kernel<float><<<grid, 128, smem, st>>>((const float*)theta0, (float*)ctx->theta, ctx->omega,
+                                                       ctx->delta, ctx->cfg.K, ctx->cfg.N, ctx->cfg.ld,
+                                                       ctx->d_status);
+  } else {
+    e = cudaFuncSetAttribute(init_stream_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem);
+    if (e != cudaSuccess) return cuda_fail(ctx, "cudaFuncSetAttribute", e);
+    init_stream_kernel<__nv_bfloat16><<<grid, 128, smem, st>>>((const __nv_bfloat16*)theta0,
+                                                               (__nv_bfloat16*)ctx->theta, ctx->omega,
+                                                               ctx->delta, ctx->cfg.K, ctx->cfg.N,
+                                                               ctx->cfg.ld, ctx->d_status);
+  }
+  e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, "launch of the init kernel", e);
   return GBMUF_OK;
 }

@@ -302,41 +302,93 @@ __global__ void __launch_bounds__(544, 1) adagrad_stream_kernel(const AdagradPar
 // =================================================================================================
 // Initialisation line of Algorithm 1 and its return line.
 // =================================================================================================
+// Initialisation as a copy-engine job: a chunk of theta_0 is fetched into shared memory once and
+// sent out 3K times -- to theta^k and omega^k of every worker, plus a block of zeros to Delta^k
+// -- by bulk stores; the threads only widen bf16 to fp32 for omega and handle the few elements
+// after the last whole 16-byte piece of theta_0.  4 + 12K bytes per parameter, all but 4 written.
+constexpr int kInitChunk = 4096;     // elements per chunk
+constexpr int kInitSlots = 3;        // chunks whose stores may be in flight
+
 template <typename TH>
-__global__ void __launch_bounds__(256) init_kernel(const TH* theta0, TH* theta, float* omega,
-                                                   float* delta, int K, long long N, long long ld) {
-  constexpr int VEC = ThetaTraits<TH>::VEC;
-  const long long nvec = (N + VEC - 1) / VEC;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec;
-       i += (long long)gridDim.x * blockDim.x) {
-    const long long e = i * VEC;
-    if (e + VEC <= N) {
-      const uint4 raw = *reinterpret_cast<const uint4*>(theta0 + e);   // 16 bytes of theta_0
-      float f[VEC];
-      ThetaTraits<TH>::lds(theta0 + e, f);
-      const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int k = 0; k < K; ++k) {
-        const long long at = (long long)k * ld + e;
-        __stcs(reinterpret_cast<uint4*>(theta + at), raw);
-#pragma unroll
-        for (int h = 0; h < VEC / 4; ++h) {
-          __stcs(reinterpret_cast<float4*>(omega + at) + h,
-                 make_float4(f[4 * h], f[4 * h + 1], f[4 * h + 2], f[4 * h + 3]));
-          __stcs(reinterpret_cast<float4*>(delta + at) + h, zero);
+__global__ void __launch_bounds__(128) init_stream_kernel(const TH* theta0, TH* theta, float* omega,
+                                                          float* delta, int K, long long N,
+                                                          long long ld, int32_t* status) {
+  constexpr int EB = (int)sizeof(TH);
+  constexpr int T = kInitChunk, R = kInitSlots;
+  constexpr bool WIDEN = EB != 4;                       // omega needs its own fp32 copy
+  constexpr uint32_t SLOT = (uint32_t)T * EB + (WIDEN ? (uint32_t)T * 4u : 0u);
+  extern __shared__ __align__(128) unsigned char smem[];
+  // [0, 64) barriers | [128, 128 + 4T) zeros | slots: [theta_0 chunk | (bf16) the chunk as fp32]
+  const uint32_t bars = smem_u32(smem);
+  float* zeros = reinterpret_cast<float*>(smem + 128);
+  unsigned char* slot0 = smem + 128 + (size_t)T * 4;
+  const long long nchunks = (N + T - 1) / T;
+  if (threadIdx.x == 0) {
+    for (int r = 0; r < R; ++r) mbar_init(bars + 8 * r, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  for (int i = threadIdx.x; i < T; i += blockDim.x) zeros[i] = 0.0f;
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  __syncthreads();
+
+  int it = 0;
+  for (long long ch = blockIdx.x; ch < nchunks; ch += gridDim.x, ++it) {
+    const int slot = it % R;
+    const long long e0 = ch * T;
+    const int n = (int)(N - e0 < T ? N - e0 : T);        // elements of this chunk
+    const int nw = n & ~(16 / EB - 1);                   // ... in whole 16-byte pieces of theta_0
+    unsigned char* sb = slot0 + (size_t)slot * SLOT;
+    if (threadIdx.x == 0) {
+      // the stores issued from this slot R chunks ago must have read it
+      if (it >= R) asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(R - 1) : "memory");
+      if (nw > 0) {
+        mbar_arrive_expect_tx(bars + 8 * slot, (uint32_t)nw * EB);
+        bulk_load_row(smem_u32(sb), theta0 + e0, (uint32_t)nw * EB, bars + 8 * slot);
+      } else {
+        mbar_arrive(bars + 8 * slot);
+      }
+    }
+    // (the slot is not touched by the other threads before the barrier below completes a phase
+    // that thread 0 arms only after the wait above)
+    const bool ok = mbar_wait_bounded(bars + 8 * slot, (it / R) & 1, status);
+    if (ok) {
+      if (WIDEN) {
+        const TH* st = reinterpret_cast<const TH*>(sb);
+        float* sw = reinterpret_cast<float*>(sb + (size_t)T * EB);
+        for (int i = threadIdx.x * 4; i < nw; i += blockDim.x * 4) {
+          float f[4];
+          ThetaTraits<TH>::lds_quad(st + i, f);
+          *reinterpret_cast<float4*>(sw + i) = make_float4(f[0], f[1], f[2], f[3]);
         }
       }
-    } else {
-      for (long long x = e; x < N; ++x) {
-        const TH v = theta0[x];
+      // the elements after the last whole piece: straight from theta_0 to every worker's rows
+      for (int i = nw + threadIdx.x; i < n; i += blockDim.x) {
+        const TH v = theta0[e0 + i];
         for (int k = 0; k < K; ++k) {
-          const long long at = (long long)k * ld + x;
+          const long long at = (long long)k * ld + e0 + i;
           theta[at] = v;
           omega[at] = ThetaTraits<TH>::widen(v);
           delta[at] = 0.0f;
         }
       }
     }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    if (__syncthreads_or(!ok)) break;                    // a wait expired: everybody leaves
+    if (threadIdx.x == 0) {
+      if (nw > 0) {
+        const uint32_t s_th = smem_u32(sb), s_om = WIDEN ? s_th + (uint32_t)T * EB : s_th;
+        const uint32_t s_ze = smem_u32(zeros);
+        for (int k = 0; k < K; ++k) {
+          const long long at = (long long)k * ld + e0;
+          asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(theta + at), "r"(s_th), "r"((uint32_t)nw * EB) : "memory");
+          asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(omega + at), "r"(s_om), "r"((uint32_t)nw * 4u) : "memory");
+          asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(delta + at), "r"(s_ze), "r"((uint32_t)nw * 4u) : "memory");
+        }
+      }
+      asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    }
   }
+  if (threadIdx.x == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
 
 template <typename TH>

@@ -330,16 +330,12 @@ sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_th
       mbar_arrive(bars + kBarThetaEmpty + 8 * s);
       continue;
     }
+    // gossip-BMUF: worker by worker, as the omega / Delta rows arrive in the ring
     for (int k = 0; k < P.K; ++k) {
-      const float* som = nullptr;
-      const float* sde = nullptr;
-      int slot = 0;
-      if (bmuf) {
-        slot = ring_taken % R;
-        if (!mbar_wait_bounded(bars + kBarRingFull + 8 * slot, (ring_taken / R) & 1, P.status)) return;
-        som = reinterpret_cast<const float*>(ring0 + (size_t)slot * P.slot_stride);
-        sde = som + P.T;
-      }
+      const int slot = ring_taken % R;
+      if (!mbar_wait_bounded(bars + kBarRingFull + 8 * slot, (ring_taken / R) & 1, P.status)) return;
+      const float* som = reinterpret_cast<const float*>(ring0 + (size_t)slot * P.slot_stride);
+      const float* sde = som + P.T;
       for (int v = c; v < nv; v += P.ncons) {
         const int col = v * VEC;
         const long long e = e0 + col;
@@ -357,22 +353,12 @@ sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_th
         }
         average_divide(a, P.qp1, P.inv_qp1, P.inv_exact);
         const long long at = (long long)k * P.ld + e;
-        const bool whole = e >= lo && e + VEC <= hi;
-        if (!bmuf) {                                       // gossip-MA: theta <- average
-          if (whole) {
-            ThetaTraits<TH>::stg_quad(theta + at, a);
-          } else {
-            for (int x = 0; x < VEC; ++x)
-              if (e + x >= lo && e + x < hi) theta[at + x] = ThetaTraits<TH>::narrow(a[x]);
-          }
-          continue;
-        }
         const float4 W = *reinterpret_cast<const float4*>(som + col);
         const float4 D = *reinterpret_cast<const float4*>(sde + col);
         float wv[VEC] = {W.x, W.y, W.z, W.w}, dv[VEC] = {D.x, D.y, D.z, D.w};
 #pragma unroll
         for (int x = 0; x < VEC; ++x) bmuf_filter<TH>(a[x], wv[x], dv[x], t[x], P.eta, P.zeta);
-        if (whole) {
+        if (e >= lo && e + VEC <= hi) {
           __stcs(reinterpret_cast<float4*>(P.delta + at), make_float4(dv[0], dv[1], dv[2], dv[3]));
           __stcs(reinterpret_cast<float4*>(P.omega + at), make_float4(wv[0], wv[1], wv[2], wv[3]));
           ThetaTraits<TH>::stg_quad(theta + at, t);
@@ -387,10 +373,8 @@ sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_th
           }
         }
       }
-      if (bmuf) {
-        mbar_arrive(bars + kBarRingEmpty + 8 * slot);    // this thread is done with the slot
-        ++ring_taken;
-      }
+      mbar_arrive(bars + kBarRingEmpty + 8 * slot);      // this thread is done with the slot
+      ++ring_taken;
     }
     mbar_arrive(bars + kBarThetaEmpty + 8 * s);          // this thread is done with the theta stage
   }
