@@ -171,7 +171,7 @@ gbmuf_status gbmuf_selftest_divide(gbmuf_ctx* ctx, int32_t divisor, void* stream
 
 /* Launch shape of the fused kernel (one persistent CTA per SM).  Any argument may be 0 to keep
  * the built-in choice.  Two variants exist.  (a) theta tile in tensor memory, outputs through bulk
- * stores: chosen automatically in gossip-BMUF mode with 4 <= K <= 128; tile_elems must then be a
+ * stores: chosen automatically in gossip-BMUF mode with K <= 128; tile_elems must then be a
  * multiple of 512 whose K rows fit the 512 columns of tensor memory (K * tile_elems / 128 <= 512
  * for fp32 theta, <= 1024 for bf16); ring_slots (2..8, at most three tiles' worth of rows) is the
  * number of shared-memory slots every row streams through.  (b) theta tile in shared memory: everything

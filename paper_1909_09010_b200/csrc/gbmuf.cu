@@ -170,16 +170,16 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
   const long long cap = ctx->max_smem < ctx->smem_per_sm - 1024 ? ctx->max_smem : ctx->smem_per_sm - 1024;
   // Variant: flags bit 3 forces the shared-memory theta tile, bit 1 forces the tensor-memory tile
   // (bit 2: with bulk stores); with neither, the tensor-memory tile with bulk stores is used
-  // wherever it applies (gossip-BMUF, 4 <= K <= 128) -- it is the faster one.
+  // wherever it applies (gossip-BMUF, K <= 128) -- it is the faster one.
   const int cw = esz == 4 ? 4 : 2;                       // TMEM columns per group of 4 elements
-  const bool tmem_ok = bmuf && K >= 4 && K <= 128;
+  const bool tmem_ok = bmuf && K <= 128;
   // (automatic choice only when the caller has not asked for anything specific to the
   // shared-memory tile: consumer threads, theta stages, or a tile width it cannot have)
   const bool auto_tmem = !(t.flags & 8) && tmem_ok && t.ncons == 0 && t.stages == 0 &&
                          (t.T == 0 || (t.T % 512 == 0 && (t.T / 512) * K * cw <= 512));
   const bool want_tmem = (t.flags & 2) || auto_tmem;
   if ((t.flags & 2) && !tmem_ok)
-    return fail(ctx, GBMUF_ERR_UNSUPPORTED, "the tensor-memory variant needs gossip-BMUF mode and 4 <= K <= 128");
+    return fail(ctx, GBMUF_ERR_UNSUPPORTED, "the tensor-memory variant needs gossip-BMUF mode and K <= 128");
   if (want_tmem) {
     const bool bulk = (t.flags & 2) ? (t.flags & 4) != 0 : true;
     const bool forced = (t.flags & 2) != 0;

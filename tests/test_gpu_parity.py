@@ -75,7 +75,7 @@ RAGGED = [
 def test_ragged_shapes(K, offsets, p, q, dtype):
     case = Case(K=K, offsets=offsets, p=p, q=q, eta=0.875, zeta=1.0, dtype=dtype, seed=K * 31 + q)
     run(case, random_theta0(case.N, seed=K, dtype=dtype), rounds=3, sigma=5e-2)
-    if dtype == 0 and 4 <= K <= 128:      # the default was the tensor-memory tile: also the shared-memory one
+    if K <= 128:                          # the default was the tensor-memory tile: also the shared-memory one
         run(case, random_theta0(case.N, seed=K, dtype=dtype), rounds=3, sigma=5e-2, tuning=dict(flags=8),
             check_nbr=False)
 
@@ -487,10 +487,10 @@ def test_averaging_division_equals_the_ieee_division_for_every_dividend():
 
 def test_tensor_memory_variant_is_refused_where_it_does_not_apply():
     dev = torch.device("cuda:0")
-    th = torch.zeros((2, 1024), device=dev)
-    g = binding.Gbmuf(th, th.clone(), th.clone(), K=2, N=1024, ld=1024, p=1, q=1, eta=0.9, zeta=1.0)
+    th = torch.zeros((130, 1024), device=dev)
+    g = binding.Gbmuf(th, th.clone(), th.clone(), K=130, N=1024, ld=1024, p=1, q=1, eta=0.9, zeta=1.0)
     with pytest.raises(binding.GbmufError) as e:
-        g.set_tuning(flags=2)                      # fewer than 4 workers
+        g.set_tuning(flags=2)                      # more workers than tensor memory has room for
     assert e.value.status == binding.ERR_UNSUPPORTED
     g.destroy()
     th = torch.zeros((8, 1024), device=dev)
