@@ -37,8 +37,8 @@ FALLBACK_HBM_GBS = 6650.0
 # dtype: 0 fp32 from workload profile16, 1 bf16 from profile16bf, both the tensor-memory
 # kernel), valid only
 # for the kernel source it was taken from (source_sha() below).
-NCU_TRAFFIC = {"source_sha": "e997b695ca4d", "bytes_per_replica_param": {0: 6.382833e9 / 268435536,
-                                                                   1: 5.309288e9 / 268435536}}
+NCU_TRAFFIC = {"source_sha": "872c2d58a077", "bytes_per_replica_param": {0: 6.383233e9 / 268435536,
+                                                                   1: 5.309554e9 / 268435536}}
 
 
 def algorithmic_bytes_per_replica_param(dtype: int, mode: int = 0) -> int:
