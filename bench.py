@@ -285,6 +285,20 @@ def run_gpu(args, w):
         del graph
         status = status or g.device_status()
 
+    # ---- a plain device copy of the same size class on this very GPU, as context for the
+    # roofline fraction (boxes of one pool differ by a percent or two); the state is no longer
+    # needed as a training state after this point
+    torch.cuda.synchronize()
+    ca, cb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    copy_ms = []
+    for _ in range(4):
+        ca.record()
+        delta.copy_(omega)
+        cb.record()
+        torch.cuda.synchronize()
+        copy_ms.append(ca.elapsed_time(cb))
+    copy_gbs_live = 2 * omega.numel() * 4 / (min(copy_ms[1:]) / 1e3) / 1e9
+
     # ---- end to end: the same round through the host-buffer entry point (replicas in page-locked
     # host memory; host->device and device->host copies of theta, omega and Delta inside the timed
     # call), on a bounded column sample so that all ranks together pin at most ~26 GB of host RAM
@@ -351,6 +365,7 @@ def run_gpu(args, w):
                              "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                              "frac_of_nominal_8TBs": achieved / 8000.0,
                              "algorithmic_bytes_per_replica_param": bpe, "traffic": traffic,
+                             "device_copy_gbs_on_this_gpu": copy_gbs_live,
                              "kernel": "sync_fused_tmem_kernel" if info.get("variant") == "tmem" else "sync_fused_kernel"},
                 "clocks": clocks,
                 "gpu_launches": (3 if args.local_step == "perturb" else 5) * args.steps, "e2e": e2e}
