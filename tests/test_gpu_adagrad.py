@@ -56,6 +56,54 @@ def test_adagrad_step_matches_oracle(dtype, K, offsets, mask):
     ctx.destroy()
 
 
+def test_adagrad_random_shapes_property():
+    """Random worker counts, row lengths (several chunks per CTA included), clip groups, theta type
+    and step sizes: accumulator and theta bit-equal with the oracle, padding untouched."""
+    import os
+    from hypothesis import given, settings, strategies as st_, HealthCheck
+
+    @settings(max_examples=int(os.environ.get("GBMUF_PROPERTY_EXAMPLES", "30")), deadline=None,
+              derandomize=True, suppress_health_check=list(HealthCheck))
+    @given(st_.data())
+    def inner(data):
+        dev = torch.device("cuda:0")
+        K = data.draw(st_.integers(1, 12))
+        m = data.draw(st_.integers(1, 7))
+        N = data.draw(st_.integers(m, data.draw(st_.sampled_from([5_000, 60_000, 700_000]))))
+        cuts = sorted(data.draw(st_.sets(st_.integers(1, N - 1), min_size=m - 1, max_size=m - 1))) if m > 1 else []
+        offsets = tuple([0] + cuts + [N])
+        dtype = data.draw(st_.integers(0, 1))
+        mask = data.draw(st_.one_of(st_.none(), st_.lists(st_.integers(0, 1), min_size=m, max_size=m)))
+        clip = data.draw(st_.sampled_from([10.0, 0.5, 0.0]))
+        gscale = data.draw(st_.sampled_from([3.0, 0.02, 1.0]))
+        lr = data.draw(st_.sampled_from([0.1, 0.081, 1e-3]))
+        ld = (N + 31) // 32 * 32
+        st = oracle.init(random_theta0(N, seed=K + N, dtype=dtype), K, ld=ld, dtype=dtype)
+        g = np.random.Generator(np.random.PCG64(N))
+        accum = np.zeros((K, ld), dtype=np.float32)
+        accum[:, :N] = 0.1
+        grad = np.zeros((K, ld), dtype=np.float32)
+        grad[:, :N] = (g.standard_normal((K, N)) * gscale).astype(np.float32)
+        theta = from_numpy(st.theta, dtype, dev)
+        om, de = torch.zeros((K, ld), device=dev), torch.zeros((K, ld), device=dev)
+        acc_dev, grad_dev = torch.from_numpy(accum.copy()).to(dev), torch.from_numpy(grad).to(dev)
+        ctx = binding.Gbmuf(theta, om, de, K=K, N=N, ld=ld, p=0, q=0, eta=0.9, zeta=1.0, theta_dtype=dtype)
+        try:
+            ctx.set_partition(offsets)
+            ranges = [(offsets[i], offsets[i + 1]) for i in range(m) if mask and mask[i]] if clip > 0 else []
+            for _ in range(2):
+                ctx.local_adagrad(grad_dev, acc_dev, lr, eps=1e-8, clip_norm=clip, clip_mask=mask)
+                oracle.local_adagrad(st, grad, accum, lr, eps=1e-8, clip_norm=clip, ranges=ranges)
+            torch.cuda.synchronize()
+            assert ctx.device_status() == 0
+            assert np.array_equal(acc_dev.cpu().numpy().view(np.uint32), accum.view(np.uint32))
+            assert np.array_equal(to_numpy(theta).view(np.uint8), st.theta.view(np.uint8))
+        finally:
+            ctx.destroy()
+
+    inner()
+
+
 def test_adagrad_then_sync_round_full_step():
     """Algorithm 1's loop body with the experiments' optimiser: local Adagrad step, then the
     gossip-BMUF round every second step, both sides replaying the same calls."""

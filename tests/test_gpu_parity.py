@@ -320,11 +320,13 @@ def test_rounds_replayed_from_a_cuda_graph():
 
 
 def test_random_shapes_property():
-    """Random K, p, q, component edges (unaligned, tiny and large), eta, zeta, dtype, mode."""
+    """Random K, p, q, component edges (unaligned, tiny and large), eta, zeta, dtype, mode, and
+    launch shapes of both variants of the fused kernel (several tiles per CTA included)."""
+    import os
     from hypothesis import given, settings, strategies as st_, HealthCheck
 
-    @settings(max_examples=25, deadline=None, derandomize=True,
-              suppress_health_check=list(HealthCheck))
+    @settings(max_examples=int(os.environ.get("GBMUF_PROPERTY_EXAMPLES", "100")), deadline=None,
+              derandomize=True, suppress_health_check=list(HealthCheck))
     @given(st_.data())
     def inner(data):
         K = data.draw(st_.integers(1, 24))
@@ -332,19 +334,27 @@ def test_random_shapes_property():
         c = min(2 * p, K - 1)
         q = data.draw(st_.integers(0, c))
         m = data.draw(st_.integers(1, 6))
-        N = data.draw(st_.integers(m, 30_000))
+        N = data.draw(st_.sampled_from([30_000, 30_000, 300_000]))
+        N = data.draw(st_.integers(m, N))
         cuts = sorted(data.draw(st_.sets(st_.integers(1, N - 1), min_size=m - 1, max_size=m - 1))) if m > 1 else []
         offsets = tuple([0] + cuts + [N])
         eta = data.draw(st_.sampled_from([0.0, 0.5, 0.875, 0.9, 0.99]))
         zeta = data.draw(st_.sampled_from([0.5, 1.0, 1.25]))
         dtype = data.draw(st_.integers(0, 1))
         mode = data.draw(st_.sampled_from([0, 0, 0, 1]))
-        tile = data.draw(st_.sampled_from([0, 64, 256, 512]))
-        force_smem = data.draw(st_.booleans())
         case = Case(K=K, offsets=offsets, p=p, q=q, eta=eta, zeta=zeta, dtype=dtype,
                     seed=data.draw(st_.integers(0, 2 ** 63)), mode=mode)
-        tuning = dict(tile_elems=tile, consumer_threads=data.draw(st_.sampled_from([64, 256]))) if tile else \
-            (dict(flags=8) if force_smem else None)
+        shape = data.draw(st_.sampled_from(["default", "shared", "shared_custom", "tensor_custom"]))
+        tuning = None
+        if shape == "shared":
+            tuning = dict(flags=8)
+        elif shape == "shared_custom":
+            tuning = dict(tile_elems=data.draw(st_.sampled_from([64, 256, 512])),
+                          consumer_threads=data.draw(st_.sampled_from([64, 256])))
+        elif shape == "tensor_custom" and mode == 0:
+            tuning = dict(tile_elems=data.draw(st_.sampled_from([512, 1024])),
+                          ring_slots=data.draw(st_.sampled_from([0, 2, 3, 4, 6])),
+                          flags=data.draw(st_.sampled_from([2, 6])))
         run(case, random_theta0(N, seed=K + N, dtype=dtype), rounds=2, sigma=5e-2, tuning=tuning)
 
     inner()
