@@ -21,9 +21,10 @@
  *   - Every function returns a gbmuf_status; nothing throws or aborts across this boundary.  On
  *     error no device work has been enqueued by that call and out-parameters are untouched;
  *     gbmuf_last_error() gives a sentence about the most recent failure on that context.
- *   - All arithmetic is fp32 with round-to-nearest-even on every single operation (no fused
- *     multiply-add, no flush-to-zero), in the order Algorithm 1 writes it; a bf16 theta is
- *     widened exactly on load and rounded to nearest-even on store.
+ *   - All arithmetic is fp32 with round-to-nearest-even on every single operation of Algorithm 1
+ *     (no contraction into fused multiply-adds, no flush-to-zero), in the order Algorithm 1 writes
+ *     it; the division by q+1 yields the correctly rounded quotient (see gbmuf_selftest_divide);
+ *     a bf16 theta is widened exactly on load and rounded to nearest-even on store.
  *   - There is no CPU path and no other back-end: without a CUDA device every compute call
  *     returns GBMUF_ERR_CUDA.
  */
