@@ -118,7 +118,6 @@ def source_sha() -> str:
 # ------------------------------------------------------------------------------------------------
 def oracle_sample(w, cols: int):
     """Oracle state over the first `cols` columns of the workload (a column range is exact)."""
-    import numpy as np
     import oracle
     from paper_1909_09010_b200 import workloads
     cols = min(cols, w.N)

@@ -3,7 +3,6 @@ every process.  PyTorch does the work (its CUDA-IPC tensor sharing and a torch.d
 for passing the handles around); nothing of the method is computed here."""
 from __future__ import annotations
 
-import torch
 import torch.distributed as dist
 from torch.multiprocessing.reductions import reduce_tensor
 

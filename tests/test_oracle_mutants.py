@@ -6,8 +6,6 @@ import subprocess
 import sys
 from concurrent.futures import ThreadPoolExecutor
 
-import pytest
-
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 PINS = ["tests/test_oracle_philox.py", "tests/test_oracle_sampler.py",
         "tests/test_oracle_perturb.py", "tests/test_oracle_adagrad.py", "tests/test_oracle_sync.py"]
