@@ -365,7 +365,7 @@ def run_gpu(args, w):
                              "frac_of_nominal_8TBs": achieved / 8000.0,
                              "algorithmic_bytes_per_replica_param": bpe, "traffic": traffic,
                              "device_copy_gbs_on_this_gpu": copy_gbs_live,
-                             "kernel": "sync_fused_tmem_kernel" if info.get("variant") == "tmem" else "sync_fused_kernel"},
+                             "kernel": "sync_fused_tmem_kernel" if str(info.get("variant")).startswith("tmem") else "sync_fused_kernel"},
                 "clocks": clocks,
                 "gpu_launches": (3 if args.local_step == "perturb" else 5) * args.steps, "e2e": e2e}
         if not args.no_cpu_baseline and world == 1:

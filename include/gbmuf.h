@@ -56,8 +56,7 @@ typedef enum { GBMUF_F32 = 0, GBMUF_BF16 = 1 } gbmuf_dtype;
 typedef enum { GBMUF_MODE_BMUF = 0, GBMUF_MODE_MA = 1 } gbmuf_mode;
 
 typedef struct {
-  int32_t K;           /* number of workers n (Definition 1), 1 <= K <= 256 (all K slices of a
-                          tile are staged together on one SM)                                     */
+  int32_t K;           /* number of workers n (Definition 1), 1 <= K <= 256                       */
   int64_t N;           /* parameters per replica, >= 1                                            */
   int64_t ld;          /* row stride in elements: >= N, multiple of 32                            */
   int32_t p;           /* symmetric degree of the ring (Definition 1), >= 0; the candidate set of
@@ -172,23 +171,29 @@ gbmuf_status gbmuf_selftest_divide(gbmuf_ctx* ctx, int32_t divisor, void* stream
 
 /* Launch shape of the fused kernel (one persistent CTA per SM).  Any argument may be 0 to keep
  * the built-in choice.  Two variants exist.  (a) theta tile in tensor memory, outputs through bulk
- * stores: chosen automatically in gossip-BMUF mode with K <= 128; tile_elems must then be a
- * multiple of 512 whose K rows fit the 512 columns of tensor memory (K * tile_elems / 128 <= 512
- * for fp32 theta, <= 1024 for bf16); ring_slots (2..8, at most three tiles' worth of rows) is the
- * number of shared-memory slots every row streams through.  (b) theta tile in shared memory: everything
- * else, and whenever consumer_threads or theta_stages is given or flags bit 3 is set;
- * consumer_threads: multiple of 32 in 32..992 (one more warp issues the copies); tile_elems: a
- * multiple of 8 and, above 256, of 256; theta_stages: 1..4; ring_slots: 2..8 rows of omega/Delta in
- * flight.  flags: bit 0 = 256-byte L2 promotion for the theta loads of (b); bit 1 = force (a),
- * bit 2 (with bit 1) = with bulk stores (without: stores from registers); bit 3 = force (b).
+ * stores: chosen automatically in gossip-BMUF mode when the resident rows of a tile fit the 512
+ * columns of tensor memory.  Resident rows r: all K workers' rows, or -- because worker k only ever
+ * averages with workers within ring distance p (Definition 1) -- a window of 2p + i rows that
+ * slides along the ring plus the first p rows kept for the last workers, r = 3p + i (i = 2 for
+ * fp32 theta, 4 for bf16); the window is possible when 2p + i < K and is taken when it allows a
+ * wider tile than K rows would (in practice from about 20 workers on).  tile_elems must be a
+ * multiple of 512 with r * tile_elems / 128 <= 512 for fp32 theta, <= 1024 for bf16; ring_slots
+ * (2..8, at most three tiles' worth of rows) is the number of shared-memory slots every row
+ * streams through.  (b) theta tile in shared memory: everything else, and whenever
+ * consumer_threads or theta_stages is given or flags bit 3 is set; consumer_threads: multiple of
+ * 32 in 32..992 (one more warp issues the copies); tile_elems: a multiple of 8 and, above 256, of
+ * 256; theta_stages: 1..4; ring_slots: 2..8 rows of omega/Delta in flight.  flags: bit 0 =
+ * 256-byte L2 promotion for the theta loads of (b); bit 1 = force (a), bit 2 (with bit 1) = with
+ * bulk stores (without: stores from registers); bit 3 = force (b); bit 4 = force the ring window
+ * of (a), bit 5 = never use it.  All choices give the same bits.
  * Errors: INVALID_ARG, UNSUPPORTED (does not fit, or (a) forced where it does not apply). */
 gbmuf_status gbmuf_set_tuning(gbmuf_ctx* ctx, int32_t consumer_threads, int32_t tile_elems,
                               int32_t theta_stages, int32_t ring_slots, int32_t flags);
 
 /* What the next full round would launch: tiles (work items), grid and block size, dynamic shared
  * memory in bytes, elements per tile, theta stages in shared memory (0 = the theta tile is kept in
- * tensor memory).  Any out pointer may be NULL.  Requires
- * set_partition. */
+ * tensor memory, all K rows; -r = in tensor memory as a ring window, r resident rows).  Any out
+ * pointer may be NULL.  Requires set_partition. */
 gbmuf_status gbmuf_get_launch_info(gbmuf_ctx* ctx, int64_t* tiles, int32_t* grid, int32_t* block,
                                    int32_t* smem_bytes, int32_t* tile_elems, int32_t* stages);
 

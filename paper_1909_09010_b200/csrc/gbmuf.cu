@@ -58,6 +58,9 @@ struct Launch {
   uint32_t stage_stride, nbr_off, desc_off, ring_off, slot_stride, smem;
   int tmem_cols;                     // TMEM variant: columns to allocate (0 = shared-memory tile)
   uint32_t meta_off, meta_stride;
+  // TMEM variant, which rows of a tile are resident: all K (win_rows = cell_rows = npos = K,
+  // lead = K, pshift = 0) or a window along the ring plus the kept first p rows
+  int win_rows, cell_rows, npos, lead, pshift;
 };
 
 int host_candidates(int K, int p) {
@@ -130,6 +133,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 // Tensor map for boxes of K rows x BW columns over the [K][ld] theta array.
 gbmuf_status build_tensor_maps(gbmuf_ctx* ctx, const Launch& L) {
+  if (L.tmem_cols > 0) return GBMUF_OK;      // the tensor-memory variant stages rows by 1-D copies
   static EncodeTiledFn encode = nullptr;
   if (!encode) {
     void* fn = nullptr;
@@ -167,41 +171,69 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
   Launch L;
   L.flags = t.flags;
   L.tmem_cols = 0; L.meta_off = 0; L.meta_stride = 0;
+  L.win_rows = 0; L.cell_rows = 0; L.npos = 0; L.lead = 0; L.pshift = 0;
   const long long cap = ctx->max_smem < ctx->smem_per_sm - 1024 ? ctx->max_smem : ctx->smem_per_sm - 1024;
   // Variant: flags bit 3 forces the shared-memory theta tile, bit 1 forces the tensor-memory tile
   // (bit 2: with bulk stores); with neither, the tensor-memory tile with bulk stores is used
-  // wherever it applies (gossip-BMUF, K <= 128) -- it is the faster one.
+  // wherever it applies (gossip-BMUF, resident rows that fit) -- it is the faster one.  Bit 4
+  // forces, bit 5 forbids the ring window of the tensor-memory tile.
   const int cw = esz == 4 ? 4 : 2;                       // TMEM columns per group of 4 elements
-  const bool tmem_ok = bmuf && K <= 128;
+  const int in_rows = 8 / esz;                           // theta rows per load item
+  // Rows resident in tensor memory: all K, or -- Definition 1's ring: a worker only averages with
+  // workers within distance p -- a window of 2p + in_rows rows that slides along the ring plus
+  // the first p rows kept for the last workers.  The window needs 2p + in_rows < K (then also
+  // 2p < K - 1 and signed ring distances are unambiguous).
+  const int p = ctx->cfg.p;
+  const int win_w = 2 * p + in_rows, win_cells = win_w + p;
+  const bool win_possible = win_w < K;
+  const int T_default = esz == 4 ? 3584 : 3072;          // measured best with 16 replicas
+  auto fits_cols = [&](int T, int rows) { return T >= 512 && T % 512 == 0 && (T / 512) * rows * cw <= 512; };
+  auto widest = [&](int rows) {                          // widest tile up to the default, 0 = none
+    int T = T_default;
+    while (T > 512 && !fits_cols(T, rows)) T -= 512;
+    return fits_cols(T, rows) ? T : 0;
+  };
+  if ((t.flags & 16) && (t.flags & 32))
+    return fail(ctx, GBMUF_ERR_INVALID_ARG, "flags bits 4 and 5 (force / forbid the ring window) exclude each other");
+  if ((t.flags & 16) && !(win_possible && bmuf))
+    return fail(ctx, GBMUF_ERR_UNSUPPORTED, "the ring window needs gossip-BMUF mode and 2p + rows per load item < K");
+  bool use_win = false;
+  if (win_possible && !(t.flags & 32)) {
+    if (t.flags & 16) use_win = true;
+    else if (t.T) use_win = !fits_cols(t.T, K) && fits_cols(t.T, win_cells);
+    else use_win = widest(win_cells) > widest(K);        // the window buys a wider tile
+  }
+  const int cells = use_win ? win_cells : K;
+  const bool tmem_ok = bmuf && widest(cells) > 0;
   // (automatic choice only when the caller has not asked for anything specific to the
   // shared-memory tile: consumer threads, theta stages, or a tile width it cannot have)
   const bool auto_tmem = !(t.flags & 8) && tmem_ok && t.ncons == 0 && t.stages == 0 &&
-                         (t.T == 0 || (t.T % 512 == 0 && (t.T / 512) * K * cw <= 512));
-  const bool want_tmem = (t.flags & 2) || auto_tmem;
-  if ((t.flags & 2) && !tmem_ok)
-    return fail(ctx, GBMUF_ERR_UNSUPPORTED, "the tensor-memory variant needs gossip-BMUF mode and K <= 128");
+                         (t.T == 0 || fits_cols(t.T, cells));
+  const bool want_tmem = (t.flags & (2 | 16)) || auto_tmem;
+  if ((t.flags & (2 | 16)) && !tmem_ok)
+    return fail(ctx, GBMUF_ERR_UNSUPPORTED, "the tensor-memory variant needs gossip-BMUF mode and resident rows that fit 512 columns (K <= 128, or a ring window)");
   if (want_tmem) {
+    const bool forced = (t.flags & (2 | 16)) != 0;
     const bool bulk = (t.flags & 2) ? (t.flags & 4) != 0 : true;
-    const bool forced = (t.flags & 2) != 0;
-    // theta tile in tensor memory: K * (T/512) * cw <= 512 columns; T a multiple of 512
+    // theta tile in tensor memory: cells * (T/512) * cw <= 512 columns; T a multiple of 512
     // default width: measured best with 16 replicas (fp32: 3584 x 4 slots; bf16: 3072 x 6 slots)
-    int T = t.T ? t.T : (esz == 4 ? 3584 : 3072);
-    while (!t.T && T > 512 && (T / 512) * K * cw > 512) T -= 512;
-    bool fits = T >= 512 && T % 512 == 0 && (T / 512) * K * cw <= 512;
+    const int T = t.T ? t.T : widest(cells);
+    const bool fits = fits_cols(T, cells);
     if (!fits && (forced || t.T))
-      return fail(ctx, GBMUF_ERR_INVALID_ARG, "tensor-memory variant: tile_elems must be a multiple of 512 whose K rows fit 512 columns of tensor memory");
+      return fail(ctx, GBMUF_ERR_INVALID_ARG, "tensor-memory variant: tile_elems must be a multiple of 512 whose resident rows fit 512 columns of tensor memory");
     if (fits) {
       L.T = T; L.BW = 256; L.stages = 1;
       L.ncons = 512;
-      L.flags = (t.flags & 1) | 2 | (bulk ? 4 : 0);
+      L.flags = (t.flags & 1) | 2 | (bulk ? 4 : 0) | (use_win ? 16 : 0);
+      L.win_rows = use_win ? win_w : K; L.cell_rows = cells;
+      L.npos = use_win ? K + p : K; L.lead = use_win ? 2 * p : K; L.pshift = use_win ? p : 0;
       L.meta_off = 512;
       L.meta_stride = (uint32_t)(((long long)sizeof(TileDesc) + (long long)K * q * 4 + 127) / 128 * 128);
       L.ring_off = L.meta_off + 4 * L.meta_stride;
       L.slot_stride = (uint32_t)((bulk ? 8 + esz : 8) * T);
       // ring items per tile; the 4-entry descriptor ring needs the producer to stay within three
       // tiles of the consumers, i.e. a ring no deeper than three tiles' worth of items
-      const int in_rows = 8 / esz;
-      const int per_tile = (K + in_rows - 1) / in_rows + K;
+      const int per_tile = (L.npos + in_rows - 1) / in_rows + K;
       const int ring_cap = 3 * per_tile < kMaxRing ? 3 * per_tile : kMaxRing;
       // Ring depth: 4 slots of the default width measured best (3 starve the pipeline, 5 and more
       // put too much in flight; even counts did better than odd ones); narrower slots: more of them.
@@ -217,7 +249,7 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
         L.ring = R;
         L.smem = (uint32_t)(L.ring_off + (long long)R * L.slot_stride);
         int cols = 32;
-        while (cols < (T / 512) * K * cw) cols <<= 1;
+        while (cols < (T / 512) * cells * cw) cols <<= 1;
         L.tmem_cols = cols;
         L.stage_stride = 0; L.nbr_off = 0; L.desc_off = 0;
         *out = L;
@@ -335,6 +367,7 @@ gbmuf_status launch_round(gbmuf_ctx* ctx, const gbmuf_config& cfg, const Launch&
     Q.ld = ld; Q.K = cfg.K; Q.m = m; Q.q = cfg.q;
     Q.eta = P.eta; Q.zeta = P.zeta; Q.qp1 = P.qp1; Q.inv_qp1 = P.inv_qp1; Q.inv_exact = P.inv_exact;
     Q.T = L.T; Q.ring = L.ring; Q.ncols = L.tmem_cols;
+    Q.W = L.win_rows; Q.wtot = L.cell_rows; Q.npos = L.npos; Q.lead = L.lead; Q.pshift = L.pshift;
     Q.ring_off = L.ring_off; Q.meta_off = L.meta_off; Q.meta_stride = L.meta_stride; Q.slot_stride = L.slot_stride;
     const bool bulk = (L.flags & 4) != 0, bf = cfg.theta_dtype != GBMUF_F32;
     void (*kern)(const TmemParams);
@@ -425,7 +458,7 @@ gbmuf_status gbmuf_create(const gbmuf_config* cfg, void* theta, float* omega, fl
   if (cand > kMaxCand)
     return fail(nullptr, GBMUF_ERR_UNSUPPORTED, "more than 64 ring neighbours per worker");
   if (cfg->K > 256)
-    return fail(nullptr, GBMUF_ERR_UNSUPPORTED, "more than 256 workers (one staged box holds all K rows)");
+    return fail(nullptr, GBMUF_ERR_UNSUPPORTED, "more than 256 workers");
   if (cfg->ld > 0x7fffffffLL)
     return fail(nullptr, GBMUF_ERR_UNSUPPORTED, "ld above 2^31 - 1 elements");
   if (!theta || !omega || !delta)
@@ -510,7 +543,7 @@ gbmuf_status gbmuf_set_tuning(gbmuf_ctx* ctx, int32_t ncons, int32_t tile_elems,
                               int32_t ring, int32_t flags) {
   if (!ctx) return GBMUF_ERR_INVALID_ARG;
   if (ncons < 0 || ncons > 992 || ncons % 32 != 0 || tile_elems < 0 || tile_elems > (1 << 16) ||
-      stages < 0 || stages > kMaxThetaStages || ring < 0 || ring > kMaxRing || ring == 1 || flags < 0 || flags > 15 || ((flags & 4) && !(flags & 2)) || ((flags & 8) && (flags & 2)))
+      stages < 0 || stages > kMaxThetaStages || ring < 0 || ring > kMaxRing || ring == 1 || flags < 0 || flags > 63 || ((flags & 4) && !(flags & 2)) || ((flags & 8) && (flags & (2 | 16))))
     return fail(ctx, GBMUF_ERR_INVALID_ARG, "tuning value out of range");
   Tuning t;
   t.ncons = ncons; t.T = tile_elems; t.stages = stages; t.ring = ring; t.flags = flags;
@@ -538,7 +571,9 @@ gbmuf_status gbmuf_get_launch_info(gbmuf_ctx* ctx, int64_t* tiles, int32_t* grid
   if (block) *block = 32 + ctx->launch.ncons;
   if (smem) *smem = (int32_t)ctx->launch.smem;
   if (tile_elems) *tile_elems = ctx->launch.T;
-  if (stages) *stages = ctx->launch.tmem_cols > 0 ? 0 : ctx->launch.stages;
+  if (stages)
+    *stages = ctx->launch.tmem_cols == 0 ? ctx->launch.stages
+              : ctx->launch.pshift > 0 || ctx->launch.cell_rows < ctx->cfg.K ? -ctx->launch.cell_rows : 0;
   return GBMUF_OK;
 }
 

@@ -23,9 +23,30 @@ namespace {
 // TMEM addressing: a warp reaches the 32 lanes 32 * (warp id % 4) ..; with the .32x32b.xN shape
 // each thread moves the N consecutive 32-bit columns of its lane that start at the given column.
 // Four consecutive elements of a row are one cell: 4 columns for fp32, 2 for bf16 (kept packed).
-// Element group g (4 elements) of a tile lives in lane g % 128, columns ((g / 128) * K + row) *
-// cell width.  The allocation is released by the warp that made it after every thread has
-// reached the end of the kernel; no path returns early.
+// Element group g (4 elements) of a tile lives in lane g % 128, columns ((g / 128) * W + cell row)
+// * cell width, W the number of rows held at once.  The allocation is released by the warp that
+// made it after every thread has reached the end of the kernel; no path returns early.
+//
+// Which rows are held.  Definition 1's ring means worker k only ever averages with workers within
+// ring distance p, so with many workers the K rows of a tile need not all be resident.  The rows
+// of a tile are requested in a sequence of `npos` positions and worker k's output item is issued
+// once position k + lead has been requested (or all have).
+//   all rows (W = K):     npos = K, position s is row s and lives in cell row s; every row is
+//                         requested before the first output item (lead >= K).
+//   ring window (W < K):  npos = K + p, position s is row (s - p) mod K, lead = 2p: worker k
+//                         needs exactly positions k .. k + 2p (its own row is position k + p).
+//                         Position s lives in cell row s mod W, W = 2p + rows per load item: a
+//                         load item requested while worker k is next overwrites positions below
+//                         k only.  Positions K + p .. K + 2p - 1 would be rows 0 .. p - 1 again,
+//                         which the first workers have overwritten in global memory by then (the
+//                         round is in place), so those rows are not requested a second time:
+//                         when they first arrive they are also put into p extra cell rows
+//                         W .. W + p - 1, where they stay for the last workers.  Cost: the last p
+//                         rows are read twice (p extra row reads per tile out of K) and W + p =
+//                         3p + rows-per-item cell rows instead of K, so the tile keeps its full
+//                         width however many workers there are.
+// Consumers take the items in the same order as the producer requests them, so "overwrites only
+// what no later worker needs" holds by program order; no extra synchronisation is involved.
 // =================================================================================================
 struct TmemParams {
   const void* theta_in;    // same array as theta (read side)
@@ -41,6 +62,8 @@ struct TmemParams {
   float eta, zeta, qp1, inv_qp1;
   int inv_exact;
   int T, ring, ncols;      // T multiple of 512; ring slots; TMEM columns (power of 2)
+  int W, wtot, npos, lead, pshift;   // window cell rows, all cell rows (W + kept rows),
+                                     // positions per tile, output lead, p (window) or 0
   uint32_t ring_off, meta_off, meta_stride;   // meta ring (4 entries): [TileDesc | nbr K*q ints]
   uint32_t slot_stride;    // bytes per ring slot
 };
@@ -89,12 +112,13 @@ template <> struct TmemCell<__nv_bfloat16> {
   }
 };
 
-// Sum of worker k's own cell and its q drawn neighbours' cells of element group `cell0` (the
-// TMEM address of row 0's cell), own first, then draw order, each addition rounded.
+// Sum of a worker's own cell (cell row `own`) and its q drawn neighbours' cells (cell rows nb[])
+// of element group `cell0` (the TMEM address of cell row 0), own first, then draw order, each
+// addition rounded.
 template <typename TH>
-__device__ __forceinline__ void tmem_gather(uint32_t cell0, int k, const int* nb, int q, float (&a)[4]) {
+__device__ __forceinline__ void tmem_gather(uint32_t cell0, int own, const int* nb, int q, float (&a)[4]) {
   constexpr int CW = TmemCell<TH>::COLS;
-  TmemCell<TH>::fetch(cell0 + (uint32_t)(k * CW), a);
+  TmemCell<TH>::fetch(cell0 + (uint32_t)(own * CW), a);
   for (int j = 0; j < q; ++j) {
     float t[4];
     TmemCell<TH>::fetch(cell0 + (uint32_t)(nb[j] * CW), t);
@@ -128,10 +152,11 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
   TH* const theta = reinterpret_cast<TH*>(P.theta);
   const TH* const theta_in = reinterpret_cast<const TH*>(P.theta_in);
   const int total = P.tile_prefix[P.m];
-  const int R = P.ring, K = P.K, q = P.q, T = P.T;
+  const int R = P.ring, K = P.K, q = P.q, T = P.T, W = P.W;
   const int my_tiles = (int)blockIdx.x < total ? (total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
-  const int ntheta = (K + IN_ROWS - 1) / IN_ROWS;                  // load items per tile
-  const int nout = K;                                              // output items per tile
+  // Items of a tile, in the order both sides generate them: with `s` positions requested and `k`
+  // workers put out, the next item is a load item (positions s .. s + IN_ROWS - 1) while
+  // s < npos and s <= k + lead, else worker k's output item.
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
@@ -214,8 +239,22 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
       TileDesc* d = reinterpret_cast<TileDesc*>(meta);
       int* snb = reinterpret_cast<int*>(meta + sizeof(TileDesc));
       if (d->comp != comp || it < 4) {
+        // the drawn neighbours as cell rows: the worker id itself when all rows are held, else
+        // the neighbour's position k + p + (signed ring distance), folded into the window or, past
+        // the last requested position, one of the kept first rows
         const int32_t* gnb = P.nbr + (size_t)comp * K * q;
-        for (int x = lane; x < K * q; x += 32) snb[x] = __ldg(gnb + x);
+        for (int x = lane; x < K * q; x += 32) {
+          int n = __ldg(gnb + x);
+          if (W < K) {
+            const int k = x / q;
+            int dist = n - k;
+            if (dist > P.pshift) dist -= K;
+            if (dist < -P.pshift) dist += K;
+            const int pos = k + P.pshift + dist;
+            n = pos < P.npos ? pos % W : W + (pos - P.npos);
+          }
+          snb[x] = n;
+        }
       }
       __syncwarp();
       if (lane == 0) {
@@ -225,7 +264,8 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
         d->comp = comp;
       }
       __syncwarp();
-      for (int item = 0; item < ntheta + nout && ok; ++item, ++gi) {
+      for (int s = 0, k = 0; k < K && ok; ++gi) {
+        const bool is_load = s < P.npos && s <= k + P.lead;
         const int slot = gi % R;
         if (BULK) {
           if (gi >= R - 1) ok = retire(gi - (R - 1));       // consumers done with it; its stores go out
@@ -246,25 +286,27 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
             si.e0 = e0;
             si.sb = (lo + ALN - 1) & ~(ALN - 1);
             si.se = hi & ~(ALN - 1);
-            si.k = item < ntheta ? -1 : item - ntheta;
+            si.k = is_load ? -1 : k;
             si.pad = 0;
             sinfo[slot] = si;
           }
-          if (item < ntheta) {
-            const int r0 = IN_ROWS * item;
-            const int rows = K - r0 < IN_ROWS ? K - r0 : IN_ROWS;
+          if (is_load) {
+            const int rows = P.npos - s < IN_ROWS ? P.npos - s : IN_ROWS;
             const uint32_t bytes = (uint32_t)run * EB;
             mbar_arrive_expect_tx(full, (uint32_t)rows * bytes);
-            for (int r = 0; r < rows; ++r)
-              bulk_load_row(dst + (uint32_t)r * (uint32_t)T * EB, theta_in + (long long)(r0 + r) * P.ld + e0, bytes, full);
+            for (int r = 0; r < rows; ++r) {
+              const int row = (s + r + K - P.pshift) % K;
+              bulk_load_row(dst + (uint32_t)r * (uint32_t)T * EB, theta_in + (long long)row * P.ld + e0, bytes, full);
+            }
           } else {
-            const long long at = (long long)(item - ntheta) * P.ld + e0;
+            const long long at = (long long)k * P.ld + e0;
             const uint32_t bytes = (uint32_t)run * 4u;
             mbar_arrive_expect_tx(full, 2u * bytes);
             bulk_load_row(dst, P.omega + at, bytes, full);
             bulk_load_row(dst + (uint32_t)T * 4u, P.delta + at, bytes, full);
           }
         }
+        if (is_load) s += IN_ROWS; else ++k;
       }
     }
     if (BULK) {
@@ -290,31 +332,43 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
       const TileDesc* d = reinterpret_cast<const TileDesc*>(meta);
       const int* snb = reinterpret_cast<const int*>(meta + sizeof(TileDesc));
       long long e0 = 0, lo = 0, hi = 0, sb = 0, se = 0;
-      for (int item = 0; item < ntheta + nout && ok; ++item, ++gi) {
+      bool first = true;
+      for (int s = 0, k = 0; k < K && ok; ++gi) {
+        const bool is_load = s < P.npos && s <= k + P.lead;
         const int slot = gi % R;
         bool fine = mbar_wait_bounded(bars + 8 * slot, (gi / R) & 1, P.status);
         ok = __all_sync(0xffffffffu, fine);
         if (!ok) break;
-        if (item == 0) {
+        if (first) {
+          first = false;
           e0 = d->e0; lo = d->lo; hi = d->hi;
           sb = (lo + ALN - 1) & ~(ALN - 1);       // whole 16-byte pieces of theta inside the tile
           se = hi & ~(ALN - 1);
         }
         unsigned char* const sbase = ring0 + (size_t)slot * P.slot_stride;
-        if (item < ntheta) {
+        if (is_load) {
           // deposit the theta rows of this item into this thread's TMEM cells
-          const int r0 = IN_ROWS * item;
           const TH* rows_in = reinterpret_cast<const TH*>(sbase);
+          int cell[IN_ROWS], keep[IN_ROWS];         // keep: cell row of a kept first row, or -1
+#pragma unroll
+          for (int r = 0; r < IN_ROWS; ++r) {
+            cell[r] = (s + r) % W;
+            const int row = s + r - P.pshift;
+            keep[r] = (W < K && row >= 0 && row < P.pshift) ? W + row : -1;
+          }
           for (int g = sub; g < ngroups; g += 4) {
             const int col = (g * 128 + quarter * 32 + lane) * 4;
 #pragma unroll
             for (int r = 0; r < IN_ROWS; ++r)
-              if (r0 + r < K)
-                TmemCell<TH>::deposit(tlane + (uint32_t)((g * K + r0 + r) * CW), rows_in + (size_t)r * T + col);
+              if (s + r < P.npos) {
+                TmemCell<TH>::deposit(tlane + (uint32_t)((g * P.wtot + cell[r]) * CW), rows_in + (size_t)r * T + col);
+                if (keep[r] >= 0)
+                  TmemCell<TH>::deposit(tlane + (uint32_t)((g * P.wtot + keep[r]) * CW), rows_in + (size_t)r * T + col);
+              }
           }
           asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         } else {
-          const int k = item - ntheta;
+          const int own = (k + P.pshift) % W;
           float* row0 = reinterpret_cast<float*>(sbase);
           float* row1 = row0 + T;
           TH* row2 = reinterpret_cast<TH*>(row1 + T);      // BULK: the new theta
@@ -323,12 +377,12 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
             const long long e = e0 + col;
             float a[4], t[4];
             __syncwarp();                          // lanes that left the last group early rejoin
-            tmem_gather<TH>(tlane + (uint32_t)(g * K * CW), k, snb + k * q, q, a);
+            tmem_gather<TH>(tlane + (uint32_t)(g * P.wtot * CW), own, snb + k * q, q, a);
             if (e >= hi || e + 4 <= lo) continue;
             average_divide(a, P.qp1, P.inv_qp1, P.inv_exact);
-            const float4 W = *reinterpret_cast<const float4*>(row0 + col);
-            const float4 D = *reinterpret_cast<const float4*>(row1 + col);
-            float wv[4] = {W.x, W.y, W.z, W.w}, dv[4] = {D.x, D.y, D.z, D.w};
+            const float4 Wv = *reinterpret_cast<const float4*>(row0 + col);
+            const float4 Dv = *reinterpret_cast<const float4*>(row1 + col);
+            float wv[4] = {Wv.x, Wv.y, Wv.z, Wv.w}, dv[4] = {Dv.x, Dv.y, Dv.z, Dv.w};
 #pragma unroll
             for (int x = 0; x < 4; ++x) bmuf_filter<TH>(a[x], wv[x], dv[x], t[x], P.eta, P.zeta);
             const long long at = (long long)k * P.ld + e;
@@ -351,8 +405,9 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
             }
           }
         }
-        if (BULK && item >= ntheta) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        if (BULK && !is_load) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         mbar_arrive(bars + 64 + 8 * slot);
+        if (is_load) s += IN_ROWS; else ++k;
       }
     }
   }

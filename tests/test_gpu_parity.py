@@ -478,6 +478,55 @@ def test_tensor_memory_variant(K, p, q, tile, ring, dtype, flags):
         tuning=dict(tile_elems=tile, ring_slots=ring, flags=flags), check_nbr=False)
 
 
+@pytest.mark.parametrize("flags", [16, 18])        # 18: window with stores from registers
+@pytest.mark.parametrize("dtype", [0, 1])
+@pytest.mark.parametrize("K,p,q,tile,ring", [(16, 3, 2, 0, 0), (9, 2, 4, 1024, 3), (12, 1, 2, 512, 8),
+                                              (24, 4, 8, 2048, 0), (64, 5, 7, 512, 4), (7, 1, 1, 512, 2),
+                                              (40, 0, 0, 1024, 4), (256, 7, 3, 512, 0), (23, 8, 16, 512, 0)])
+def test_ring_window_variant(K, p, q, tile, ring, dtype, flags):
+    """Tensor-memory tile that holds only a window of rows along the ring (plus the first p rows
+    kept for the last workers) gives the same bits as the oracle: wrap-around at both ends of the
+    worker range, several tiles per CTA, ragged component edges, masks, partly filled load items."""
+    if 2 * p + (2 if dtype == 0 else 4) >= K:
+        pytest.skip("no window for this shape: 2p + rows per load item must be below K")
+    offsets = (0, 100_003, 100_004, 350_001, 777_777) if K <= 64 else (0, 10_003, 10_004, 35_001, 77_777)
+    case = Case(K=K, offsets=offsets, p=p, q=q, eta=0.875, zeta=1.0, dtype=dtype, seed=K + q)
+    masks = [None, [1, 0, 1, 1], None]
+    run(case, random_theta0(case.N, seed=K, dtype=dtype), rounds=3, sigma=5e-2, masks=masks,
+        tuning=dict(tile_elems=tile, ring_slots=ring, flags=flags), check_nbr=False)
+
+
+@pytest.mark.parametrize("K,p,q,dtype,expect", [(64, 5, 7, 0, "tmem-window"), (128, 6, 3, 1, "tmem-window"),
+                                                  (256, 7, 2, 0, "tmem-window"), (16, 3, 2, 0, "tmem"),
+                                                  (32, 15, 30, 0, "tmem"), (200, 32, 64, 0, "tmem-window")])
+def test_which_rows_are_resident_follows_the_ring(K, p, q, dtype, expect):
+    """The window is taken by itself exactly when it buys a wider tile; flags bit 5 switches it
+    off; forcing it where the ring is too dense for a window is refused."""
+    dev = torch.device("cuda:0")
+    th = torch.zeros((K, 8192), device=dev, dtype=torch.float32 if dtype == 0 else torch.bfloat16)
+    om = torch.zeros((K, 8192), device=dev)
+    g = binding.Gbmuf(th, om, om.clone(), K=K, N=8192, ld=8192, p=p, q=q, eta=0.9, zeta=1.0, theta_dtype=dtype)
+    try:
+        g.set_partition([0, 8192])
+        info = g.launch_info()
+        assert info["variant"] == expect, info
+        rows_per_item = 2 if dtype == 0 else 4
+        if expect == "tmem-window":
+            assert -info["stages"] == 3 * p + rows_per_item
+            assert info["tile_elems"] >= (2560 if p <= 7 else 512)
+            g.set_tuning(flags=32)
+            assert g.launch_info()["variant"] in ("tmem", "smem")
+        elif 2 * p + rows_per_item >= K:
+            with pytest.raises(binding.GbmufError) as e:
+                g.set_tuning(flags=16)
+            assert e.value.status == binding.ERR_UNSUPPORTED
+        else:                                      # possible, but buys nothing at this K: only on request
+            g.set_tuning(flags=16)
+            assert g.launch_info()["variant"] == "tmem-window"
+    finally:
+        g.destroy()
+
+
 def test_averaging_division_equals_the_ieee_division_for_every_dividend():
     """The kernels divide the gossip sum by q+1 through a multiply and a residual correction;
     for every divisor they can meet (q+1 <= 65) and some beyond, all 2^32 dividends -- zeros,
@@ -500,7 +549,7 @@ def test_tensor_memory_variant_is_refused_where_it_does_not_apply():
     th = torch.zeros((130, 1024), device=dev)
     g = binding.Gbmuf(th, th.clone(), th.clone(), K=130, N=1024, ld=1024, p=1, q=1, eta=0.9, zeta=1.0)
     with pytest.raises(binding.GbmufError) as e:
-        g.set_tuning(flags=2)                      # more workers than tensor memory has room for
+        g.set_tuning(flags=2 | 32)                 # all rows resident: more workers than tensor memory has room for
     assert e.value.status == binding.ERR_UNSUPPORTED
     g.destroy()
     th = torch.zeros((8, 1024), device=dev)
