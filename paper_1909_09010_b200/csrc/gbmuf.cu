@@ -9,7 +9,8 @@
 //   sync_fused.cuh       sync_fused_kernel: gather + average + block-momentum filter, one pass, in
 //                        place, theta tile in shared memory (also gossip-MA)
 //   sync_fused_tmem.cuh  sync_fused_tmem_kernel: the same with the theta tile in tensor memory and
-//                        bulk stores (the default in gossip-BMUF mode); device self-tests
+//                        bulk stores (the default in gossip-BMUF mode); with many workers only a
+//                        window of rows along the ring is resident; device self-tests
 //   local_step.cuh       perturb_kernel (synthetic local steps), the Adagrad local step,
 //                        init_stream_kernel (theta^k <- theta_0, omega^k <- theta_0, Delta^k <- 0),
 //                        final_average_kernel (theta = (1/K) sum_k theta^k)
@@ -217,7 +218,18 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
     const bool bulk = (t.flags & 2) ? (t.flags & 4) != 0 : true;
     // theta tile in tensor memory: cells * (T/512) * cw <= 512 columns; T a multiple of 512
     // default width: measured best with 16 replicas (fp32: 3584 x 4 slots; bf16: 3072 x 6 slots)
-    const int T = t.T ? t.T : widest(cells);
+    // Window: widths whose element groups share out evenly over the consumer warps measured best
+    // (fp32, K = 64..256: 4096 x 4 slots, 3072 x 6, 2048 x 8 ahead of 3584 x 4 and 2560 x 6; bf16:
+    // 5120 x 4 and 4096 x 4 ahead of 3584 x 6 and 3072 x 6), the ring as deep as fits.
+    static const int kWinF32[][2] = {{4096, 4}, {3072, 6}, {2048, 8}, {1024, 8}, {512, 8}};
+    static const int kWinBf16[][2] = {{5120, 4}, {4096, 4}, {3584, 6}, {3072, 6}, {2048, 8}, {1024, 8}, {512, 8}};
+    int T = t.T ? t.T : widest(cells), ring_pref = 0;
+    if (use_win && !t.T && bulk) {
+      const int (*tab)[2] = esz == 4 ? kWinF32 : kWinBf16;
+      const int n = esz == 4 ? 5 : 7;
+      for (int i = 0; i < n; ++i)
+        if (fits_cols(tab[i][0], cells)) { T = tab[i][0]; ring_pref = tab[i][1]; break; }
+    }
     const bool fits = fits_cols(T, cells);
     if (!fits && (forced || t.T))
       return fail(ctx, GBMUF_ERR_INVALID_ARG, "tensor-memory variant: tile_elems must be a multiple of 512 whose resident rows fit 512 columns of tensor memory");
@@ -237,9 +249,9 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
       const int ring_cap = 3 * per_tile < kMaxRing ? 3 * per_tile : kMaxRing;
       // Ring depth: 4 slots of the default width measured best (3 starve the pipeline, 5 and more
       // put too much in flight; even counts did better than odd ones); narrower slots: more of them.
-      int R = t.ring ? t.ring : (bulk ? 4 : 3);
+      int R = t.ring ? t.ring : ring_pref ? ring_pref : (bulk ? 4 : 3);
       while (!t.ring && R > 2 && (long long)L.ring_off + (long long)R * L.slot_stride > cap) --R;
-      while (!t.ring && bulk && R + 2 <= ring_cap && (long long)R * L.slot_stride < 160 * 1024 &&
+      while (!t.ring && !ring_pref && bulk && R + 2 <= ring_cap && (long long)R * L.slot_stride < 160 * 1024 &&
              (long long)L.ring_off + (long long)(R + 2) * L.slot_stride <= cap) R += 2;
       if (!t.ring && R > ring_cap) R = ring_cap;
       const bool ring_fits = (long long)L.ring_off + (long long)R * L.slot_stride <= cap && R >= 2 && R <= ring_cap;
@@ -369,12 +381,14 @@ gbmuf_status launch_round(gbmuf_ctx* ctx, const gbmuf_config& cfg, const Launch&
     Q.T = L.T; Q.ring = L.ring; Q.ncols = L.tmem_cols;
     Q.W = L.win_rows; Q.wtot = L.cell_rows; Q.npos = L.npos; Q.lead = L.lead; Q.pshift = L.pshift;
     Q.ring_off = L.ring_off; Q.meta_off = L.meta_off; Q.meta_stride = L.meta_stride; Q.slot_stride = L.slot_stride;
-    const bool bulk = (L.flags & 4) != 0, bf = cfg.theta_dtype != GBMUF_F32;
+    const bool bulk = (L.flags & 4) != 0, bf = cfg.theta_dtype != GBMUF_F32, win = L.pshift > 0 || L.cell_rows < cfg.K;
     void (*kern)(const TmemParams);
     if (bf)
-      kern = bulk ? sync_fused_tmem_kernel<__nv_bfloat16, true> : sync_fused_tmem_kernel<__nv_bfloat16, false>;
+      kern = bulk ? (win ? sync_fused_tmem_kernel<__nv_bfloat16, true, true> : sync_fused_tmem_kernel<__nv_bfloat16, true, false>)
+                  : (win ? sync_fused_tmem_kernel<__nv_bfloat16, false, true> : sync_fused_tmem_kernel<__nv_bfloat16, false, false>);
     else
-      kern = bulk ? sync_fused_tmem_kernel<float, true> : sync_fused_tmem_kernel<float, false>;
+      kern = bulk ? (win ? sync_fused_tmem_kernel<float, true, true> : sync_fused_tmem_kernel<float, true, false>)
+                  : (win ? sync_fused_tmem_kernel<float, false, true> : sync_fused_tmem_kernel<float, false, false>);
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem);
     if (e != cudaSuccess) return cuda_fail(ctx, "cudaFuncSetAttribute", e);
     kern<<<grid, 544, L.smem, st>>>(Q);

@@ -135,7 +135,8 @@ struct SlotInfo { long long e0, sb, se; int k; int pad; };
 // [omega T floats | Delta T floats | (BULK) new theta T elements].
 // BULK: the outputs leave through bulk stores from the ring slot instead of st.global from
 // registers.
-template <typename TH, bool BULK>
+// WIN: ring window (else all K rows resident; the window's arithmetic then folds away).
+template <typename TH, bool BULK, bool WIN>
 __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParams P) {
   constexpr int EB = (int)sizeof(TH);
   constexpr int CW = TmemCell<TH>::COLS;
@@ -152,7 +153,8 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
   TH* const theta = reinterpret_cast<TH*>(P.theta);
   const TH* const theta_in = reinterpret_cast<const TH*>(P.theta_in);
   const int total = P.tile_prefix[P.m];
-  const int R = P.ring, K = P.K, q = P.q, T = P.T, W = P.W;
+  const int R = P.ring, K = P.K, q = P.q, T = P.T;
+  const int W = WIN ? P.W : K, wtot = WIN ? P.wtot : K, npos = WIN ? P.npos : K, pshift = WIN ? P.pshift : 0;
   const int my_tiles = (int)blockIdx.x < total ? (total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
   // Items of a tile, in the order both sides generate them: with `s` positions requested and `k`
   // workers put out, the next item is a load item (positions s .. s + IN_ROWS - 1) while
@@ -245,13 +247,13 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
         const int32_t* gnb = P.nbr + (size_t)comp * K * q;
         for (int x = lane; x < K * q; x += 32) {
           int n = __ldg(gnb + x);
-          if (W < K) {
+          if (WIN) {
             const int k = x / q;
             int dist = n - k;
-            if (dist > P.pshift) dist -= K;
-            if (dist < -P.pshift) dist += K;
-            const int pos = k + P.pshift + dist;
-            n = pos < P.npos ? pos % W : W + (pos - P.npos);
+            if (dist > pshift) dist -= K;
+            if (dist < -pshift) dist += K;
+            const int pos = k + pshift + dist;
+            n = pos < npos ? pos % W : W + (pos - npos);
           }
           snb[x] = n;
         }
@@ -265,7 +267,7 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
       }
       __syncwarp();
       for (int s = 0, k = 0; k < K && ok; ++gi) {
-        const bool is_load = s < P.npos && s <= k + P.lead;
+        const bool is_load = s < npos && (!WIN || s <= k + P.lead);
         const int slot = gi % R;
         if (BULK) {
           if (gi >= R - 1) ok = retire(gi - (R - 1));       // consumers done with it; its stores go out
@@ -291,11 +293,11 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
             sinfo[slot] = si;
           }
           if (is_load) {
-            const int rows = P.npos - s < IN_ROWS ? P.npos - s : IN_ROWS;
+            const int rows = npos - s < IN_ROWS ? npos - s : IN_ROWS;
             const uint32_t bytes = (uint32_t)run * EB;
             mbar_arrive_expect_tx(full, (uint32_t)rows * bytes);
             for (int r = 0; r < rows; ++r) {
-              const int row = (s + r + K - P.pshift) % K;
+              const int row = WIN ? (s + r + K - pshift) % K : s + r;
               bulk_load_row(dst + (uint32_t)r * (uint32_t)T * EB, theta_in + (long long)row * P.ld + e0, bytes, full);
             }
           } else {
@@ -334,7 +336,7 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
       long long e0 = 0, lo = 0, hi = 0, sb = 0, se = 0;
       bool first = true;
       for (int s = 0, k = 0; k < K && ok; ++gi) {
-        const bool is_load = s < P.npos && s <= k + P.lead;
+        const bool is_load = s < npos && (!WIN || s <= k + P.lead);
         const int slot = gi % R;
         bool fine = mbar_wait_bounded(bars + 8 * slot, (gi / R) & 1, P.status);
         ok = __all_sync(0xffffffffu, fine);
@@ -352,23 +354,23 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
           int cell[IN_ROWS], keep[IN_ROWS];         // keep: cell row of a kept first row, or -1
 #pragma unroll
           for (int r = 0; r < IN_ROWS; ++r) {
-            cell[r] = (s + r) % W;
-            const int row = s + r - P.pshift;
-            keep[r] = (W < K && row >= 0 && row < P.pshift) ? W + row : -1;
+            cell[r] = WIN ? (s + r) % W : s + r;
+            const int row = s + r - pshift;
+            keep[r] = (WIN && row >= 0 && row < pshift) ? W + row : -1;
           }
           for (int g = sub; g < ngroups; g += 4) {
             const int col = (g * 128 + quarter * 32 + lane) * 4;
 #pragma unroll
             for (int r = 0; r < IN_ROWS; ++r)
-              if (s + r < P.npos) {
-                TmemCell<TH>::deposit(tlane + (uint32_t)((g * P.wtot + cell[r]) * CW), rows_in + (size_t)r * T + col);
-                if (keep[r] >= 0)
-                  TmemCell<TH>::deposit(tlane + (uint32_t)((g * P.wtot + keep[r]) * CW), rows_in + (size_t)r * T + col);
+              if (s + r < npos) {
+                TmemCell<TH>::deposit(tlane + (uint32_t)((g * wtot + cell[r]) * CW), rows_in + (size_t)r * T + col);
+                if (WIN && keep[r] >= 0)
+                  TmemCell<TH>::deposit(tlane + (uint32_t)((g * wtot + keep[r]) * CW), rows_in + (size_t)r * T + col);
               }
           }
           asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         } else {
-          const int own = (k + P.pshift) % W;
+          const int own = WIN ? (k + pshift) % W : k;
           float* row0 = reinterpret_cast<float*>(sbase);
           float* row1 = row0 + T;
           TH* row2 = reinterpret_cast<TH*>(row1 + T);      // BULK: the new theta
@@ -377,7 +379,7 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
             const long long e = e0 + col;
             float a[4], t[4];
             __syncwarp();                          // lanes that left the last group early rejoin
-            tmem_gather<TH>(tlane + (uint32_t)(g * P.wtot * CW), own, snb + k * q, q, a);
+            tmem_gather<TH>(tlane + (uint32_t)(g * wtot * CW), own, snb + k * q, q, a);
             if (e >= hi || e + 4 <= lo) continue;
             average_divide(a, P.qp1, P.inv_qp1, P.inv_exact);
             const float4 Wv = *reinterpret_cast<const float4*>(row0 + col);

@@ -189,6 +189,13 @@ def get(name: str, **over) -> Workload:
         cuts = tuple(int(x) // 8 * 8 for x in np.linspace(0, n, 65)[:-1]) + (n,)
         w = Workload("profile16bf", K=16, vocab=0, hidden=0, layers=0, p=3, q=3, eta=0.9, zeta=1.0,
                      dtype=BF16, seed=4, rounds=4, local_steps=1, lr=0.1, sigma=1e-3, offsets=cuts)
+    elif name == "profile64":
+        # 64 workers on the ring the paper's rule gives them (p = log2(64) - 1 = 5), 2^22+5 columns
+        # (3.2 GB of state): the many-worker case profiler captures run on
+        n = (1 << 22) + 5
+        cuts = tuple(int(x) // 4 * 4 for x in np.linspace(0, n, 17)[:-1]) + (n,)
+        w = Workload("profile64", K=64, vocab=0, hidden=0, layers=0, p=5, q=2, eta=0.875, zeta=1.0,
+                     dtype=F32, seed=2, rounds=4, local_steps=1, lr=0.1, sigma=1e-3, offsets=cuts)
     else:
         raise KeyError(name)
     return replace(w, **over) if over else w

@@ -344,7 +344,7 @@ def test_random_shapes_property():
         mode = data.draw(st_.sampled_from([0, 0, 0, 1]))
         case = Case(K=K, offsets=offsets, p=p, q=q, eta=eta, zeta=zeta, dtype=dtype,
                     seed=data.draw(st_.integers(0, 2 ** 63)), mode=mode)
-        shape = data.draw(st_.sampled_from(["default", "shared", "shared_custom", "tensor_custom"]))
+        shape = data.draw(st_.sampled_from(["default", "shared", "shared_custom", "tensor_custom", "window"]))
         tuning = None
         if shape == "shared":
             tuning = dict(flags=8)
@@ -355,6 +355,10 @@ def test_random_shapes_property():
             tuning = dict(tile_elems=data.draw(st_.sampled_from([512, 1024])),
                           ring_slots=data.draw(st_.sampled_from([0, 2, 3, 4, 6])),
                           flags=data.draw(st_.sampled_from([2, 6])))
+        elif shape == "window" and mode == 0 and 2 * p + (2 if dtype == 0 else 4) < K:
+            tuning = dict(tile_elems=data.draw(st_.sampled_from([512, 1024])),
+                          ring_slots=data.draw(st_.sampled_from([0, 2, 3, 4, 6])),
+                          flags=data.draw(st_.sampled_from([16, 18, 22])))
         run(case, random_theta0(N, seed=K + N, dtype=dtype), rounds=2, sigma=5e-2, tuning=tuning)
 
     inner()
@@ -496,6 +500,16 @@ def test_ring_window_variant(K, p, q, tile, ring, dtype, flags):
         tuning=dict(tile_elems=tile, ring_slots=ring, flags=flags), check_nbr=False)
 
 
+@pytest.mark.parametrize("K,p,q,dtype", [(64, 5, 3, 0), (64, 5, 3, 1), (24, 3, 2, 0), (130, 6, 2, 1)])
+def test_ring_window_default_shape(K, p, q, dtype):
+    """The launch shape the library picks by itself for many workers (window, widest tile, deep
+    ring), with more tiles than CTAs so that every CTA goes round its ring several times."""
+    N = 148 * 4096 * 2 + 12_345 if K <= 64 else 148 * 5120 + 777
+    offsets = (0, N // 3 + 1, N // 3 + 2, N)
+    case = Case(K=K, offsets=offsets, p=p, q=q, eta=0.9, zeta=1.0, dtype=dtype, seed=K + p)
+    run(case, random_theta0(N, seed=K, dtype=dtype), rounds=2, sigma=5e-2, check_nbr=False)
+
+
 @pytest.mark.parametrize("K,p,q,dtype,expect", [(64, 5, 7, 0, "tmem-window"), (128, 6, 3, 1, "tmem-window"),
                                                   (256, 7, 2, 0, "tmem-window"), (16, 3, 2, 0, "tmem"),
                                                   (32, 15, 30, 0, "tmem"), (200, 32, 64, 0, "tmem-window")])
@@ -513,7 +527,7 @@ def test_which_rows_are_resident_follows_the_ring(K, p, q, dtype, expect):
         rows_per_item = 2 if dtype == 0 else 4
         if expect == "tmem-window":
             assert -info["stages"] == 3 * p + rows_per_item
-            assert info["tile_elems"] >= (2560 if p <= 7 else 512)
+            assert info["tile_elems"] >= (2048 if p <= 7 else 512)
             g.set_tuning(flags=32)
             assert g.launch_info()["variant"] in ("tmem", "smem")
         elif 2 * p + rows_per_item >= K:
