@@ -33,12 +33,16 @@ UNIT = "replica-params/s"
 FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of the fused kernel per replica-parameter from an ncu capture (dram__bytes_read.sum
-# + dram__bytes_write.sum divided by the replica-parameters of the captured launch; key = theta
-# dtype: 0 fp32 from workload profile16, 1 bf16 from profile16bf, both the tensor-memory
-# kernel), valid only
-# for the kernel source it was taken from (source_sha() below).
-NCU_TRAFFIC = {"source_sha": "872c2d58a077", "bytes_per_replica_param": {0: 6.383233e9 / 268435536,
-                                                                   1: 5.309554e9 / 268435536}}
+# + dram__bytes_write.sum divided by the replica-parameters of the captured launch), valid only
+# for the kernel source it was taken from (source_sha() below) and for the launch variant and
+# theta dtype it was taken with: key = (variant, dtype); 0 fp32 from workload profile16, 1 bf16
+# from profile16bf (all K rows in tensor memory); the ring-window figure is from profile64 and
+# holds for that ring only (K = 64, p = 5: p / K extra theta row reads).
+NCU_TRAFFIC = {"source_sha": "99b75b6ab307",
+               "bytes_per_replica_param": {("tmem", 0): 6.384655e9 / 268435536,
+                                           ("tmem", 1): 5.309743e9 / 268435536,
+                                           ("tmem-window", 0): 6.469851e9 / 268435776},
+               "window_ring": (64, 5)}
 
 
 def algorithmic_bytes_per_replica_param(dtype: int, mode: int = 0) -> int:
@@ -344,8 +348,11 @@ def run_gpu(args, w):
         t_launch = (sum(sync_ms) / len(sync_ms)) / 1e3
         achieved = bpe * K * N / t_launch / 1e9
         traffic = None
-        if NCU_TRAFFIC["source_sha"] == source_sha():
-            traffic = NCU_TRAFFIC["bytes_per_replica_param"][w.dtype] * K * N
+        per_param = NCU_TRAFFIC["bytes_per_replica_param"].get((info.get("variant"), w.dtype))
+        if info.get("variant") == "tmem-window" and (K, w.p) != NCU_TRAFFIC["window_ring"]:
+            per_param = None
+        if per_param is not None and not args.tuning and NCU_TRAFFIC["source_sha"] == source_sha():
+            traffic = per_param * K * N
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": total_sync_s / args.steps * 1e3,
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
