@@ -175,8 +175,10 @@ gbmuf_status gbmuf_selftest_divide(gbmuf_ctx* ctx, int32_t divisor, void* stream
  * columns of tensor memory.  Resident rows r: all K workers' rows, or -- because worker k only ever
  * averages with workers within ring distance p (Definition 1) -- a window of 2p + i rows that
  * slides along the ring plus the first p rows kept for the last workers, r = 3p + i (i = 2 for
- * fp32 theta, 4 for bf16); the window is possible when 2p + i < K and is taken when it allows a
- * wider tile than K rows would (in practice from about 20 workers on).  tile_elems must be a
+ * fp32 theta, 4 for bf16; the last p rows of a tile are then read twice), or r = 4p + i with the
+ * last p rows kept as well (every row read once; taken when it costs no tile width); the window
+ * is possible when 2p + i < K and is taken when it allows a wider tile than K rows would (in
+ * practice from about 20 workers on).  tile_elems must be a
  * multiple of 512 with r * tile_elems / 128 <= 512 for fp32 theta, <= 1024 for bf16; ring_slots
  * (2..8, at most three tiles' worth of rows) is the number of shared-memory slots every row
  * streams through.  (b) theta tile in shared memory: everything else, and whenever
@@ -185,7 +187,8 @@ gbmuf_status gbmuf_selftest_divide(gbmuf_ctx* ctx, int32_t divisor, void* stream
  * 256; theta_stages: 1..4; ring_slots: 2..8 rows of omega/Delta in flight.  flags: bit 0 =
  * 256-byte L2 promotion for the theta loads of (b); bit 1 = force (a), bit 2 (with bit 1) = with
  * bulk stores (without: stores from registers); bit 3 = force (b); bit 4 = force the ring window
- * of (a), bit 5 = never use it.  All choices give the same bits.
+ * of (a), bit 5 = never use it, bit 6 = window with every row read once.  All choices give the
+ * same bits.
  * Errors: INVALID_ARG, UNSUPPORTED (does not fit, or (a) forced where it does not apply). */
 gbmuf_status gbmuf_set_tuning(gbmuf_ctx* ctx, int32_t consumer_threads, int32_t tile_elems,
                               int32_t theta_stages, int32_t ring_slots, int32_t flags);

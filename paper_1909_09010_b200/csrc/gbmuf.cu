@@ -61,7 +61,7 @@ struct Launch {
   uint32_t meta_off, meta_stride;
   // TMEM variant, which rows of a tile are resident: all K (win_rows = cell_rows = npos = K,
   // lead = K, pshift = 0) or a window along the ring plus the kept first p rows
-  int win_rows, cell_rows, npos, lead, pshift;
+  int win_rows, cell_rows, npos, lead, pshift, keep_lo;
 };
 
 int host_candidates(int K, int p) {
@@ -172,7 +172,7 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
   Launch L;
   L.flags = t.flags;
   L.tmem_cols = 0; L.meta_off = 0; L.meta_stride = 0;
-  L.win_rows = 0; L.cell_rows = 0; L.npos = 0; L.lead = 0; L.pshift = 0;
+  L.win_rows = 0; L.cell_rows = 0; L.npos = 0; L.lead = 0; L.pshift = 0; L.keep_lo = 0;
   const long long cap = ctx->max_smem < ctx->smem_per_sm - 1024 ? ctx->max_smem : ctx->smem_per_sm - 1024;
   // Variant: flags bit 3 forces the shared-memory theta tile, bit 1 forces the tensor-memory tile
   // (bit 2: with bulk stores); with neither, the tensor-memory tile with bulk stores is used
@@ -185,7 +185,26 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
   // the first p rows kept for the last workers.  The window needs 2p + in_rows < K (then also
   // 2p < K - 1 and signed ring distances are unambiguous).
   const int p = ctx->cfg.p;
-  const int win_w = 2 * p + in_rows, win_cells = win_w + p;
+  // Window, kept rows: the first p rows always; the last p rows are either requested twice
+  // (3p + in_rows cell rows) or kept too (4p + in_rows cell rows, every row read once).  The
+  // second form is taken when it costs no tile width (or on request: flags bit 6).
+  const int win_w = 2 * p + in_rows, cells_twice = win_w + p, cells_once = win_w + 2 * p;
+  // widths whose element groups share out evenly over the consumer warps measured best for the
+  // window (fp32, K = 64..256: 4096 x 4 slots, 3072 x 6, 2048 x 8 ahead of 3584 x 4 and 2560 x 6;
+  // bf16: 5120 x 4 and 4096 x 4 ahead of 3584 x 6 and 3072 x 6), the ring as deep as fits
+  static const int kWinF32[][2] = {{4096, 4}, {3072, 6}, {2048, 8}, {1024, 8}, {512, 8}};
+  static const int kWinBf16[][2] = {{5120, 4}, {4096, 4}, {3584, 6}, {3072, 6}, {2048, 8}, {1024, 8}, {512, 8}};
+  auto window_shape = [&](int rows, int* ring) {         // widest listed tile for `rows` cell rows
+    const int (*tab)[2] = esz == 4 ? kWinF32 : kWinBf16;
+    const int n = esz == 4 ? 5 : 7;
+    for (int i = 0; i < n; ++i)
+      if ((tab[i][0] / 512) * rows * cw <= 512) { if (ring) *ring = tab[i][1]; return tab[i][0]; }
+    return 0;
+  };
+  const bool keep_both = (t.flags & 64) != 0 ||
+                         (!t.T && window_shape(cells_once, nullptr) >= window_shape(cells_twice, nullptr) &&
+                          window_shape(cells_once, nullptr) > 0);
+  const int win_cells = keep_both ? cells_once : cells_twice;
   const bool win_possible = win_w < K;
   const int T_default = esz == 4 ? 3584 : 3072;          // measured best with 16 replicas
   auto fits_cols = [&](int T, int rows) { return T >= 512 && T % 512 == 0 && (T / 512) * rows * cw <= 512; };
@@ -202,7 +221,7 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
   if (win_possible && !(t.flags & 32)) {
     if (t.flags & 16) use_win = true;
     else if (t.T) use_win = !fits_cols(t.T, K) && fits_cols(t.T, win_cells);
-    else use_win = widest(win_cells) > widest(K);        // the window buys a wider tile
+    else use_win = widest(cells_twice) > widest(K);      // the window buys a wider tile
   }
   const int cells = use_win ? win_cells : K;
   const bool tmem_ok = bmuf && widest(cells) > 0;
@@ -218,17 +237,10 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
     const bool bulk = (t.flags & 2) ? (t.flags & 4) != 0 : true;
     // theta tile in tensor memory: cells * (T/512) * cw <= 512 columns; T a multiple of 512
     // default width: measured best with 16 replicas (fp32: 3584 x 4 slots; bf16: 3072 x 6 slots)
-    // Window: widths whose element groups share out evenly over the consumer warps measured best
-    // (fp32, K = 64..256: 4096 x 4 slots, 3072 x 6, 2048 x 8 ahead of 3584 x 4 and 2560 x 6; bf16:
-    // 5120 x 4 and 4096 x 4 ahead of 3584 x 6 and 3072 x 6), the ring as deep as fits.
-    static const int kWinF32[][2] = {{4096, 4}, {3072, 6}, {2048, 8}, {1024, 8}, {512, 8}};
-    static const int kWinBf16[][2] = {{5120, 4}, {4096, 4}, {3584, 6}, {3072, 6}, {2048, 8}, {1024, 8}, {512, 8}};
     int T = t.T ? t.T : widest(cells), ring_pref = 0;
     if (use_win && !t.T && bulk) {
-      const int (*tab)[2] = esz == 4 ? kWinF32 : kWinBf16;
-      const int n = esz == 4 ? 5 : 7;
-      for (int i = 0; i < n; ++i)
-        if (fits_cols(tab[i][0], cells)) { T = tab[i][0]; ring_pref = tab[i][1]; break; }
+      const int Tw = window_shape(cells, &ring_pref);
+      if (Tw > 0) T = Tw; else ring_pref = 0;
     }
     const bool fits = fits_cols(T, cells);
     if (!fits && (forced || t.T))
@@ -238,7 +250,8 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
       L.ncons = 512;
       L.flags = (t.flags & 1) | 2 | (bulk ? 4 : 0) | (use_win ? 16 : 0);
       L.win_rows = use_win ? win_w : K; L.cell_rows = cells;
-      L.npos = use_win ? K + p : K; L.lead = use_win ? 2 * p : K; L.pshift = use_win ? p : 0;
+      L.npos = use_win && !keep_both ? K + p : K; L.lead = use_win ? 2 * p : K; L.pshift = use_win ? p : 0;
+      L.keep_lo = keep_both ? 0 : p;
       L.meta_off = 512;
       L.meta_stride = (uint32_t)(((long long)sizeof(TileDesc) + (long long)K * q * 4 + 127) / 128 * 128);
       L.ring_off = L.meta_off + 4 * L.meta_stride;
@@ -379,7 +392,7 @@ gbmuf_status launch_round(gbmuf_ctx* ctx, const gbmuf_config& cfg, const Launch&
     Q.ld = ld; Q.K = cfg.K; Q.m = m; Q.q = cfg.q;
     Q.eta = P.eta; Q.zeta = P.zeta; Q.qp1 = P.qp1; Q.inv_qp1 = P.inv_qp1; Q.inv_exact = P.inv_exact;
     Q.T = L.T; Q.ring = L.ring; Q.ncols = L.tmem_cols;
-    Q.W = L.win_rows; Q.wtot = L.cell_rows; Q.npos = L.npos; Q.lead = L.lead; Q.pshift = L.pshift;
+    Q.W = L.win_rows; Q.wtot = L.cell_rows; Q.npos = L.npos; Q.lead = L.lead; Q.pshift = L.pshift; Q.keep_lo = L.keep_lo;
     Q.ring_off = L.ring_off; Q.meta_off = L.meta_off; Q.meta_stride = L.meta_stride; Q.slot_stride = L.slot_stride;
     const bool bulk = (L.flags & 4) != 0, bf = cfg.theta_dtype != GBMUF_F32, win = L.pshift > 0 || L.cell_rows < cfg.K;
     void (*kern)(const TmemParams);
@@ -557,7 +570,7 @@ gbmuf_status gbmuf_set_tuning(gbmuf_ctx* ctx, int32_t ncons, int32_t tile_elems,
                               int32_t ring, int32_t flags) {
   if (!ctx) return GBMUF_ERR_INVALID_ARG;
   if (ncons < 0 || ncons > 992 || ncons % 32 != 0 || tile_elems < 0 || tile_elems > (1 << 16) ||
-      stages < 0 || stages > kMaxThetaStages || ring < 0 || ring > kMaxRing || ring == 1 || flags < 0 || flags > 63 || ((flags & 4) && !(flags & 2)) || ((flags & 8) && (flags & (2 | 16))))
+      stages < 0 || stages > kMaxThetaStages || ring < 0 || ring > kMaxRing || ring == 1 || flags < 0 || flags > 127 || ((flags & 4) && !(flags & 2)) || ((flags & 8) && (flags & (2 | 16))))
     return fail(ctx, GBMUF_ERR_INVALID_ARG, "tuning value out of range");
   Tuning t;
   t.ncons = ncons; t.T = tile_elems; t.stages = stages; t.ring = ring; t.flags = flags;

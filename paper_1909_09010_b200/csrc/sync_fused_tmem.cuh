@@ -33,18 +33,21 @@ namespace {
 // once position k + lead has been requested (or all have).
 //   all rows (W = K):     npos = K, position s is row s and lives in cell row s; every row is
 //                         requested before the first output item (lead >= K).
-//   ring window (W < K):  npos = K + p, position s is row (s - p) mod K, lead = 2p: worker k
-//                         needs exactly positions k .. k + 2p (its own row is position k + p).
-//                         Position s lives in cell row s mod W, W = 2p + rows per load item: a
-//                         load item requested while worker k is next overwrites positions below
-//                         k only.  Positions K + p .. K + 2p - 1 would be rows 0 .. p - 1 again,
-//                         which the first workers have overwritten in global memory by then (the
-//                         round is in place), so those rows are not requested a second time:
-//                         when they first arrive they are also put into p extra cell rows
-//                         W .. W + p - 1, where they stay for the last workers.  Cost: the last p
-//                         rows are read twice (p extra row reads per tile out of K) and W + p =
-//                         3p + rows-per-item cell rows instead of K, so the tile keeps its full
-//                         width however many workers there are.
+//   ring window (W < K):  position s is row (s - p) mod K, lead = 2p: worker k needs exactly
+//                         positions k .. k + 2p (its own row is position k + p).  Position s
+//                         lives in cell row s mod W, W = 2p + rows per load item: a load item
+//                         requested while worker k is next overwrites positions below k only.
+//                         The ring closes on itself, so the last workers need the first rows
+//                         again (positions K + p .. K + 2p - 1 = rows 0 .. p - 1), which the
+//                         first workers have overwritten in global memory by then (the round
+//                         is in place): those rows are put into p extra cell rows when they
+//                         first arrive and stay there.  The last p rows, which the first
+//                         workers need before everything else and the last workers own, are
+//                         either requested twice (npos = K + p, keep_lo = p, 3p + rows-per-item
+//                         cell rows, p extra row reads per tile out of K) or kept as well
+//                         (npos = K, keep_lo = 0, 4p + rows-per-item cell rows, every row read
+//                         once).  A position at or beyond npos is a kept row and lives in cell
+//                         row W + (position - npos).
 // Consumers take the items in the same order as the producer requests them, so "overwrites only
 // what no later worker needs" holds by program order; no extra synchronisation is involved.
 // =================================================================================================
@@ -64,6 +67,7 @@ struct TmemParams {
   int T, ring, ncols;      // T multiple of 512; ring slots; TMEM columns (power of 2)
   int W, wtot, npos, lead, pshift;   // window cell rows, all cell rows (W + kept rows),
                                      // positions per tile, output lead, p (window) or 0
+  int keep_lo;                       // window: positions keep_lo .. 2p - 1 are also kept
   uint32_t ring_off, meta_off, meta_stride;   // meta ring (4 entries): [TileDesc | nbr K*q ints]
   uint32_t slot_stride;    // bytes per ring slot
 };
@@ -355,8 +359,7 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
 #pragma unroll
           for (int r = 0; r < IN_ROWS; ++r) {
             cell[r] = WIN ? (s + r) % W : s + r;
-            const int row = s + r - pshift;
-            keep[r] = (WIN && row >= 0 && row < pshift) ? W + row : -1;
+            keep[r] = (WIN && s + r >= P.keep_lo && s + r < 2 * pshift) ? W + s + r - P.keep_lo : -1;
           }
           for (int g = sub; g < ngroups; g += 4) {
             const int col = (g * 128 + quarter * 32 + lane) * 4;
@@ -370,7 +373,7 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
           }
           asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         } else {
-          const int own = WIN ? (k + pshift) % W : k;
+          const int own = !WIN ? k : k + pshift < npos ? (k + pshift) % W : W + k + pshift - npos;
           float* row0 = reinterpret_cast<float*>(sbase);
           float* row1 = row0 + T;
           TH* row2 = reinterpret_cast<TH*>(row1 + T);      // BULK: the new theta
