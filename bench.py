@@ -143,7 +143,7 @@ def time_oracle_rounds(w, cols: int, rounds: int, first_round: int = 1):
         oracle.local_perturb(st, w.seed, r, w.lr or 0.1, w.sigma or 1e-3, 1, elem_base=0)
         t0 = time.perf_counter()
         nbr = oracle.sample_neighbors(w.seed, r, w.K, sh.m, w.p, w.q, comp_base=sh.comp_base)
-        oracle.sync_round(st, sh.offsets, nbr, w.eta, w.zeta)
+        oracle.sync_round(st, sh.offsets, nbr, w.eta, w.zeta, mode=w.mode)
         times.append(time.perf_counter() - t0)
     return times, w.K * sh.n
 
@@ -200,7 +200,7 @@ def run_gpu(args, w):
     delta = torch.empty((K, ld), dtype=torch.float32, device=dev)
     g = binding.Gbmuf(theta, omega, delta, K=K, N=N, ld=ld, p=w.p, q=w.q, eta=w.eta, zeta=w.zeta,
                       seed=w.seed, theta_dtype=w.dtype, device=local, comp_base=rank * w.m,
-                      elem_base=rank * N)
+                      elem_base=rank * N, mode=w.mode)
     if args.tuning:
         t = [int(x) for x in args.tuning.split(",")]
         g.set_tuning(*t)
@@ -318,7 +318,8 @@ def run_gpu(args, w):
         hde[:, :C].copy_(delta[:, :C])
         torch.cuda.synchronize()
         kw = dict(K=K, N=C, ld=cld, p=w.p, q=w.q, eta=w.eta, zeta=w.zeta, seed=w.seed,
-                  theta_dtype=w.dtype, device=local, comp_base=rank * w.m, elem_base=rank * N)
+                  theta_dtype=w.dtype, device=local, comp_base=rank * w.m, elem_base=rank * N,
+                  mode=w.mode)
         binding.sync_round_host(hth, hom, hde, sh.offsets, rnd, **kw)          # warm-up
         barrier()
         t0 = time.perf_counter()
@@ -342,7 +343,7 @@ def run_gpu(args, w):
         units = world * K * N * args.steps
         value = units / total_sync_s
         peak, peak_kind = measured_peak()
-        bpe = algorithmic_bytes_per_replica_param(w.dtype)
+        bpe = algorithmic_bytes_per_replica_param(w.dtype, w.mode)
         # per-launch figures of the fused kernel on this rank (the set-up kernel that shares the
         # event bracket runs for microseconds)
         t_launch = (sum(sync_ms) / len(sync_ms)) / 1e3
@@ -351,14 +352,15 @@ def run_gpu(args, w):
         per_param = NCU_TRAFFIC["bytes_per_replica_param"].get((info.get("variant"), w.dtype))
         if info.get("variant") == "tmem-window" and (K, w.p) != NCU_TRAFFIC["window_ring"]:
             per_param = None
-        if per_param is not None and not args.tuning and NCU_TRAFFIC["source_sha"] == source_sha():
+        if per_param is not None and not args.tuning and w.mode == 0 and NCU_TRAFFIC["source_sha"] == source_sha():
             traffic = per_param * K * N
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": total_sync_s / args.steps * 1e3,
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "f32" if w.dtype == 0 else "bf16-stored/f32", "data": "synthetic",
                 "config": {"workload": w.name, "K": K, "N": N, "components": w.m, "p": w.p, "q": w.q,
-                           "eta": w.eta, "zeta": w.zeta, "replica_params_per_gpu": K * N,
+                           "eta": w.eta, "zeta": w.zeta, "mode": "gossip-MA" if w.mode else "gossip-BMUF",
+                           "replica_params_per_gpu": K * N,
                            "parallelism": f"element-range shards x{world}, no collective",
                            "l2": "inputs_larger_than_l2 (state %.1f GB per GPU)" %
                                  ((K * ld * (8 + (4 if w.dtype == 0 else 2))) / 1e9),
@@ -411,7 +413,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     args = ap.parse_args()
     from paper_1909_09010_b200 import workloads
-    name, _, opts = args.workload.partition(":")           # e.g. sweep:C=64,q=4,eta=0.5
+    name, _, opts = args.workload.partition(":")           # e.g. sweep:C=64,q=4,eta=0.5 or wikitext103:mode=1
     over = {}
     for kv in filter(None, opts.split(",")):
         k, v = kv.split("=")

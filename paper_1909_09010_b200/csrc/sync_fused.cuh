@@ -77,11 +77,13 @@ struct SyncParams {
 //    division over all 2^32 bit patterns for a given divisor.
 // Costs 3 arithmetic instructions per element instead of about 10; gossip-MA with q+1 = 3 was
 // limited by the divide.
-// Exponent test: the result has one of its two top bits set iff the biased exponent of s is
-// outside [64, 191], i.e. unless 2^-63 <= |s| < 2^65; results of several values may be OR-ed.
-__device__ __forceinline__ uint32_t outside_mid_range(float s) {
-  return (__float_as_uint(s) & 0x7F800000u) - 0x20000000u;
+// Exponent test: bit 30 of the result is set iff the biased exponent of s is in [64, 191], i.e.
+// iff 2^-63 <= |s| < 2^65 (exponent bits 7 and 6 differ); results of several values may be AND-ed.
+__device__ __forceinline__ uint32_t mid_range_bit(float s) {
+  const uint32_t u = __float_as_uint(s);
+  return u ^ (u + u);
 }
+constexpr uint32_t kMidRange = 0x40000000u;
 __device__ __forceinline__ float divide_corrected(float s, float b, float y) {
   const float q0 = __fmul_rn(s, y);
   const float r = __fmaf_rn(-b, q0, s);
@@ -91,8 +93,7 @@ __device__ __forceinline__ void average_divide(float (&a)[4], float b, float y, 
   if (y_exact) {
 #pragma unroll
     for (int x = 0; x < 4; ++x) a[x] = __fmul_rn(a[x], y);
-  } else if (!((outside_mid_range(a[0]) | outside_mid_range(a[1]) | outside_mid_range(a[2]) |
-                outside_mid_range(a[3])) & 0xC0000000u)) {
+  } else if (mid_range_bit(a[0]) & mid_range_bit(a[1]) & mid_range_bit(a[2]) & mid_range_bit(a[3]) & kMidRange) {
 #pragma unroll
     for (int x = 0; x < 4; ++x) a[x] = divide_corrected(a[x], b, y);
   } else {
@@ -281,9 +282,13 @@ sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_th
       const int nvm = P.T / MV;
       const int kg = P.ncons > nvm ? P.ncons / nvm : 1;
       const int k_first = P.ncons > nvm ? c / nvm : 0;
-      auto ma_pass = [&](auto div_tag) -> bool {
+      // The neighbour count is a compile-time constant for q = 1 .. 4 (QC; 0 = any q at run
+      // time): the gather loop then unrolls completely, which halves the instructions per element.
+      auto ma_pass = [&](auto div_tag, auto q_tag) -> bool {
         constexpr int DIV = decltype(div_tag)::value;
-        uint32_t oor = 0;
+        constexpr int QC = decltype(q_tag)::value;
+        const int qn = QC ? QC : q;
+        uint32_t mid = 0xFFFFFFFFu;                 // bit 30 stays set while every sum is in the middle range
         for (int v = P.ncons > nvm ? c - k_first * nvm : c; v < nvm && k_first < kg; v += P.ncons) {
           const int col = v * MV;
           const long long e = e0 + col;
@@ -295,8 +300,9 @@ sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_th
           for (int k = k_first; k < P.K; k += kg) {
             float a[MV], t[MV];
             ThetaTraits<TH>::lds(sth + boxbase + k * BW, a);
-            for (int j = 0; j < q; ++j) {
-              ThetaTraits<TH>::lds(sth + boxbase + snb[k * q + j] * BW, t);
+#pragma unroll
+            for (int j = 0; j < qn; ++j) {
+              ThetaTraits<TH>::lds(sth + boxbase + snb[k * qn + j] * BW, t);
 #pragma unroll
               for (int x = 0; x < MV; ++x) a[x] = __fadd_rn(a[x], t[x]);
             }
@@ -305,7 +311,7 @@ sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_th
               if (DIV == 0) {
                 a[x] = __fmul_rn(a[x], P.inv_qp1);
               } else if (DIV == 1) {
-                oor |= outside_mid_range(a[x]);
+                mid &= mid_range_bit(a[x]);
                 a[x] = divide_corrected(a[x], P.qp1, P.inv_qp1);
               } else {
                 a[x] = __fdiv_rn(a[x], P.qp1);
@@ -320,12 +326,30 @@ sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_th
             }
           }
         }
-        return (oor & 0xC0000000u) != 0;
+        return (mid & kMidRange) == 0;
       };
-      if (P.inv_exact) {
-        ma_pass(std::integral_constant<int, 0>{});
-      } else if (ma_pass(std::integral_constant<int, 1>{})) {
-        ma_pass(std::integral_constant<int, 2>{});
+      auto ma_tile = [&](auto q_tag) {
+        constexpr int QC = decltype(q_tag)::value;
+        constexpr bool pow2 = QC == 1 || QC == 3;          // q + 1 a power of two: exact reciprocal
+        if (QC ? pow2 : P.inv_exact != 0) {
+          if constexpr (QC == 0 || pow2) ma_pass(std::integral_constant<int, 0>{}, q_tag);
+        } else {
+          if constexpr (!pow2)
+            if (ma_pass(std::integral_constant<int, 1>{}, q_tag)) ma_pass(std::integral_constant<int, 2>{}, q_tag);
+        }
+      };
+      // (bf16 theta only: its consumers are bound by instruction issue and gain 10 %; the fp32
+      // round is bound by memory and measured 2-3 % slower with the unrolled gather at q = 2)
+      if constexpr (sizeof(TH) == 2) {
+        switch (q) {
+          case 1: ma_tile(std::integral_constant<int, 1>{}); break;
+          case 2: ma_tile(std::integral_constant<int, 2>{}); break;
+          case 3: ma_tile(std::integral_constant<int, 3>{}); break;
+          case 4: ma_tile(std::integral_constant<int, 4>{}); break;
+          default: ma_tile(std::integral_constant<int, 0>{}); break;
+        }
+      } else {
+        ma_tile(std::integral_constant<int, 0>{});
       }
       mbar_arrive(bars + kBarThetaEmpty + 8 * s);
       continue;

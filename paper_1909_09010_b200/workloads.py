@@ -38,6 +38,7 @@ class Workload:
     offsets: tuple = field(repr=False, default=())
     drift_sigma: float = 0.0   # one-off per-replica drift added before the first round
     init_sigma: float = 0.1
+    mode: int = 0          # 0 gossip-BMUF, 1 gossip-MA (Algorithm 1's other branch)
 
     @property
     def N(self) -> int:
