@@ -38,10 +38,10 @@ FALLBACK_HBM_GBS = 6650.0
 # theta dtype it was taken with: key = (variant, dtype); 0 fp32 from workload profile16, 1 bf16
 # from profile16bf (all K rows in tensor memory); the ring-window figure is from profile64 and
 # holds for that ring only (K = 64, p = 5: p / K extra theta row reads).
-NCU_TRAFFIC = {"source_sha": "9e464fa3f81a",
-               "bytes_per_replica_param": {("tmem", 0): 6.383435e9 / 268435536,
-                                           ("tmem", 1): 5.309279e9 / 268435536,
-                                           ("tmem-window", 0): 6.469051e9 / 268435776},
+NCU_TRAFFIC = {"source_sha": "00d9b693dee9",
+               "bytes_per_replica_param": {("tmem", 0): 6.383437e9 / 268435536,
+                                           ("tmem", 1): 5.308850e9 / 268435536,
+                                           ("tmem-window", 0): 6.469350e9 / 268435776},
                "window_ring": (64, 5)}
 
 
