@@ -16,6 +16,7 @@ from __future__ import annotations
 
 import argparse
 import hashlib
+import re
 import json
 import os
 import statistics
@@ -38,7 +39,7 @@ FALLBACK_HBM_GBS = 6650.0
 # theta dtype it was taken with: key = (variant, dtype); 0 fp32 from workload profile16, 1 bf16
 # from profile16bf (all K rows in tensor memory); the ring-window figure is from profile64 and
 # holds for that ring only (K = 64, p = 5: p / K extra theta row reads).
-NCU_TRAFFIC = {"source_sha": "00d9b693dee9",
+NCU_TRAFFIC = {"source_sha": "0e09b2d1894a",
                "bytes_per_replica_param": {("tmem", 0): 6.383437e9 / 268435536,
                                            ("tmem", 1): 5.308850e9 / 268435536,
                                            ("tmem-window", 0): 6.469350e9 / 268435776},
@@ -107,13 +108,17 @@ class ClockSampler:
 
 
 def source_sha() -> str:
-    """Fingerprint of the fused kernels' source: the files that hold the barrier / bulk-copy
+    """Fingerprint of the fused kernels' code: the files that hold the barrier / bulk-copy
     primitives and theta traits, the shared-memory-tile kernel (with the averaging division and
-    the filter) and the tensor-memory-tile kernel."""
+    the filter) and the tensor-memory-tile kernel, with comments and white space left out (so that
+    rewording a comment does not invalidate the counters taken from the same code)."""
     h = hashlib.sha256()
     for name in ("primitives.cuh", "sync_fused.cuh", "sync_fused_tmem.cuh"):
-        with open(os.path.join(ROOT, "paper_1909_09010_b200", "csrc", name), "rb") as f:
-            h.update(f.read())
+        with open(os.path.join(ROOT, "paper_1909_09010_b200", "csrc", name), "r") as f:
+            text = f.read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        text = re.sub(r"//[^\n]*", "", text)
+        h.update("".join(text.split()).encode())
     return h.hexdigest()[:12]
 
 

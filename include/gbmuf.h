@@ -252,7 +252,7 @@ gbmuf_status gbmuf_sync_round_noalloc(const gbmuf_config* cfg, void* theta_devic
  * pointers to every other worker's two theta buffers, mapped into this process (CUDA IPC / peer
  * access; setting that up is the caller's business).  A round draws this worker's neighbours
  * exactly as gbmuf_sync_round does for worker `rank` (same seed, round, global component index),
- * and ONE kernel pulls their slices from peer memory (bulk copies without multicast), averages
+ * and ONE kernel pulls their slices from peer memory (single-destination bulk copies), averages
  * (own value first, then draw order), filters, writes omega and Delta in place and the new theta
  * into the worker's other buffer.  Components that do not take part are copied to the other
  * buffer unchanged, so after the round the other buffer is the worker's complete theta.

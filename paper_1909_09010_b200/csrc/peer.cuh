@@ -10,7 +10,7 @@ namespace {
 // write the other), omega and Delta; the other workers' theta buffers are peer-mapped pointers.
 // For every participating component the worker's q neighbours are drawn exactly as in the
 // resident form, and the fused kernel pulls their slices straight from peer memory with
-// non-multicast bulk copies into the same shared-memory stage as its own theta, omega and Delta
+// plain (single-destination) bulk copies into the same shared-memory stage as its own theta, omega and Delta
 // slices, averages (own first, then draw order), filters, and writes omega and Delta in place and
 // the new theta into the OTHER buffer: peers that are still reading this worker's current buffer
 // never see a half-updated replica.  Components that do not take part are copied through to the

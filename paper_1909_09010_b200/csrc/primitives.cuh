@@ -55,7 +55,7 @@ __device__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, int32_t* status
 }
 // Two-dimensional tiled TMA load: the box [rows 0..K) x [columns x, x + box width) of a row-major
 // [K][ld] array lands in shared memory as K consecutive rows of box-width elements.  One request
-// per box (no multicast); completion is counted in bytes on the mbarrier, out-of-range columns
+// per box, delivered to this CTA only; completion is counted in bytes on the mbarrier, out-of-range columns
 // are zero-filled and still counted.  x * element size must be a multiple of 16 bytes.
 __device__ __forceinline__ void tma_load_box(uint32_t dst_smem, const CUtensorMap* map, int x, int y,
                                              uint32_t bar) {
@@ -66,7 +66,7 @@ __device__ __forceinline__ void tma_load_box(uint32_t dst_smem, const CUtensorMa
       : "memory");
 }
 
-// One-dimensional bulk copy global -> shared through the copy engine (no multicast); completion
+// One-dimensional bulk copy global -> shared through the copy engine (to this CTA only); completion
 // is counted in bytes on the mbarrier.  Addresses and size are multiples of 16 bytes.
 __device__ __forceinline__ void bulk_load_row(uint32_t dst_smem, const void* src, uint32_t bytes,
                                               uint32_t bar) {

@@ -13,8 +13,9 @@ pytestmark = pytest.mark.gpu
 
 @pytest.mark.parametrize("dtype,chunk,pinned", [(0, 4096, True), (0, 1024, False), (1, 2048, True),
                                                 (0, 0, True)])
-def test_host_round_matches_oracle(dtype, chunk, pinned):
-    K, p, q, eta, zeta, seed = 8, 2, 2, 0.9, 1.0, 21
+@pytest.mark.parametrize("K,p,q", [(8, 2, 2), (40, 4, 3)])      # 40 workers: ring-window launch shape
+def test_host_round_matches_oracle(dtype, chunk, pinned, K, p, q):
+    eta, zeta, seed = 0.9, 1.0, 21
     offsets = (0, 1000, 1001, 4096, 9999, 20001, 50003)
     N = offsets[-1]
     ld = N + 13                                           # host arrays need no padding rule
