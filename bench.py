@@ -383,11 +383,11 @@ def run_gpu(args, w):
                 "clocks": clocks,
                 "gpu_launches": (3 if args.local_step == "perturb" else 5) * args.steps, "e2e": e2e}
         if not args.no_cpu_baseline and world == 1:
-            times, units_cpu = time_oracle_rounds(w, args.ref_cols, 3)
+            times, units_cpu = time_oracle_rounds(w, args.ref_cols, args.ref_rounds)
             t = sum(times) / len(times)
             line["cpu_baseline"] = {
                 "value": units_cpu / t, "unit": UNIT, "cores": 1, "kind": "oracle",
-                "sample": f"columns [0,{min(args.ref_cols, N)}) of {w.name}, K={K}, 3 rounds, "
+                "sample": f"columns [0,{min(args.ref_cols, N)}) of {w.name}, K={K}, {args.ref_rounds} rounds, "
                           f"{t:.2f} s per round"}
     g.destroy()
     if world > 1:
@@ -407,6 +407,8 @@ def main():
     ap.add_argument("--tuning", default="", help="consumer_threads,tile_elems,theta_stages,ring_slots,flags")
     ap.add_argument("--ref-cols", type=int, default=1 << 23,
                     help="columns of the workload the CPU oracle is timed on")
+    ap.add_argument("--ref-rounds", type=int, default=12,
+                    help="oracle rounds timed for the cpu_baseline entry (about 20 s of CPU work in all)")
     ap.add_argument("--local-step", default="perturb", choices=["perturb", "adagrad"],
                     help="what moves the replicas between rounds (launched outside the timed interval)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
