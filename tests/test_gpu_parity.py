@@ -493,7 +493,8 @@ def test_ring_window_variant(K, p, q, tile, ring, dtype, flags):
     worker range, several tiles per CTA, ragged component edges, masks, partly filled load items."""
     if 2 * p + (2 if dtype == 0 else 4) >= K:
         pytest.skip("no window for this shape: 2p + rows per load item must be below K")
-    offsets = (0, 100_003, 100_004, 350_001, 777_777) if K <= 64 else (0, 10_003, 10_004, 35_001, 77_777)
+    offsets = ((0, 100_003, 100_004, 350_001, 777_777) if K <= 16 else
+               (0, 40_003, 40_004, 140_001, 300_001) if K <= 64 else (0, 10_003, 10_004, 35_001, 77_777))
     case = Case(K=K, offsets=offsets, p=p, q=q, eta=0.875, zeta=1.0, dtype=dtype, seed=K + q)
     masks = [None, [1, 0, 1, 1], None]
     run(case, random_theta0(case.N, seed=K, dtype=dtype), rounds=3, sigma=5e-2, masks=masks,
