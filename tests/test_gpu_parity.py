@@ -572,4 +572,16 @@ def test_tensor_memory_variant_is_refused_where_it_does_not_apply():
                       mode=binding.MODE_MA)
     with pytest.raises(binding.GbmufError):
         g.set_tuning(flags=6)                      # gossip-MA
+    with pytest.raises(binding.GbmufError):
+        g.set_tuning(flags=16)                     # the ring window belongs to the tensor-memory tile
+    g.destroy()
+    th = torch.zeros((24, 1024), device=dev)
+    g = binding.Gbmuf(th, th.clone(), th.clone(), K=24, N=1024, ld=1024, p=3, q=2, eta=0.9, zeta=1.0)
+    for flags in (16 | 32, 8 | 16, 8 | 2, 4, 128):     # force and forbid at once; two variants at once; out of range
+        with pytest.raises(binding.GbmufError) as e:
+            g.set_tuning(flags=flags)
+        assert e.value.status == binding.ERR_INVALID_ARG, flags
+    g.set_tuning(flags=64)                         # "every row once" alone only shapes a window that is taken anyway
+    g.set_partition([0, 1024])
+    assert g.launch_info()["variant"] == "tmem-window"
     g.destroy()
