@@ -11,16 +11,32 @@
  * Conventions
  *   - "device" pointers are CUDA device memory of the context's GPU, owned by the CALLER (the
  *     library never frees or reallocates them); "host" pointers are ordinary host memory read or
- *     written before the call returns.
+ *     written before the call returns -- also when that memory is page-locked: small host tables
+ *     (masks, offsets) are copied into the library's own staging memory before their upload is
+ *     enqueued, so the caller may overwrite or free them as soon as the call is back.
  *   - theta, omega, delta are row-major [K][ld]: worker k's element e is at k*ld + e.  ld >= N,
  *     ld a multiple of 32, base pointers 128-byte aligned.  Columns N..ld-1 are padding: never
  *     written, contents irrelevant.  theta is fp32 or bf16 (theta_dtype); omega and delta are
  *     always fp32.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls that
  *     take a stream only enqueue work; they do not wait for it.
- *   - Every function returns a gbmuf_status; nothing throws or aborts across this boundary.  On
- *     error no device work has been enqueued by that call and out-parameters are untouched;
+ *   - Every function returns a gbmuf_status; nothing throws or aborts across this boundary.
+ *     Argument, state and size errors are found before any device work is enqueued, and
+ *     out-parameters are untouched on error.  Only if a kernel launch itself is refused by the
+ *     CUDA runtime (GBMUF_ERR_CUDA) may earlier steps of the same call (a table upload, the
+ *     set-up kernel) already be in the stream; no round kernel has run in that case.
  *     gbmuf_last_error() gives a sentence about the most recent failure on that context.
+ *   - Device-side waits are bounded (see gbmuf_selftest_wait_timeout).  A kernel whose wait
+ *     expired leaves early and records GBMUF_ERR_TIMEOUT in the context's status word; nothing
+ *     else reports it.  The buffers a round has written are therefore known to be good once
+ *     gbmuf_device_status has returned GBMUF_OK for the stream the round ran in; one check after
+ *     a sequence of rounds covers all of them (the word keeps the error until it is read).
+ *   - Stream capture: calls that only launch kernels (gbmuf_init, gbmuf_local_perturb,
+ *     gbmuf_local_adagrad without a new clip scratch, gbmuf_sync_round with comp_mask == NULL,
+ *     gbmuf_final_average) may be recorded into a capture.  Calls that upload host tables
+ *     (a comp_mask, gbmuf_sync_round_noalloc, gbmuf_set_partition) or wait for the device
+ *     (gbmuf_device_status, gbmuf_get_neighbors, the host-memory calls) may not; the first two
+ *     kinds return GBMUF_ERR_BAD_STATE inside a capture.
  *   - All arithmetic is fp32 with round-to-nearest-even on every single operation of Algorithm 1
  *     (no contraction into fused multiply-adds, no flush-to-zero), in the order Algorithm 1 writes
  *     it; the division by q+1 yields the correctly rounded quotient (see gbmuf_selftest_divide);
@@ -87,7 +103,8 @@ gbmuf_status gbmuf_create(const gbmuf_config* cfg, void* theta_device, float* om
  * elements offsets[i] .. offsets[i+1]-1.  offsets: host, m+1 entries, offsets[0] = 0, strictly
  * increasing, offsets[m] = N; no alignment is required of interior offsets.  periods: host, m
  * entries >= 1 (the synchronous period H_i of each component), or NULL for all 1.  May be called
- * again to re-partition; waits for the context's earlier work first.  1 <= m <= 65536.
+ * again to re-partition; it then waits for the work THIS context has enqueued (in whatever
+ * streams), not for the rest of the device.  1 <= m <= 65536.
  * Errors: INVALID_ARG, ALLOC, CUDA. */
 gbmuf_status gbmuf_set_partition(gbmuf_ctx* ctx, int32_t m, const int64_t* offsets_host,
                                  const int32_t* periods_host);
@@ -132,7 +149,8 @@ gbmuf_status gbmuf_local_adagrad(gbmuf_ctx* ctx, const float* grad_device, float
  * itself, rather than through gbmuf_init and earlier rounds, thereby defines R).  In MA mode
  * theta <- theta_bar only.
  * Everything happens in place in one pass; components not taking part are not touched.
- * Requires set_partition.  Errors: BAD_STATE, INVALID_ARG, CUDA. */
+ * Requires set_partition.  With a comp_mask the call may not be recorded into a stream capture
+ * (BAD_STATE).  Errors: BAD_STATE, INVALID_ARG, CUDA. */
 gbmuf_status gbmuf_sync_round(gbmuf_ctx* ctx, uint64_t round, const uint8_t* comp_mask_host,
                               void* stream);
 
@@ -200,16 +218,30 @@ gbmuf_status gbmuf_set_tuning(gbmuf_ctx* ctx, int32_t consumer_threads, int32_t 
 gbmuf_status gbmuf_get_launch_info(gbmuf_ctx* ctx, int64_t* tiles, int32_t* grid, int32_t* block,
                                    int32_t* smem_bytes, int32_t* tile_elems, int32_t* stages);
 
-/* One synchronisation round (as gbmuf_sync_round, same arithmetic and the same neighbour draws)
- * over replicas that live in HOST memory: theta, omega, delta are host arrays [K][ld] (ld >= N, no
- * alignment rule; page-locked memory lets the copies overlap, pageable memory works but
- * serialises them).  Given the neighbour table every element of the round is independent, so the
- * columns are cut into chunks of chunk_cols (a multiple of 32; 0 = 4,194,304) that rotate through
- * three sets of device buffers: copy in, set-up + fused kernel, copy out, each set on its own
- * stream.  Chunks in which no component takes part are not copied at all.  The call allocates
- * its device buffers (3 * K * chunk_cols * (element size + 8) bytes), returns when the host
- * arrays hold the result, and frees them.  comp_mask: host [m] or NULL (= all take part).
+/* Synchronisation rounds (as gbmuf_sync_round, same arithmetic and the same neighbour draws --
+ * Algorithm 1, the body of `if t mod H_i == 0`) over replicas that live in HOST memory: theta,
+ * omega, delta are host arrays [K][ld] (ld >= N, no alignment rule; page-locked memory lets the
+ * copies overlap, pageable memory works but serialises them).  Given the neighbour table every
+ * element of the round is independent, so the columns are cut into chunks of chunk_cols (a
+ * multiple of 32; 0 = 2,097,152) that rotate through three sets of device buffers: copy in,
+ * set-up + fused kernel, copy out, each set on its own stream.  Chunks in which no component
+ * takes part are not copied at all.
+ *   gbmuf_host_create allocates the device buffers (3 * K * chunk_cols * (element size + 8)
+ *   bytes; gossip-MA: 3 * K * chunk_cols * element size), the three streams and the chunk tables
+ *   once; cfg as for gbmuf_create (ld is the row stride of the HOST arrays), offsets host [m+1].
+ *   flags: bit 0 = move each array of a chunk by K row copies instead of one 2-D copy.
+ *   gbmuf_host_sync_round runs one round over the given host arrays (omega, delta may be NULL in
+ *   gossip-MA mode) and returns when they hold the result; it allocates nothing.  comp_mask: host
+ *   [m] or NULL (= all components take part).  Calls on one handle must not overlap.
+ *   gbmuf_host_destroy frees everything (NULL is accepted).
+ *   gbmuf_sync_round_host is create + one round + destroy in one call, for a single round.
  * Errors: INVALID_ARG, ALLOC, CUDA, TIMEOUT, UNSUPPORTED; text via gbmuf_last_error(NULL). */
+typedef struct gbmuf_host gbmuf_host;
+gbmuf_status gbmuf_host_create(const gbmuf_config* cfg, int32_t m, const int64_t* offsets_host,
+                               int64_t chunk_cols, int32_t flags, gbmuf_host** out);
+gbmuf_status gbmuf_host_sync_round(gbmuf_host* h, void* theta_host, float* omega_host,
+                                   float* delta_host, const uint8_t* comp_mask_host, uint64_t round);
+gbmuf_status gbmuf_host_destroy(gbmuf_host* h);
 gbmuf_status gbmuf_sync_round_host(const gbmuf_config* cfg, void* theta_host, float* omega_host,
                                    float* delta_host, int32_t m, const int64_t* offsets_host,
                                    const uint8_t* comp_mask_host, uint64_t round, int64_t chunk_cols);
@@ -232,13 +264,18 @@ gbmuf_status gbmuf_sync_round_host(const gbmuf_config* cfg, void* theta_host, fl
  *   gbmuf_sync_round; stream a cudaStream_t.  device_status_out: NULL, or a host int32 -- then the
  *   call waits for the stream and stores the device status word (GBMUF_OK or GBMUF_ERR_TIMEOUT).
  *   First use on a device: the first call on each GPU looks up the device address of the array
- *   (cudaGetSymbolAddress, with that GPU current) and sets the kernel's shared-memory limit; make
- *   that first call outside any stream capture.
+ *   (cudaGetSymbolAddress, with that GPU current) and raises the kernels' shared-memory limit.
+ *   Stream capture: every call uploads two small host tables (offsets, participation flags), so
+ *   this entry point is not meant to be recorded into a stream capture at all, first call or
+ *   later: inside a capture it returns GBMUF_ERR_BAD_STATE and enqueues nothing.  The tables
+ *   are copied into static staging memory of the library before the upload, so offsets and
+ *   comp_mask may be page-locked and may be overwritten as soon as the call returns.
  *   Sharing: all calls on a GPU use the same array.  It keeps the previous call's contents; this
  *   function clears the status word and rewrites every table it reads, so calls one after another
  *   on one stream are independent.  Calls that overlap on the GPU (different streams, or several
  *   host threads) race on the array and give undefined results: serialise them.
- * Errors: INVALID_ARG, UNSUPPORTED, CUDA; text via gbmuf_last_error(NULL) on the calling thread. */
+ * Errors: INVALID_ARG, UNSUPPORTED, BAD_STATE, CUDA; text via gbmuf_last_error(NULL) on the
+ * calling thread. */
 gbmuf_status gbmuf_sync_round_noalloc(const gbmuf_config* cfg, void* theta_device,
                                       float* omega_device, float* delta_device, int32_t m,
                                       const int64_t* offsets_host, const uint8_t* comp_mask_host,
@@ -278,7 +315,8 @@ gbmuf_status gbmuf_peer_destroy(gbmuf_peer* h);
  * With ctx == NULL: the last error of a failed gbmuf_create on this thread. */
 const char* gbmuf_last_error(const gbmuf_ctx* ctx);
 
-/* Waits for the context's work, frees the library's tables.  NULL is accepted. */
+/* Waits for the work this context has enqueued (not for the whole device), frees the library's
+ * tables.  NULL is accepted. */
 gbmuf_status gbmuf_destroy(gbmuf_ctx* ctx);
 
 #ifdef __cplusplus

@@ -23,7 +23,8 @@ MODE_BMUF, MODE_MA = 0, 1
 EXPORTS = ["gbmuf_create", "gbmuf_set_partition", "gbmuf_init", "gbmuf_local_perturb",
            "gbmuf_sync_round", "gbmuf_get_neighbors", "gbmuf_final_average", "gbmuf_device_status",
            "gbmuf_set_tuning", "gbmuf_get_launch_info", "gbmuf_last_error", "gbmuf_destroy",
-           "gbmuf_sync_round_noalloc", "gbmuf_sync_round_host", "gbmuf_local_adagrad",
+           "gbmuf_sync_round_noalloc", "gbmuf_sync_round_host", "gbmuf_host_create",
+           "gbmuf_host_sync_round", "gbmuf_host_destroy", "gbmuf_local_adagrad",
            "gbmuf_selftest_wait_timeout", "gbmuf_selftest_divide", "gbmuf_peer_create", "gbmuf_peer_set_partition",
            "gbmuf_peer_sync_round", "gbmuf_peer_device_status", "gbmuf_peer_destroy"]
 
@@ -74,6 +75,9 @@ def lib() -> ctypes.CDLL:
     L.gbmuf_sync_round_noalloc.argtypes = [ctypes.POINTER(Config), vp, vp, vp, i32, vp, vp, u64, vp,
                                            ctypes.POINTER(i32)]
     L.gbmuf_sync_round_host.argtypes = [ctypes.POINTER(Config), vp, vp, vp, i32, vp, vp, u64, i64]
+    L.gbmuf_host_create.argtypes = [ctypes.POINTER(Config), i32, vp, i64, i32, ctypes.POINTER(vp)]
+    L.gbmuf_host_sync_round.argtypes = [vp, vp, vp, vp, vp, u64]
+    L.gbmuf_host_destroy.argtypes = [vp]
     L.gbmuf_selftest_wait_timeout.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_double)]
     L.gbmuf_selftest_divide.argtypes = [vp, i32, vp, ctypes.POINTER(u64), ctypes.POINTER(ctypes.c_uint32)]
     L.gbmuf_peer_create.argtypes = [ctypes.POINTER(Config), i32, vp, vp, vp, ctypes.POINTER(vp)]
@@ -140,6 +144,41 @@ def sync_round_host(theta, omega, delta, offsets, rnd, *, K, N, ld, p, q, eta, z
                                      off.shape[0] - 1, _ptr(off), _ptr(mask), rnd, chunk_cols)
     if st != GBMUF_OK:
         raise GbmufError(st, lib().gbmuf_last_error(None).decode())
+
+
+class GbmufHost:
+    """``gbmuf_host_*``: rounds over HOST arrays [K][ld] with the device chunk buffers, streams and
+    chunk tables kept across rounds (``sync_round_host`` sets them up and frees them per call)."""
+
+    def __init__(self, offsets, *, K, N, ld, p, q, eta, zeta, seed=0, mode=MODE_BMUF, theta_dtype=F32,
+                 device=0, comp_base=0, elem_base=0, chunk_cols=0, row_copies=False):
+        self._h = ctypes.c_void_p()
+        cfg = Config(K, N, ld, p, q, eta, zeta, mode, theta_dtype, seed, device, comp_base, elem_base)
+        off = np.ascontiguousarray(offsets, dtype=np.int64)
+        self.m = off.shape[0] - 1
+        st = lib().gbmuf_host_create(ctypes.byref(cfg), self.m, _ptr(off), chunk_cols,
+                                     1 if row_copies else 0, ctypes.byref(self._h))
+        if st != GBMUF_OK:
+            raise GbmufError(st, lib().gbmuf_last_error(None).decode())
+
+    def sync_round(self, theta, omega, delta, rnd, comp_mask=None):
+        mask = None if comp_mask is None else np.ascontiguousarray(comp_mask, dtype=np.uint8)
+        if mask is not None and mask.shape[0] != self.m:
+            raise ValueError("comp_mask must have one entry per component")
+        st = lib().gbmuf_host_sync_round(self._h, _ptr(theta), _ptr(omega), _ptr(delta), _ptr(mask), rnd)
+        if st != GBMUF_OK:
+            raise GbmufError(st, lib().gbmuf_last_error(None).decode())
+
+    def destroy(self):
+        if self._h:
+            lib().gbmuf_host_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
 
 
 class GbmufPeer:
@@ -248,7 +287,18 @@ class Gbmuf:
         return out
 
     def final_average(self, out, stream=None):
+        """The returned model of Algorithm 1.  Also the point where a training run ends, so the
+        device status word is read here (this waits for the stream): a bounded device-side wait
+        that expired in any earlier round would otherwise go unnoticed."""
         self._check(lib().gbmuf_final_average(self._h, _ptr(out), _stream(stream)))
+        self.raise_on_device_error(stream)
+
+    def raise_on_device_error(self, stream=None):
+        """Reads (and clears) the device status word; raises if a kernel reported a failure."""
+        word = self.device_status(stream)
+        if word != GBMUF_OK:
+            raise GbmufError(word, "a device-side wait expired in an earlier call on this context; "
+                                   "theta, omega and Delta are unspecified")
 
     def device_status(self, stream=None) -> int:
         v = ctypes.c_int32(-1)
@@ -286,13 +336,24 @@ class Gbmuf:
     def last_error(self) -> str:
         return lib().gbmuf_last_error(self._h).decode()
 
-    def destroy(self):
+    def destroy(self, check_status=True):
+        """Frees the context.  Reads the device status word first (unless told not to) and raises
+        after freeing if an earlier round reported a failure nobody has looked at."""
         if self._h:
+            word = GBMUF_OK
+            if check_status:
+                try:
+                    word = self.device_status()
+                except Exception:
+                    word = GBMUF_OK
             st = lib().gbmuf_destroy(self._h)
             self._h = ctypes.c_void_p()
             self._keep = None
             if st != GBMUF_OK:
                 raise GbmufError(st, "destroy failed")
+            if word != GBMUF_OK:
+                raise GbmufError(word, "a device-side wait expired in an earlier call on this context "
+                                       "and was never read; its results were unspecified")
 
     def __del__(self):
         try:

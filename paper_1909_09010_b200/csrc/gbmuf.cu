@@ -28,6 +28,7 @@
 
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 #include <type_traits>
@@ -70,6 +71,52 @@ int host_candidates(int K, int p) {
   return (int)c;
 }
 
+// Is `st` recording a stream capture?  (The legacy default stream never is.)
+bool is_capturing(cudaStream_t st) {
+  if (!st) return false;
+  cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(st, &cs) != cudaSuccess) { cudaGetLastError(); return false; }
+  return cs != cudaStreamCaptureStatusNone;
+}
+
+// Which streams a handle has put work into, as one event per stream recorded after the latest
+// piece of work.  Re-partitioning and destruction wait for these events: for the handle's own
+// work and nothing else on the device.  Events outlive the streams they were recorded in, so a
+// stream the caller has destroyed in the meantime is no problem.  Work recorded into a stream
+// capture is not tracked (an event recorded there cannot be waited for from the host); the
+// caller keeps the handle alive while such a graph can still run.
+struct WorkMarks {
+  struct Mark { cudaStream_t s; cudaEvent_t ev; };
+  std::vector<Mark> marks;
+  static constexpr size_t kMaxStreams = 16;
+  void note(cudaStream_t st) {
+    if (is_capturing(st)) return;
+    for (Mark& mk : marks)
+      if (mk.s == st) { cudaEventRecord(mk.ev, st); return; }
+    if (marks.size() == kMaxStreams) {               // many streams: retire the oldest mark
+      cudaEventSynchronize(marks.front().ev);
+      cudaEventDestroy(marks.front().ev);
+      marks.erase(marks.begin());
+    }
+    Mark mk{st, nullptr};
+    if (cudaEventCreateWithFlags(&mk.ev, cudaEventDisableTiming) != cudaSuccess) { cudaGetLastError(); return; }
+    cudaEventRecord(mk.ev, st);
+    marks.push_back(mk);
+  }
+  cudaError_t wait() {
+    cudaError_t first = cudaSuccess;
+    for (Mark& mk : marks) {
+      const cudaError_t e = cudaEventSynchronize(mk.ev);
+      if (e != cudaSuccess && first == cudaSuccess) first = e;
+    }
+    return first;
+  }
+  void release() {
+    for (Mark& mk : marks) cudaEventDestroy(mk.ev);
+    marks.clear();
+  }
+};
+
 }  // namespace
 
 struct gbmuf_ctx {
@@ -98,6 +145,10 @@ struct gbmuf_ctx {
   Tuning tuning;
   Launch launch;
   CUtensorMap map_theta;   // boxes [K rows][launch.BW columns] over theta
+  std::vector<uint8_t> mask_stage;   // the library's own (pageable) copy of a caller's mask
+  int cap_m = 0;                     // sizes the device tables were allocated for
+  size_t cap_nbr_bytes = 0;
+  WorkMarks work;
   std::string err;
 };
 
@@ -126,6 +177,33 @@ gbmuf_status cuda_fail(gbmuf_ctx* ctx, const char* what, cudaError_t e) {
 }
 
 size_t theta_size(const gbmuf_ctx* c) { return c->cfg.theta_dtype == GBMUF_F32 ? 4 : 2; }
+
+// The streaming kernels use more dynamic shared memory than a kernel gets by default; the limit
+// is a per-device property of each kernel and is raised once per device (that device current),
+// when a handle is created, not on every launch.
+std::mutex g_attr_mutex;
+constexpr int kAttrDevices = 64;
+bool g_attr_done[kAttrDevices] = {};
+
+cudaError_t ensure_kernel_attributes(int device, int max_smem) {
+  std::lock_guard<std::mutex> lock(g_attr_mutex);
+  if (device >= 0 && device < kAttrDevices && g_attr_done[device]) return cudaSuccess;
+  const void* kernels[] = {
+      (const void*)sync_fused_tmem_kernel<float, true, true>, (const void*)sync_fused_tmem_kernel<float, true, false>,
+      (const void*)sync_fused_tmem_kernel<float, false, true>, (const void*)sync_fused_tmem_kernel<float, false, false>,
+      (const void*)sync_fused_tmem_kernel<__nv_bfloat16, true, true>, (const void*)sync_fused_tmem_kernel<__nv_bfloat16, true, false>,
+      (const void*)sync_fused_tmem_kernel<__nv_bfloat16, false, true>, (const void*)sync_fused_tmem_kernel<__nv_bfloat16, false, false>,
+      (const void*)sync_fused_kernel<float>, (const void*)sync_fused_kernel<__nv_bfloat16>,
+      (const void*)init_stream_kernel<float>, (const void*)init_stream_kernel<__nv_bfloat16>,
+      (const void*)adagrad_stream_kernel<float>, (const void*)adagrad_stream_kernel<__nv_bfloat16>,
+      (const void*)peer_round_kernel<float>, (const void*)peer_round_kernel<__nv_bfloat16>};
+  for (const void* k : kernels) {
+    const cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+    if (e != cudaSuccess) return e;
+  }
+  if (device >= 0 && device < kAttrDevices) g_attr_done[device] = true;
+  return cudaSuccess;
+}
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
                                   const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
@@ -376,7 +454,8 @@ void fill_sync_params(const gbmuf_config& cfg, const Launch& L, void* theta, flo
 }
 
 // Launches the fused round in the variant the launch shape names.  `ctx` supplies the error
-// slot, the device limits and (shared-memory variant) the tensor map of theta.
+// slot, the device limits and (shared-memory variant) the tensor map of theta.  The kernels'
+// shared-memory limit has been raised before (ensure_kernel_attributes).
 gbmuf_status launch_round(gbmuf_ctx* ctx, const gbmuf_config& cfg, const Launch& L, void* theta,
                           float* omega, float* delta, long long ld, int m, const int64_t* off,
                           const int32_t* prefix, const int32_t* nbr, int32_t* status,
@@ -402,16 +481,10 @@ gbmuf_status launch_round(gbmuf_ctx* ctx, const gbmuf_config& cfg, const Launch&
     else
       kern = bulk ? (win ? sync_fused_tmem_kernel<float, true, true> : sync_fused_tmem_kernel<float, true, false>)
                   : (win ? sync_fused_tmem_kernel<float, false, true> : sync_fused_tmem_kernel<float, false, false>);
-    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem);
-    if (e != cudaSuccess) return cuda_fail(ctx, "cudaFuncSetAttribute", e);
     kern<<<grid, 544, L.smem, st>>>(Q);
   } else if (cfg.theta_dtype == GBMUF_F32) {
-    e = cudaFuncSetAttribute(sync_fused_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem);
-    if (e != cudaSuccess) return cuda_fail(ctx, "cudaFuncSetAttribute", e);
     sync_fused_kernel<float><<<grid, 32 + L.ncons, L.smem, st>>>(P, ctx->map_theta);
   } else {
-    e = cudaFuncSetAttribute(sync_fused_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem);
-    if (e != cudaSuccess) return cuda_fail(ctx, "cudaFuncSetAttribute", e);
     sync_fused_kernel<__nv_bfloat16><<<grid, 32 + L.ncons, L.smem, st>>>(P, ctx->map_theta);
   }
   e = cudaGetLastError();
@@ -512,6 +585,8 @@ gbmuf_status gbmuf_create(const gbmuf_config* cfg, void* theta, float* omega, fl
   gbmuf_status st = plan_launch(ctx, ctx->tuning, &ctx->launch);
   if (st == GBMUF_OK) st = build_tensor_maps(ctx, ctx->launch);
   if (st != GBMUF_OK) { g_create_error = ctx->err; delete ctx; return st; }
+  e = ensure_kernel_attributes(cfg->device, ctx->max_smem);
+  if (e != cudaSuccess) { delete ctx; return cuda_fail(nullptr, "raising the kernels' shared-memory limit", e); }
   e = cudaMalloc(&ctx->d_status, sizeof(int32_t));
   if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(int32_t));
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->priv, cudaStreamNonBlocking);
@@ -541,25 +616,37 @@ gbmuf_status gbmuf_set_partition(gbmuf_ctx* ctx, int32_t m, const int64_t* offse
     return fail(ctx, GBMUF_ERR_INVALID_ARG, "comp_base + m overflows");
   DeviceGuard guard(ctx->cfg.device);
   if (!guard.ok) return fail(ctx, GBMUF_ERR_CUDA, "cudaSetDevice failed");
-  cudaError_t e = cudaDeviceSynchronize();
-  if (e != cudaSuccess) return cuda_fail(ctx, "cudaDeviceSynchronize", e);
-  free_tables(ctx);
+  // the tables are about to be replaced: wait for the work this context has enqueued (and only
+  // for that; other streams of the process keep running)
+  cudaError_t e = ctx->work.wait();
+  if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->priv);
+  if (e != cudaSuccess) return cuda_fail(ctx, "waiting for the context's earlier work", e);
   ctx->partitioned = false;
   ctx->m = m;
   ctx->off.assign(offsets, offsets + m + 1);
   if (periods) ctx->periods.assign(periods, periods + m); else ctx->periods.assign(m, 1);
   const size_t nb = (size_t)ctx->cfg.K * m * (ctx->cfg.q > 0 ? ctx->cfg.q : 1) * sizeof(int32_t);
-  e = cudaMalloc(&ctx->d_off, (m + 1) * sizeof(int64_t));
-  if (e == cudaSuccess) e = cudaMalloc(&ctx->d_periods, m * sizeof(int32_t));
-  if (e == cudaSuccess) e = cudaMalloc(&ctx->d_mask, m);
-  if (e == cudaSuccess) e = cudaMalloc(&ctx->d_prefix, (m + 1) * sizeof(int32_t));
-  if (e == cudaSuccess) e = cudaMalloc(&ctx->d_nbr, nb);
-  if (e == cudaSuccess) e = cudaMalloc(&ctx->d_nbr_export, nb);
-  if (e == cudaSuccess) e = cudaMemcpy(ctx->d_off, ctx->off.data(), (m + 1) * sizeof(int64_t), cudaMemcpyHostToDevice);
-  if (e == cudaSuccess) e = cudaMemcpy(ctx->d_periods, ctx->periods.data(), m * sizeof(int32_t), cudaMemcpyHostToDevice);
-  if (e == cudaSuccess) e = cudaMemset(ctx->d_mask, 1, m);
+  if (m > ctx->cap_m || nb > ctx->cap_nbr_bytes) {
+    // (tables that are already large enough are kept: freeing device memory stalls the device)
+    free_tables(ctx);
+    ctx->cap_m = 0; ctx->cap_nbr_bytes = 0;
+    e = cudaMalloc(&ctx->d_off, (m + 1) * sizeof(int64_t));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_periods, m * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_mask, m);
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_prefix, (m + 1) * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_nbr, nb);
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_nbr_export, nb);
+    if (e == cudaSuccess) { ctx->cap_m = m; ctx->cap_nbr_bytes = nb; }
+  }
+  // copies from the context's own vectors, complete when the private stream has been waited
+  // for: nothing of the caller's is read later, and a round on any stream finds the tables
+  if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->d_off, ctx->off.data(), (m + 1) * sizeof(int64_t), cudaMemcpyHostToDevice, ctx->priv);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->d_periods, ctx->periods.data(), m * sizeof(int32_t), cudaMemcpyHostToDevice, ctx->priv);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_mask, 1, m, ctx->priv);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->priv);
   if (e != cudaSuccess) {
     free_tables(ctx);
+    ctx->cap_m = 0; ctx->cap_nbr_bytes = 0;
     return e == cudaErrorMemoryAllocation ? fail(ctx, GBMUF_ERR_ALLOC, "partition tables") : cuda_fail(ctx, "partition upload", e);
   }
   ctx->partitioned = true;
@@ -618,14 +705,10 @@ gbmuf_status gbmuf_init(gbmuf_ctx* ctx, const void* theta0, void* stream) {
                       (size_t)kInitSlots * ((size_t)kInitChunk * esz + (esz != 4 ? (size_t)kInitChunk * 4 : 0));
   cudaError_t e;
   if (ctx->cfg.theta_dtype == GBMUF_F32) {
-    e = cudaFuncSetAttribute(init_stream_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem);
-    if (e != cudaSuccess) return cuda_fail(ctx, "cudaFuncSetAttribute", e);
     init_stream_kernel<float><<<grid, 128, smem, st>>>((const float*)theta0, (float*)ctx->theta, ctx->omega,
                                                        ctx->delta, ctx->cfg.K, ctx->cfg.N, ctx->cfg.ld,
                                                        ctx->d_status);
   } else {
-    e = cudaFuncSetAttribute(init_stream_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem);
-    if (e != cudaSuccess) return cuda_fail(ctx, "cudaFuncSetAttribute", e);
     init_stream_kernel<__nv_bfloat16><<<grid, 128, smem, st>>>((const __nv_bfloat16*)theta0,
                                                                (__nv_bfloat16*)ctx->theta, ctx->omega,
                                                                ctx->delta, ctx->cfg.K, ctx->cfg.N,
@@ -633,6 +716,7 @@ gbmuf_status gbmuf_init(gbmuf_ctx* ctx, const void* theta0, void* stream) {
   }
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, "launch of the init kernel", e);
+  ctx->work.note(st);
   return GBMUF_OK;
 }
 
@@ -661,6 +745,7 @@ gbmuf_status gbmuf_local_perturb(gbmuf_ctx* ctx, uint64_t step, float lr, float 
   }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, "launch of the local-step kernel", e);
+  ctx->work.note(st);
   return GBMUF_OK;
 }
 
@@ -718,16 +803,13 @@ gbmuf_status gbmuf_local_adagrad(gbmuf_ctx* ctx, const float* grad, float* accum
   const long long chunks = cpr * K;
   const int grid = (int)(chunks < ctx->num_sms ? chunks : ctx->num_sms);
   if (ctx->cfg.theta_dtype == GBMUF_F32) {
-    e = cudaFuncSetAttribute(adagrad_stream_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem);
-    if (e != cudaSuccess) return cuda_fail(ctx, "cudaFuncSetAttribute", e);
     adagrad_stream_kernel<float><<<grid, 544, smem_bytes, st>>>(A);
   } else {
-    e = cudaFuncSetAttribute(adagrad_stream_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem);
-    if (e != cudaSuccess) return cuda_fail(ctx, "cudaFuncSetAttribute", e);
     adagrad_stream_kernel<__nv_bfloat16><<<grid, 544, smem_bytes, st>>>(A);
   }
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, "launch of the Adagrad local-step kernels", e);
+  ctx->work.note(st);
   return GBMUF_OK;
 }
 
@@ -744,7 +826,18 @@ gbmuf_status gbmuf_sync_round(gbmuf_ctx* ctx, uint64_t round, const uint8_t* com
   cudaStream_t st = (cudaStream_t)stream;
   cudaError_t e;
   if (comp_mask) {
-    e = cudaMemcpyAsync(ctx->d_mask, comp_mask, ctx->m, cudaMemcpyHostToDevice, st);
+    // A mask is host data that must reach the device.  It cannot be recorded into a stream
+    // capture (a replay would upload whatever the staging copy holds by then); rounds selected
+    // by periods can.
+    if (is_capturing(st))
+      return fail(ctx, GBMUF_ERR_BAD_STATE,
+                  "a component mask cannot be recorded into a stream capture; select components by periods there");
+    // The caller's array may be page-locked, and a copy from page-locked memory really is
+    // asynchronous.  The upload therefore starts from the library's own pageable copy: the
+    // runtime moves pageable bytes into its staging area before cudaMemcpyAsync returns, so
+    // neither the caller's array nor this copy is read after the call.
+    ctx->mask_stage.assign(comp_mask, comp_mask + ctx->m);
+    e = cudaMemcpyAsync(ctx->d_mask, ctx->mask_stage.data(), ctx->m, cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return cuda_fail(ctx, "upload of the component mask", e);
   }
   SetupParams S;
@@ -754,8 +847,10 @@ gbmuf_status gbmuf_sync_round(gbmuf_ctx* ctx, uint64_t round, const uint8_t* com
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, "launch of the round set-up kernel", e);
 
-  return launch_round(ctx, ctx->cfg, L, ctx->theta, ctx->omega, ctx->delta, ctx->cfg.ld, ctx->m, ctx->d_off,
-                      ctx->d_prefix, ctx->d_nbr, ctx->d_status, total, st);
+  const gbmuf_status rc = launch_round(ctx, ctx->cfg, L, ctx->theta, ctx->omega, ctx->delta, ctx->cfg.ld, ctx->m,
+                                       ctx->d_off, ctx->d_prefix, ctx->d_nbr, ctx->d_status, total, st);
+  ctx->work.note(st);
+  return rc;
 }
 
 gbmuf_status gbmuf_get_neighbors(gbmuf_ctx* ctx, uint64_t round, int32_t* out) {
@@ -801,6 +896,7 @@ gbmuf_status gbmuf_final_average(gbmuf_ctx* ctx, void* out, void* stream) {
                                                               ctx->cfg.N, ctx->cfg.ld);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, "launch of the final-average kernel", e);
+  ctx->work.note(st);
   return GBMUF_OK;
 }
 
@@ -889,7 +985,10 @@ gbmuf_status gbmuf_destroy(gbmuf_ctx* ctx) {
   {
     DeviceGuard guard(ctx->cfg.device);
     if (guard.ok) {
-      if (cudaDeviceSynchronize() != cudaSuccess) rc = GBMUF_ERR_CUDA;
+      // wait for this context's own work, not for the whole device
+      if (ctx->work.wait() != cudaSuccess) rc = GBMUF_ERR_CUDA;
+      if (ctx->priv && cudaStreamSynchronize(ctx->priv) != cudaSuccess) rc = GBMUF_ERR_CUDA;
+      ctx->work.release();
       free_tables(ctx);
       cudaFree(ctx->d_status);
       cudaFree(ctx->d_norm_partial);
@@ -926,6 +1025,15 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
 constexpr int kNoAllocMaxDevices = 64;
 unsigned char* g_noalloc_ptr[kNoAllocMaxDevices] = {};   // device address of the array, per GPU
 
+// Host-side staging of the two tables a call uploads, in ordinary (pageable) static memory: the
+// caller's arrays may be page-locked, from which an asynchronous copy reads later, whereas the
+// runtime has moved pageable bytes into its own staging area by the time cudaMemcpyAsync
+// returns.  The mutex covers filling and handing over; it does not make overlapping calls
+// safe on the GPU (they share the device array).
+std::mutex g_noalloc_mutex;
+int64_t g_noalloc_off_stage[kNoAllocMaxM + 1];
+uint8_t g_noalloc_flag_stage[kNoAllocMaxM];
+
 }  // namespace
 
 gbmuf_status gbmuf_sync_round_noalloc(const gbmuf_config* cfg, void* theta, float* omega,
@@ -961,12 +1069,25 @@ gbmuf_status gbmuf_sync_round_noalloc(const gbmuf_config* cfg, void* theta, floa
 
   DeviceGuard guard(cfg->device);
   if (!guard.ok) return fail(nullptr, GBMUF_ERR_CUDA, "cudaSetDevice failed");
+  cudaStream_t cs = (cudaStream_t)stream;
+  // The call uploads host tables, so it cannot be part of a stream capture: the recorded copies
+  // would read this library's staging arrays again at every replay, with whatever a later call
+  // left there.  Refused before anything is enqueued.
+  if (is_capturing(cs))
+    return fail(nullptr, GBMUF_ERR_BAD_STATE,
+                "gbmuf_sync_round_noalloc uploads host tables and cannot be recorded into a stream capture");
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
   cudaError_t e;
+  int v = 0;
   if (!g_noalloc_ptr[cfg->device]) {
-    // once per device, with that device current: ask the runtime where the array lives there
+    // once per device, with that device current: ask the runtime where the array lives there,
+    // and raise the kernels' shared-memory limit
     unsigned char* ptr = nullptr;
     e = cudaGetSymbolAddress((void**)&ptr, g_noalloc_scratch);
     if (e != cudaSuccess || !ptr) return cuda_fail(nullptr, "cudaGetSymbolAddress of the fixed scratch array", e);
+    cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerBlockOptin, cfg->device);
+    e = ensure_kernel_attributes(cfg->device, v);
+    if (e != cudaSuccess) return cuda_fail(nullptr, "raising the kernels' shared-memory limit", e);
     g_noalloc_ptr[cfg->device] = ptr;
   }
   unsigned char* scratch = g_noalloc_ptr[cfg->device];
@@ -974,7 +1095,6 @@ gbmuf_status gbmuf_sync_round_noalloc(const gbmuf_config* cfg, void* theta, floa
   // a context on the stack: it owns nothing, it only carries the description to the helpers
   gbmuf_ctx tmp;
   tmp.cfg = *cfg; tmp.theta = theta; tmp.omega = omega; tmp.delta = delta; tmp.m = m; tmp.cand = cand;
-  int v = 0;
   cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, cfg->device); tmp.num_sms = v;
   cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerBlockOptin, cfg->device); tmp.max_smem = v;
   cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerMultiprocessor, cfg->device); tmp.smem_per_sm = v;
@@ -983,22 +1103,23 @@ gbmuf_status gbmuf_sync_round_noalloc(const gbmuf_config* cfg, void* theta, floa
   if (st != GBMUF_OK) { g_create_error = tmp.err; return st; }
   const Launch& L = tmp.launch;
 
-  uint8_t flags[kNoAllocMaxM];
+  uint8_t* const flags = g_noalloc_flag_stage;
   long long total = 0;
   for (int i = 0; i < m; ++i) {
     flags[i] = comp_mask ? (comp_mask[i] != 0) : 1;
+    g_noalloc_off_stage[i] = offsets[i];
     if (!flags[i]) continue;
     const int64_t start = offsets[i] & ~(int64_t)(kAlign - 1);
     total += (offsets[i + 1] - start + L.T - 1) / L.T;
   }
+  g_noalloc_off_stage[m] = offsets[m];
   if (total > 0x3fffffffLL) return fail(nullptr, GBMUF_ERR_UNSUPPORTED, "more than 2^30 - 1 tiles");
-  cudaStream_t cs = (cudaStream_t)stream;
   int32_t* d_status = reinterpret_cast<int32_t*>(scratch + kNaStatusOff);
   // the array keeps whatever the previous call left: the status word must start at zero, the
   // other tables are rewritten in full below for the sizes of this call
   e = cudaMemsetAsync(d_status, 0, sizeof(int32_t), cs);
   if (e == cudaSuccess && total > 0)
-    e = cudaMemcpyAsync(scratch + kNaOffsetsOff, offsets, (size_t)(m + 1) * sizeof(int64_t), cudaMemcpyHostToDevice, cs);
+    e = cudaMemcpyAsync(scratch + kNaOffsetsOff, g_noalloc_off_stage, (size_t)(m + 1) * sizeof(int64_t), cudaMemcpyHostToDevice, cs);
   if (e == cudaSuccess && total > 0)
     e = cudaMemcpyAsync(scratch + kNaMaskOff, flags, (size_t)m, cudaMemcpyHostToDevice, cs);
   if (e != cudaSuccess) return cuda_fail(nullptr, "upload of offsets and mask into the fixed scratch array", e);
@@ -1032,30 +1153,74 @@ gbmuf_status gbmuf_sync_round_noalloc(const gbmuf_config* cfg, void* theta, floa
 
 
 // -------------------------------------------------------------------------------------------------
-// gbmuf_sync_round_host: one round over replicas that live in HOST memory.
+// Replicas that live in HOST memory: gbmuf_host_* and the one-call form gbmuf_sync_round_host.
 // -------------------------------------------------------------------------------------------------
+}  // extern "C"
+
 namespace {
 
-struct HostSet {               // one of the buffer sets column chunks rotate through
+struct HostChunk {             // one column chunk [c0, c1) of the model
+  long long c0, c1;
+  int first, mc;               // first component that reaches into it, and how many do
+  size_t off_at, mask_at;      // where its local offsets (mc + 1) / flags (mc) start in the arenas
+};
+
+struct HostSet {               // one of the buffer sets the chunks rotate through
   gbmuf_ctx ctx;               // describes the device chunk buffers to the launch helpers
-  unsigned char* tables = nullptr;
+  unsigned char* tables = nullptr;   // prefix | nbr | mask | status
   cudaStream_t stream = nullptr;
 };
 
-void free_host_sets(HostSet* sets, int n) {
-  for (int i = 0; i < n; ++i) {
-    cudaFree(sets[i].ctx.theta); cudaFree(sets[i].ctx.omega); cudaFree(sets[i].ctx.delta);
-    cudaFree(sets[i].tables);
-    if (sets[i].stream) cudaStreamDestroy(sets[i].stream);
+constexpr int kHostSets = 3;
+
+}  // namespace
+
+struct gbmuf_host {
+  gbmuf_config cfg;
+  int m = 0, esz = 4, nsets = 0;
+  long long chunk_cols = 0;
+  int row_copies = 0;          // one cudaMemcpyAsync per row instead of one 2-D copy per array
+  std::vector<int64_t> off;
+  std::vector<HostChunk> chunks;
+  HostSet sets[kHostSets];
+  int64_t* d_chunk_off = nullptr;   // device: every chunk's local offsets, back to back
+  uint8_t* h_flags = nullptr;       // page-locked: every chunk's participation flags of this round
+  size_t t_nbr = 0, t_mask = 0, t_status = 0, t_bytes = 0;
+};
+
+namespace {
+
+void free_host_handle(gbmuf_host* h) {
+  for (int i = 0; i < kHostSets; ++i) {
+    HostSet& s = h->sets[i];
+    cudaFree(s.ctx.theta); cudaFree(s.ctx.omega); cudaFree(s.ctx.delta); cudaFree(s.tables);
+    if (s.stream) cudaStreamDestroy(s.stream);
   }
+  cudaFree(h->d_chunk_off);
+  if (h->h_flags) cudaFreeHost(h->h_flags);
+  delete h;
+}
+
+// rows [0, K) x columns of one array between host (row stride ld_h) and a chunk buffer (row
+// stride ld_d), as one 2-D copy or as K row copies
+cudaError_t copy_rows(void* dst, size_t dpitch, const void* src, size_t spitch, size_t width, int K,
+                      cudaMemcpyKind kind, cudaStream_t st, bool row_copies) {
+  if (!row_copies) return cudaMemcpy2DAsync(dst, dpitch, src, spitch, width, K, kind, st);
+  for (int k = 0; k < K; ++k) {
+    const cudaError_t e = cudaMemcpyAsync((char*)dst + (size_t)k * dpitch, (const char*)src + (size_t)k * spitch,
+                                          width, kind, st);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
 }
 
 }  // namespace
 
-gbmuf_status gbmuf_sync_round_host(const gbmuf_config* cfg, void* theta, float* omega, float* delta,
-                                   int32_t m, const int64_t* offsets, const uint8_t* comp_mask,
-                                   uint64_t round, int64_t chunk_cols) {
-  if (!cfg) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "cfg must not be NULL");
+extern "C" {
+
+gbmuf_status gbmuf_host_create(const gbmuf_config* cfg, int32_t m, const int64_t* offsets,
+                               int64_t chunk_cols, int32_t flags, gbmuf_host** out) {
+  if (!cfg || !out) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "cfg and out must not be NULL");
   if (cfg->K < 1 || cfg->K > 256 || cfg->N < 1 || cfg->ld < cfg->N || cfg->p < 0 || cfg->q < 0 ||
       cfg->comp_base < 0 || (cfg->mode != GBMUF_MODE_BMUF && cfg->mode != GBMUF_MODE_MA) ||
       (cfg->theta_dtype != GBMUF_F32 && cfg->theta_dtype != GBMUF_BF16) ||
@@ -1064,7 +1229,6 @@ gbmuf_status gbmuf_sync_round_host(const gbmuf_config* cfg, void* theta, float* 
   const int cand = host_candidates(cfg->K, cfg->p);
   if (cfg->q > cand || cand > kMaxCand)
     return fail(nullptr, GBMUF_ERR_INVALID_ARG, "q exceeds the ring neighbours min(2p, K-1), or more than 64 of them");
-  if (!theta || !omega || !delta) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "theta, omega and delta must not be NULL");
   if (m < 1 || m > 65536 || !offsets) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "m must be in 1..65536 and offsets not NULL");
   if (offsets[0] != 0 || offsets[m] != cfg->N)
     return fail(nullptr, GBMUF_ERR_INVALID_ARG, "offsets[0] must be 0 and offsets[m] must be N");
@@ -1072,42 +1236,72 @@ gbmuf_status gbmuf_sync_round_host(const gbmuf_config* cfg, void* theta, float* 
     if (offsets[i + 1] <= offsets[i]) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "offsets must be strictly increasing");
   if (chunk_cols < 0 || (chunk_cols > 0 && chunk_cols % 32 != 0) || chunk_cols > (1LL << 30))
     return fail(nullptr, GBMUF_ERR_INVALID_ARG, "chunk_cols must be 0 or a multiple of 32 up to 2^30");
-  if (chunk_cols == 0) chunk_cols = 1 << 22;
+  if (flags < 0 || flags > 1) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "unknown flags");
+  if (chunk_cols == 0) chunk_cols = 1 << 21;
   const long long N = cfg->N;
   if (chunk_cols > (N + 31) / 32 * 32) chunk_cols = (N + 31) / 32 * 32;
   const long long nchunks = (N + chunk_cols - 1) / chunk_cols;
-  const int esz = cfg->theta_dtype == GBMUF_F32 ? 4 : 2;
   const int K = cfg->K, q = cfg->q;
 
+  int ndev = 0;
+  cudaError_t e = cudaGetDeviceCount(&ndev);
+  if (e != cudaSuccess) return cuda_fail(nullptr, "cudaGetDeviceCount", e);
+  if (cfg->device >= ndev) return fail(nullptr, GBMUF_ERR_INVALID_ARG, "no such CUDA device");
   DeviceGuard guard(cfg->device);
   if (!guard.ok) return fail(nullptr, GBMUF_ERR_CUDA, "cudaSetDevice failed");
 
-  constexpr int kSets = 3;
-  const int nsets = nchunks < kSets ? (int)nchunks : kSets;
-  HostSet sets[kSets];
-  for (int i = 0; i < kSets; ++i) { sets[i].ctx.theta = nullptr; sets[i].ctx.omega = nullptr; sets[i].ctx.delta = nullptr; }
-  // table block of one set: offsets int64 [m+2] | prefix int32 [m+2] | nbr int32 [K*(m+1)*q] | mask
-  const size_t t_off = 0, t_prefix = ((size_t)(m + 2) * 8 + 255) / 256 * 256;
-  const size_t t_nbr = t_prefix + ((size_t)(m + 2) * 4 + 255) / 256 * 256;
-  const size_t t_mask = t_nbr + ((size_t)K * (m + 1) * (q > 0 ? q : 1) * 4 + 255) / 256 * 256;
-  const size_t t_status = t_mask + ((size_t)(m + 1) + 255) / 256 * 256;
-  const size_t t_bytes = t_status + 256;
+  gbmuf_host* h = new (std::nothrow) gbmuf_host();
+  if (!h) return fail(nullptr, GBMUF_ERR_ALLOC, "out of host memory");
+  h->cfg = *cfg; h->m = m; h->chunk_cols = chunk_cols; h->row_copies = flags & 1;
+  h->esz = cfg->theta_dtype == GBMUF_F32 ? 4 : 2;
+  h->off.assign(offsets, offsets + m + 1);
+  h->nsets = nchunks < kHostSets ? (int)nchunks : kHostSets;
+
+  // the chunks and their local partitions: fixed for the life of the handle
+  std::vector<int64_t> all_off;
+  size_t nflags = 0;
+  int first = 0, mc_max = 1;
+  for (long long ci = 0; ci < nchunks; ++ci) {
+    HostChunk c;
+    c.c0 = ci * chunk_cols;
+    c.c1 = c.c0 + chunk_cols < N ? c.c0 + chunk_cols : N;
+    while (offsets[first + 1] <= c.c0) ++first;
+    c.first = first; c.off_at = all_off.size(); c.mask_at = nflags;
+    all_off.push_back(0);
+    int i = first;
+    while (true) {
+      all_off.push_back(offsets[i + 1] < c.c1 ? offsets[i + 1] - c.c0 : c.c1 - c.c0);
+      if (offsets[i + 1] >= c.c1) break;
+      ++i;
+    }
+    c.mc = i - first + 1;
+    nflags += (size_t)c.mc;
+    if (c.mc > mc_max) mc_max = c.mc;
+    h->chunks.push_back(c);
+  }
+  // table block of one set: prefix int32 [mc_max + 1] | nbr int32 [K * mc_max * q] | mask | status
+  auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+  h->t_nbr = up((size_t)(mc_max + 1) * 4);
+  h->t_mask = h->t_nbr + up((size_t)K * mc_max * (q > 0 ? q : 1) * 4);
+  h->t_status = h->t_mask + up((size_t)mc_max);
+  h->t_bytes = h->t_status + 256;
+
   gbmuf_status st = GBMUF_OK;
-  cudaError_t e = cudaSuccess;
-  for (int i = 0; i < nsets && st == GBMUF_OK; ++i) {
-    gbmuf_ctx& c = sets[i].ctx;
-    c.cfg = *cfg; c.cfg.N = chunk_cols; c.cfg.ld = chunk_cols; c.m = m; c.cand = cand;
+  for (int i = 0; i < h->nsets && st == GBMUF_OK; ++i) {
+    gbmuf_ctx& c = h->sets[i].ctx;
+    c.cfg = *cfg; c.cfg.N = chunk_cols; c.cfg.ld = chunk_cols; c.m = mc_max; c.cand = cand;
     c.theta = nullptr; c.omega = nullptr; c.delta = nullptr;
     int v = 0;
     cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, cfg->device); c.num_sms = v;
     cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerBlockOptin, cfg->device); c.max_smem = v;
     cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerMultiprocessor, cfg->device); c.smem_per_sm = v;
-    e = cudaMalloc(&c.theta, (size_t)K * chunk_cols * esz);
-    if (e == cudaSuccess) e = cudaMalloc(&c.omega, (size_t)K * chunk_cols * 4);
-    if (e == cudaSuccess) e = cudaMalloc(&c.delta, (size_t)K * chunk_cols * 4);
-    if (e == cudaSuccess) e = cudaMalloc(&sets[i].tables, t_bytes);
-    if (e == cudaSuccess) e = cudaMemset(sets[i].tables + t_status, 0, 256);
-    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&sets[i].stream, cudaStreamNonBlocking);
+    e = cudaMalloc(&c.theta, (size_t)K * chunk_cols * h->esz);
+    if (e == cudaSuccess && cfg->mode == GBMUF_MODE_BMUF) e = cudaMalloc(&c.omega, (size_t)K * chunk_cols * 4);
+    if (e == cudaSuccess && cfg->mode == GBMUF_MODE_BMUF) e = cudaMalloc(&c.delta, (size_t)K * chunk_cols * 4);
+    if (e == cudaSuccess) e = cudaMalloc(&h->sets[i].tables, h->t_bytes);
+    if (e == cudaSuccess) e = cudaMemset(h->sets[i].tables + h->t_status, 0, 256);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->sets[i].stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess && i == 0) e = ensure_kernel_attributes(cfg->device, c.max_smem);
     if (e != cudaSuccess) {
       st = e == cudaErrorMemoryAllocation ? fail(nullptr, GBMUF_ERR_ALLOC, "device chunk buffers")
                                           : cuda_fail(nullptr, "set-up of the chunk buffers", e);
@@ -1117,89 +1311,128 @@ gbmuf_status gbmuf_sync_round_host(const gbmuf_config* cfg, void* theta, float* 
     if (st == GBMUF_OK) st = build_tensor_maps(&c, c.launch);
     if (st != GBMUF_OK) g_create_error = c.err;
   }
-  if (st != GBMUF_OK) { free_host_sets(sets, nsets); return st; }
+  if (st == GBMUF_OK) {
+    e = cudaMalloc(&h->d_chunk_off, all_off.size() * sizeof(int64_t));
+    if (e == cudaSuccess)
+      e = cudaMemcpyAsync(h->d_chunk_off, all_off.data(), all_off.size() * sizeof(int64_t), cudaMemcpyHostToDevice,
+                          h->sets[0].stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(h->sets[0].stream);   // the table is in place
+    if (e == cudaSuccess) e = cudaHostAlloc((void**)&h->h_flags, nflags, cudaHostAllocDefault);
+    if (e != cudaSuccess)
+      st = e == cudaErrorMemoryAllocation ? fail(nullptr, GBMUF_ERR_ALLOC, "chunk tables") : cuda_fail(nullptr, "chunk tables", e);
+  }
+  if (st != GBMUF_OK) { free_host_handle(h); return st; }
+  *out = h;
+  return GBMUF_OK;
+}
 
-  // per-chunk host tables must outlive the asynchronous uploads
-  std::vector<std::vector<int64_t>> chunk_off((size_t)nchunks);
-  std::vector<std::vector<uint8_t>> chunk_mask((size_t)nchunks);
-  int first = 0;   // first component that reaches into the current chunk
-  for (long long ci = 0; ci < nchunks && st == GBMUF_OK; ++ci) {
-    const long long c0 = ci * chunk_cols, c1 = c0 + chunk_cols < N ? c0 + chunk_cols : N;
-    while (offsets[first + 1] <= c0) ++first;
-    std::vector<int64_t>& lo = chunk_off[(size_t)ci];
-    std::vector<uint8_t>& mk = chunk_mask[(size_t)ci];
-    lo.push_back(0);
-    int i = first;
-    long long total = 0;
-    HostSet& hs = sets[ci % nsets];
+gbmuf_status gbmuf_host_sync_round(gbmuf_host* h, void* theta, float* omega, float* delta,
+                                   const uint8_t* comp_mask, uint64_t round) {
+  if (!h) return GBMUF_ERR_INVALID_ARG;
+  const gbmuf_config& cfg = h->cfg;
+  const bool bmuf = cfg.mode == GBMUF_MODE_BMUF;
+  if (!theta || (bmuf && (!omega || !delta)))
+    return fail(nullptr, GBMUF_ERR_INVALID_ARG, "theta, omega and delta must not be NULL");
+  DeviceGuard guard(cfg.device);
+  if (!guard.ok) return fail(nullptr, GBMUF_ERR_CUDA, "cudaSetDevice failed");
+  const int K = cfg.K, q = cfg.q, esz = h->esz;
+  const long long chunk_cols = h->chunk_cols;
+  const bool rc = h->row_copies != 0;
+  gbmuf_status st = GBMUF_OK;
+  cudaError_t e = cudaSuccess;
+  for (size_t ci = 0; ci < h->chunks.size() && st == GBMUF_OK; ++ci) {
+    const HostChunk& c = h->chunks[ci];
+    HostSet& hs = h->sets[ci % (size_t)h->nsets];
     const int T = hs.ctx.launch.T;
-    while (true) {
-      const long long b = offsets[i] > c0 ? offsets[i] - c0 : 0;
-      const long long en = offsets[i + 1] < c1 ? offsets[i + 1] - c0 : c1 - c0;
-      const uint8_t due = comp_mask ? (comp_mask[i] != 0) : 1;
-      mk.push_back(due);
-      lo.push_back(en);
-      if (due) total += (en - (b & ~(long long)(kAlign - 1)) + T - 1) / T;
-      if (offsets[i + 1] >= c1) break;
-      ++i;
+    const int64_t* lo = h->off.data();
+    uint8_t* fl = h->h_flags + c.mask_at;           // this chunk's own bytes: nothing reuses them
+    long long total = 0;                            // before the call returns
+    for (int j = 0; j < c.mc; ++j) {
+      const int i = c.first + j;
+      const long long b = lo[i] > c.c0 ? lo[i] - c.c0 : 0;
+      const long long en = lo[i + 1] < c.c1 ? lo[i + 1] - c.c0 : c.c1 - c.c0;
+      fl[j] = comp_mask ? (comp_mask[i] != 0) : 1;
+      if (fl[j]) total += (en - (b & ~(long long)(kAlign - 1)) + T - 1) / T;
     }
-    if (total == 0) continue;                    // nothing in this chunk takes part: leave it alone
-    const int mc = (int)mk.size();
+    if (total == 0) continue;                       // nothing in this chunk takes part: leave it alone
     cudaStream_t cs = hs.stream;
-    const size_t w_th = (size_t)(c1 - c0) * esz, w_f = (size_t)(c1 - c0) * 4;
-    e = cudaMemcpy2DAsync(hs.ctx.theta, (size_t)chunk_cols * esz, (const char*)theta + (size_t)c0 * esz,
-                          (size_t)cfg->ld * esz, w_th, K, cudaMemcpyHostToDevice, cs);
-    if (e == cudaSuccess && cfg->mode == GBMUF_MODE_BMUF) {
-      e = cudaMemcpy2DAsync(hs.ctx.omega, (size_t)chunk_cols * 4, omega + c0, (size_t)cfg->ld * 4, w_f, K,
-                            cudaMemcpyHostToDevice, cs);
+    const long long c0 = c.c0;
+    const size_t w_th = (size_t)(c.c1 - c0) * esz, w_f = (size_t)(c.c1 - c0) * 4;
+    e = copy_rows(hs.ctx.theta, (size_t)chunk_cols * esz, (const char*)theta + (size_t)c0 * esz,
+                  (size_t)cfg.ld * esz, w_th, K, cudaMemcpyHostToDevice, cs, rc);
+    if (e == cudaSuccess && bmuf) {
+      e = copy_rows(hs.ctx.omega, (size_t)chunk_cols * 4, omega + c0, (size_t)cfg.ld * 4, w_f, K,
+                    cudaMemcpyHostToDevice, cs, rc);
       if (e == cudaSuccess)
-        e = cudaMemcpy2DAsync(hs.ctx.delta, (size_t)chunk_cols * 4, delta + c0, (size_t)cfg->ld * 4, w_f, K,
-                              cudaMemcpyHostToDevice, cs);
+        e = copy_rows(hs.ctx.delta, (size_t)chunk_cols * 4, delta + c0, (size_t)cfg.ld * 4, w_f, K,
+                      cudaMemcpyHostToDevice, cs, rc);
     }
     if (e == cudaSuccess)
-      e = cudaMemcpyAsync(hs.tables + t_off, lo.data(), (size_t)(mc + 1) * 8, cudaMemcpyHostToDevice, cs);
-    if (e == cudaSuccess)
-      e = cudaMemcpyAsync(hs.tables + t_mask, mk.data(), (size_t)mc, cudaMemcpyHostToDevice, cs);
+      e = cudaMemcpyAsync(hs.tables + h->t_mask, fl, (size_t)c.mc, cudaMemcpyHostToDevice, cs);
     if (e != cudaSuccess) { st = cuda_fail(nullptr, "host-to-device copy of a column chunk", e); break; }
 
     SetupParams S;
-    S.K = K; S.m = mc; S.p = cfg->p; S.q = q; S.comp_base = cfg->comp_base + first; S.T = T;
-    S.use_mask = 1; S.plan = 1; S.seed = cfg->seed; S.round = round;
-    S.off = reinterpret_cast<const int64_t*>(hs.tables + t_off);
+    S.K = K; S.m = c.mc; S.p = cfg.p; S.q = q; S.comp_base = cfg.comp_base + c.first; S.T = T;
+    S.use_mask = 1; S.plan = 1; S.seed = cfg.seed; S.round = round;
+    S.off = h->d_chunk_off + c.off_at;
     S.periods = nullptr;
-    S.mask = hs.tables + t_mask;
-    S.nbr = reinterpret_cast<int32_t*>(hs.tables + t_nbr);
-    S.tile_prefix = reinterpret_cast<int32_t*>(hs.tables + t_prefix);
-    round_setup_kernel<<<(int)(((long long)K * mc + 255) / 256), 256, 0, cs>>>(S);
+    S.mask = hs.tables + h->t_mask;
+    S.nbr = reinterpret_cast<int32_t*>(hs.tables + h->t_nbr);
+    S.tile_prefix = reinterpret_cast<int32_t*>(hs.tables);
+    round_setup_kernel<<<(int)(((long long)K * c.mc + 255) / 256), 256, 0, cs>>>(S);
     e = cudaGetLastError();
     if (e != cudaSuccess) { st = cuda_fail(nullptr, "launch of the round set-up kernel", e); break; }
-    const Launch& L = hs.ctx.launch;
-    st = launch_round(&hs.ctx, *cfg, L, hs.ctx.theta, hs.ctx.omega, hs.ctx.delta, chunk_cols, mc, S.off,
-                      S.tile_prefix, S.nbr, reinterpret_cast<int32_t*>(hs.tables + t_status), total, cs);
+    st = launch_round(&hs.ctx, cfg, hs.ctx.launch, hs.ctx.theta, hs.ctx.omega, hs.ctx.delta, chunk_cols, c.mc,
+                      S.off, S.tile_prefix, S.nbr, reinterpret_cast<int32_t*>(hs.tables + h->t_status), total, cs);
     if (st != GBMUF_OK) { g_create_error = hs.ctx.err; break; }
-    e = cudaMemcpy2DAsync((char*)theta + (size_t)c0 * esz, (size_t)cfg->ld * esz, hs.ctx.theta,
-                          (size_t)chunk_cols * esz, w_th, K, cudaMemcpyDeviceToHost, cs);
-    if (e == cudaSuccess && cfg->mode == GBMUF_MODE_BMUF) {
-      e = cudaMemcpy2DAsync(omega + c0, (size_t)cfg->ld * 4, hs.ctx.omega, (size_t)chunk_cols * 4, w_f, K,
-                            cudaMemcpyDeviceToHost, cs);
+    e = copy_rows((char*)theta + (size_t)c0 * esz, (size_t)cfg.ld * esz, hs.ctx.theta, (size_t)chunk_cols * esz,
+                  w_th, K, cudaMemcpyDeviceToHost, cs, rc);
+    if (e == cudaSuccess && bmuf) {
+      e = copy_rows(omega + c0, (size_t)cfg.ld * 4, hs.ctx.omega, (size_t)chunk_cols * 4, w_f, K,
+                    cudaMemcpyDeviceToHost, cs, rc);
       if (e == cudaSuccess)
-        e = cudaMemcpy2DAsync(delta + c0, (size_t)cfg->ld * 4, hs.ctx.delta, (size_t)chunk_cols * 4, w_f, K,
-                              cudaMemcpyDeviceToHost, cs);
+        e = copy_rows(delta + c0, (size_t)cfg.ld * 4, hs.ctx.delta, (size_t)chunk_cols * 4, w_f, K,
+                      cudaMemcpyDeviceToHost, cs, rc);
     }
     if (e != cudaSuccess) { st = cuda_fail(nullptr, "device-to-host copy of a column chunk", e); break; }
   }
+  // the call returns when the host arrays hold the result: wait for every set, read its status
   int32_t worst = 0;
-  for (int i = 0; i < nsets; ++i) {
-    e = cudaStreamSynchronize(sets[i].stream);
+  for (int i = 0; i < h->nsets; ++i) {
     int32_t word = 0;
-    if (e == cudaSuccess) e = cudaMemcpy(&word, sets[i].tables + t_status, 4, cudaMemcpyDeviceToHost);
+    e = cudaMemcpyAsync(&word, h->sets[i].tables + h->t_status, 4, cudaMemcpyDeviceToHost, h->sets[i].stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(h->sets[i].stream);
     if (e != cudaSuccess && st == GBMUF_OK) st = cuda_fail(nullptr, "waiting for the column chunks", e);
-    if (word != 0) worst = word;
+    if (word != 0) {
+      worst = word;
+      cudaMemsetAsync(h->sets[i].tables + h->t_status, 0, 4, h->sets[i].stream);
+    }
   }
-  free_host_sets(sets, nsets);
   if (st == GBMUF_OK && worst != 0)
     st = fail(nullptr, GBMUF_ERR_TIMEOUT, "a bounded device-side wait expired; the host arrays are unspecified");
   return st;
+}
+
+gbmuf_status gbmuf_host_destroy(gbmuf_host* h) {
+  if (!h) return GBMUF_OK;
+  gbmuf_status rc = GBMUF_OK;
+  DeviceGuard guard(h->cfg.device);
+  if (!guard.ok) rc = GBMUF_ERR_CUDA;
+  for (int i = 0; i < h->nsets && guard.ok; ++i)
+    if (h->sets[i].stream && cudaStreamSynchronize(h->sets[i].stream) != cudaSuccess) rc = GBMUF_ERR_CUDA;
+  free_host_handle(h);
+  return rc;
+}
+
+gbmuf_status gbmuf_sync_round_host(const gbmuf_config* cfg, void* theta, float* omega, float* delta,
+                                   int32_t m, const int64_t* offsets, const uint8_t* comp_mask,
+                                   uint64_t round, int64_t chunk_cols) {
+  gbmuf_host* h = nullptr;
+  gbmuf_status st = gbmuf_host_create(cfg, m, offsets, chunk_cols, 0, &h);
+  if (st != GBMUF_OK) return st;
+  st = gbmuf_host_sync_round(h, theta, omega, delta, comp_mask, round);
+  const gbmuf_status st2 = gbmuf_host_destroy(h);
+  return st != GBMUF_OK ? st : st2;
 }
 
 
@@ -1226,6 +1459,9 @@ struct gbmuf_peer {
   int num_sms = 0, max_smem = 0;
   int T = 0, stages = 0, ncons = 0;
   uint32_t stage_stride = 0, omega_off = 0, delta_off = 0, desc_off = 0, smem = 0;
+  std::vector<uint8_t> mask_stage;   // the library's own (pageable) copy of a caller's mask
+  size_t cap_bytes = 0;              // size the table block was allocated for
+  WorkMarks work;
 };
 
 extern "C" {
@@ -1292,7 +1528,8 @@ gbmuf_status gbmuf_peer_create(const gbmuf_config* cfg, int32_t rank, void* cons
   h->smem = 128 + (uint32_t)h->stages * h->stage_stride;
   int n = (T / 4 + 31) / 32 * 32;
   h->ncons = n < 128 ? 128 : n > 992 ? 992 : n;
-  e = cudaMalloc(&h->d_status, sizeof(int32_t));
+  e = ensure_kernel_attributes(cfg->device, h->max_smem);
+  if (e == cudaSuccess) e = cudaMalloc(&h->d_status, sizeof(int32_t));
   if (e == cudaSuccess) e = cudaMemset(h->d_status, 0, sizeof(int32_t));
   for (int b = 0; b < 2 && e == cudaSuccess; ++b) {
     e = cudaMalloc(&h->d_theta_in[b], (size_t)cfg->K * sizeof(void*));
@@ -1322,10 +1559,8 @@ gbmuf_status gbmuf_peer_set_partition(gbmuf_peer* h, int32_t m, const int64_t* o
   }
   DeviceGuard guard(h->cfg.device);
   if (!guard.ok) return fail(nullptr, GBMUF_ERR_CUDA, "cudaSetDevice failed");
-  cudaError_t e = cudaDeviceSynchronize();
-  if (e != cudaSuccess) return cuda_fail(nullptr, "cudaDeviceSynchronize", e);
-  cudaFree(h->tables);
-  h->tables = nullptr;
+  cudaError_t e = h->work.wait();               // this worker's earlier rounds, nothing else
+  if (e != cudaSuccess) return cuda_fail(nullptr, "waiting for the worker's earlier work", e);
   h->partitioned = false;
   h->m = m;
   h->off.assign(offsets, offsets + m + 1);
@@ -1347,13 +1582,19 @@ gbmuf_status gbmuf_peer_set_partition(gbmuf_peer* h, int32_t m, const int64_t* o
   h->t_due = h->t_mask + up((size_t)m);
   h->t_nbr = h->t_due + up((size_t)m);
   const size_t bytes = h->t_nbr + up((size_t)m * (h->cfg.q > 0 ? h->cfg.q : 1) * 4);
-  e = cudaMalloc(&h->tables, bytes);
+  if (bytes > h->cap_bytes) {
+    cudaFree(h->tables);
+    h->tables = nullptr; h->cap_bytes = 0;
+    e = cudaMalloc(&h->tables, bytes);
+    if (e == cudaSuccess) h->cap_bytes = bytes;
+  }
   if (e == cudaSuccess) e = cudaMemcpy(h->tables, h->off.data(), (size_t)(m + 1) * 8, cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMemcpy(h->tables + h->t_prefix, prefix.data(), (size_t)(m + 1) * 4, cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMemcpy(h->tables + h->t_periods, h->periods.data(), (size_t)m * 4, cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(nullptr);   // the copies above have landed
   if (e != cudaSuccess) {
     cudaFree(h->tables);
-    h->tables = nullptr;
+    h->tables = nullptr; h->cap_bytes = 0;
     return e == cudaErrorMemoryAllocation ? fail(nullptr, GBMUF_ERR_ALLOC, "partition tables") : cuda_fail(nullptr, "partition upload", e);
   }
   h->partitioned = true;
@@ -1370,7 +1611,14 @@ gbmuf_status gbmuf_peer_sync_round(gbmuf_peer* h, uint64_t round, const uint8_t*
   cudaStream_t st = (cudaStream_t)stream;
   cudaError_t e;
   if (comp_mask) {
-    e = cudaMemcpyAsync(h->tables + h->t_mask, comp_mask, (size_t)h->m, cudaMemcpyHostToDevice, st);
+    // as in gbmuf_sync_round: no mask inside a stream capture, and the upload starts from the
+    // library's own pageable copy so that the caller's (possibly page-locked) array is not read
+    // after the call
+    if (is_capturing(st))
+      return fail(nullptr, GBMUF_ERR_BAD_STATE,
+                  "a component mask cannot be recorded into a stream capture; select components by periods there");
+    h->mask_stage.assign(comp_mask, comp_mask + h->m);
+    e = cudaMemcpyAsync(h->tables + h->t_mask, h->mask_stage.data(), (size_t)h->m, cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return cuda_fail(nullptr, "upload of the component mask", e);
   }
   PeerPlanParams Q;
@@ -1398,14 +1646,12 @@ gbmuf_status gbmuf_peer_sync_round(gbmuf_peer* h, uint64_t round, const uint8_t*
   P.stage_stride = h->stage_stride; P.omega_off = h->omega_off; P.delta_off = h->delta_off;
   P.desc_off = h->desc_off;
   const int grid = (int)(h->total_tiles < h->num_sms ? h->total_tiles : h->num_sms);
-  if (h->cfg.theta_dtype == GBMUF_F32) {
-    e = cudaFuncSetAttribute(peer_round_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, h->max_smem);
-    if (e == cudaSuccess) peer_round_kernel<float><<<grid, 32 + h->ncons, h->smem, st>>>(P);
-  } else {
-    e = cudaFuncSetAttribute(peer_round_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, h->max_smem);
-    if (e == cudaSuccess) peer_round_kernel<__nv_bfloat16><<<grid, 32 + h->ncons, h->smem, st>>>(P);
-  }
-  if (e == cudaSuccess) e = cudaGetLastError();
+  if (h->cfg.theta_dtype == GBMUF_F32)
+    peer_round_kernel<float><<<grid, 32 + h->ncons, h->smem, st>>>(P);
+  else
+    peer_round_kernel<__nv_bfloat16><<<grid, 32 + h->ncons, h->smem, st>>>(P);
+  e = cudaGetLastError();
+  h->work.note(st);
   if (e != cudaSuccess) return cuda_fail(nullptr, "launch of the peer round kernel", e);
   return GBMUF_OK;
 }
@@ -1430,7 +1676,8 @@ gbmuf_status gbmuf_peer_destroy(gbmuf_peer* h) {
   {
     DeviceGuard guard(h->cfg.device);
     if (guard.ok) {
-      if (cudaDeviceSynchronize() != cudaSuccess) rc = GBMUF_ERR_CUDA;
+      if (h->work.wait() != cudaSuccess) rc = GBMUF_ERR_CUDA;   // this worker's own rounds only
+      h->work.release();
       cudaFree(h->tables); cudaFree(h->d_status); cudaFree(h->d_theta_in[0]); cudaFree(h->d_theta_in[1]);
     } else {
       rc = GBMUF_ERR_CUDA;

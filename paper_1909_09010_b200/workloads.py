@@ -234,6 +234,19 @@ def theta0_torch(w: Workload, device, n: int | None = None):
     return t
 
 
+def replica_noise_torch(w: Workload, k: int, step: int, n: int, device):
+    """Standard-normal input noise [n] for worker k's local step `step`, drawn on `device` from a
+    torch generator seeded by (workload seed, k, step).  Used where each worker is a process of
+    its own and applies its local step with library tensor operations; a checker that wants the
+    same input calls this with the same arguments on the same kind of device."""
+    import torch
+    g = torch.Generator(device=device)
+    g.manual_seed((w.seed * 1_000_003 + k) * 1_000_003 + step)
+    t = torch.empty(n, dtype=torch.float32, device=device)
+    t.normal_(0.0, 1.0, generator=g)
+    return t
+
+
 # ------------------------------------------------------------------------------------------------
 # element-range shards: given the neighbour table every element is independent, so a column
 # range [c0, c1) of all K replicas can be processed on its own as long as components keep their

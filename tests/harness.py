@@ -177,3 +177,71 @@ def random_theta0(N, seed, dtype=0, sigma=0.1):
     g = np.random.Generator(np.random.PCG64(seed))
     x = (g.standard_normal(N, dtype=np.float32) * np.float32(sigma)).astype(np.float32)
     return oracle.f32_to_bf16(x) if dtype == 1 else x
+
+
+# ------------------------------------------------------------------------------------------------
+# one whole round of a large state, every element, checked slice by slice
+# ------------------------------------------------------------------------------------------------
+def check_round_every_element(case: Case, rnd, pre, post, mask=None, width=None, threads=None,
+                              what=""):
+    """Compares one synchronisation round over the WHOLE state with the oracle, bit for bit.
+
+    `pre` = (theta, omega, delta) device tensors as they were before the round, `post` the same
+    after it.  In `pre`, omega may be a 1-D tensor [N] that stands for K identical rows and delta
+    may be None for zeros (the state right after the initialisation line of Algorithm 1).  The
+    columns are cut into ranges of `width` (default: 2^26 replica-parameters per range); each range goes to the host, the oracle runs the round
+    on it alone (exact: with the neighbour table fixed every column is independent, and the draws
+    are keyed by the global component index), and the result must equal the same range of
+    `post`.  The block-start value the oracle stores is what the previous synchronisation left:
+    store(fl(omega + fl(eta * Delta))) of the pre-round values.  Ranges are checked by a few
+    threads (the oracle releases the interpreter while it computes)."""
+    import os
+    from concurrent.futures import ThreadPoolExecutor
+    K, N = case.K, case.N
+    th0, om0, de0 = pre
+    th1, om1, de1 = post
+    per = case.periods or [1] * case.m
+    due = [bool(x) for x in mask] if mask is not None else [rnd % h == 0 for h in per]
+    eta32 = np.float32(case.eta)
+
+    def host(t, a, b):
+        return to_numpy(t[:, a:b])
+
+    def one(rng):
+        a, b = rng
+        n = b - a
+        sh = workloads.shard_columns(case.offsets, a, b)
+        theta = np.ascontiguousarray(host(th0, a, b))
+        if om0.dim() == 1:
+            row = to_numpy(om0[a:b])
+            row = oracle.bf16_to_f32(row) if row.dtype == np.uint16 else row
+            omega = np.ascontiguousarray(np.broadcast_to(row.astype(np.float32), (K, n)))
+        else:
+            omega = np.ascontiguousarray(host(om0, a, b))
+        delta = np.zeros((K, n), dtype=np.float32) if de0 is None else np.ascontiguousarray(host(de0, a, b))
+        r32 = omega + eta32 * delta                       # two roundings, as the filter wrote it
+        rst = oracle.f32_to_bf16(r32) if case.dtype == 1 else r32
+        st = oracle.State(K, n, n, case.dtype, theta, omega, delta, np.ascontiguousarray(rst))
+        nbr = oracle.sample_neighbors(case.seed, rnd, K, sh.m, case.p, case.q, comp_base=sh.comp_base)
+        oracle.sync_round(st, sh.offsets, nbr, case.eta, case.zeta, mode=case.mode,
+                          sync=due[sh.comp_base:sh.comp_base + sh.m])
+        bad = []
+        for name, got, ref in (("theta", host(th1, a, b), st.theta), ("omega", host(om1, a, b), st.omega),
+                               ("delta", host(de1, a, b), st.delta)):
+            if case.mode == 1 and name != "theta":
+                continue
+            ne = got.view(np.uint8) != ref.view(np.uint8)
+            if ne.any():
+                bad.append(f"{what} {name} cols[{a},{b}): {int(ne.any(axis=0).sum() if ne.ndim == 2 else ne.sum())} "
+                           "columns not bit-equal")
+        return bad
+
+    width = width or max(1 << 12, ((1 << 26) // K) // 32 * 32)
+    ranges = [(a, min(N, a + width)) for a in range(0, N, width)]
+    threads = threads or max(1, min(6, (os.cpu_count() or 2) - 1))
+    problems = []
+    with ThreadPoolExecutor(max_workers=threads) as pool:
+        for bad in pool.map(one, ranges):
+            problems += bad
+    assert not problems, "; ".join(problems[:5])
+    return len(ranges)

@@ -9,8 +9,8 @@ import numpy as np
 import pytest
 import torch
 
-from paper_1909_09010_b200 import workloads
-from harness import Pair, case_of
+from paper_1909_09010_b200 import binding, workloads
+from harness import Pair, case_of, check_round_every_element, tdtype
 
 pytestmark = pytest.mark.gpu
 
@@ -40,6 +40,10 @@ def _restart_invariant(pr, eta):
 @pytest.mark.parametrize("name,over,tuning", [("wikitext103", {}, None), ("longrun", {}, None),
                                               ("sweep", dict(C=256, q=4, eta=0.5), None),
                                               ("sweep", dict(C=64, q=1, eta=0.9), None),
+                                              ("sweep", dict(C=4, q=2, eta=0.9), None),
+                                              ("sweep", dict(C=4, q=4, eta=0.5), None),
+                                              ("sweep", dict(C=16, q=2, eta=0.5), None),
+                                              ("sweep", dict(C=16, q=4, eta=0.9), None),
                                               ("wikitext103", {}, dict(flags=8))])
 def test_full_size_sampled_parity(name, over, tuning):
     w = workloads.get(name, **over)
@@ -70,3 +74,67 @@ def test_full_size_sampled_parity(name, over, tuning):
         assert not pr.theta[:, w.N:].any() and not pr.omega[:, w.N:].any()   # padding untouched
     finally:
         pr.close()
+
+
+# ------------------------------------------------------------------------------------------------
+# every element of a full-size launch
+# ------------------------------------------------------------------------------------------------
+def _full_round_check(w, second_round=True):
+    """Round 1 from the state the initialisation line leaves (plus seeded local steps), and, if
+    asked, a second round with some components idle from the state round 1 left (momentum and
+    global models no longer trivial): all K * N elements of theta, omega and Delta against the
+    oracle, in the launch configuration the bench times."""
+    dev = torch.device("cuda:0")
+    case = case_of(w)
+    K, N, ld = w.K, w.N, w.ld
+    theta0 = workloads.theta0_torch(w, dev).to(tdtype(w.dtype))
+    theta = torch.empty((K, ld), dtype=tdtype(w.dtype), device=dev)
+    omega = torch.empty((K, ld), dtype=torch.float32, device=dev)
+    delta = torch.empty((K, ld), dtype=torch.float32, device=dev)
+    g = binding.Gbmuf(theta, omega, delta, K=K, N=N, ld=ld, p=w.p, q=w.q, eta=w.eta, zeta=w.zeta,
+                      seed=w.seed, theta_dtype=w.dtype)
+    try:
+        g.set_partition(w.offsets)
+        info = g.launch_info()
+        assert info["grid"] == torch.cuda.get_device_properties(0).multi_processor_count
+        g.init(theta0)
+        g.local_perturb(1, w.lr, 10 * w.sigma, w.local_steps)       # the replicas drift apart: G != 0
+        pre_theta = theta.clone()
+        g.sync_round(1)
+        torch.cuda.synchronize()
+        assert g.device_status() == 0
+        n = check_round_every_element(case, 1, (pre_theta, theta0, None), (theta, omega, delta),
+                                      what=f"{w.name} round 1")
+        assert n >= K * N // (1 << 26)
+        if second_round:
+            g.local_perturb(2, w.lr, 10 * w.sigma, w.local_steps)
+            pre = (pre_theta.copy_(theta), omega.clone(), delta.clone())
+            mask = [i % 5 != 3 for i in range(w.m)]
+            g.sync_round(2, mask)
+            torch.cuda.synchronize()
+            assert g.device_status() == 0
+            check_round_every_element(case, 2, pre, (theta, omega, delta), mask=mask,
+                                      what=f"{w.name} round 2")
+    finally:
+        g.destroy()
+
+
+def test_every_element_of_the_headline_launch():
+    """wikitext103 (K = 16, 278.6 M columns, fp32): the launch the bench times, all 4.46 G
+    replica-parameters of two rounds."""
+    _full_round_check(workloads.get("wikitext103"))
+
+
+def test_every_element_of_a_long_run_round():
+    """The mixed-precision workload (bf16 theta, K = 16, 238.5 M columns, 64 components)."""
+    _full_round_check(workloads.get("longrun"), second_round=False)
+
+
+def test_every_element_of_a_ring_window_round():
+    """64 workers on the ring the paper's rule gives them (p = 5): the ring-window launch over
+    1.07 G replica-parameters."""
+    n = (1 << 24) + 5
+    cuts = tuple(int(x) // 4 * 4 for x in np.linspace(0, n, 17)[:-1]) + (n,)
+    w = workloads.get("profile64", offsets=cuts)
+    assert w.K * w.N >= 1 << 30
+    _full_round_check(w)

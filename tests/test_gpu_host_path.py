@@ -49,6 +49,38 @@ def test_host_round_matches_oracle(dtype, chunk, pinned, K, p, q):
         assert np.array_equal(got_t.view(np.uint8), st.theta.view(np.uint8)), "theta"
 
 
+@pytest.mark.parametrize("dtype,mode,row_copies", [(0, 0, False), (1, 0, True), (0, 1, True)])
+def test_host_handle_over_several_rounds(dtype, mode, row_copies):
+    """The handle form: chunk buffers, streams and chunk tables made once and used for four
+    rounds (masks changing from round to round), against the oracle after every round."""
+    K, p, q, eta, zeta, seed = 8, 2, 2, 0.875, 1.0, 5
+    offsets = (0, 1000, 1001, 4096, 9999, 20001, 50003)
+    N = offsets[-1]
+    ld = N + 5
+    st = oracle.init(random_theta0(N, seed=9, dtype=dtype), K, ld=ld, dtype=dtype)
+    oracle.local_perturb(st, seed, 0, 1.0, 0.05)
+
+    def host(a):
+        t = torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a).clone()
+        return (t.view(torch.bfloat16) if a.dtype == np.uint16 else t).pin_memory()
+
+    th, om, de = host(st.theta), host(st.omega), host(st.delta)
+    h = binding.GbmufHost(offsets, K=K, N=N, ld=ld, p=p, q=q, eta=eta, zeta=zeta, seed=seed,
+                          theta_dtype=dtype, mode=mode, chunk_cols=2048, row_copies=row_copies)
+    try:
+        masks = [None, [1, 0, 1, 1, 0, 1], [0, 0, 0, 0, 0, 0], [0, 1, 0, 0, 1, 0]]
+        for rnd, mask in enumerate(masks, start=1):
+            h.sync_round(th, om if mode == 0 else None, de if mode == 0 else None, rnd, mask)
+            nbr = oracle.sample_neighbors(seed, rnd, K, len(offsets) - 1, p, q)
+            oracle.sync_round(st, offsets, nbr, eta, zeta, mode=mode, sync=mask)
+            got_t = th.view(torch.int16).numpy().view(np.uint16) if dtype == 1 else th.numpy()
+            assert np.array_equal(got_t.view(np.uint8), st.theta.view(np.uint8)), f"theta, round {rnd}"
+            assert np.array_equal(om.numpy().view(np.uint32), st.omega.view(np.uint32)), f"omega, round {rnd}"
+            assert np.array_equal(de.numpy().view(np.uint32), st.delta.view(np.uint32)), f"delta, round {rnd}"
+    finally:
+        h.destroy()
+
+
 def test_host_round_argument_errors():
     K, N = 4, 1000
     th = torch.zeros((K, N))

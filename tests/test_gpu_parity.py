@@ -319,6 +319,55 @@ def test_rounds_replayed_from_a_cuda_graph():
         pr.close()
 
 
+def test_page_locked_mask_may_be_reused_at_once():
+    """A comp_mask in page-locked memory, overwritten as soon as gbmuf_sync_round returns while the
+    stream is still busy with earlier work: the round must use the mask as it was at the call."""
+    offsets = (0, 3000, 3001, 9000, 20000, 40001)
+    case = Case(K=8, offsets=offsets, p=2, q=2, seed=12)
+    pr = Pair(case, random_theta0(case.N, seed=4))
+    try:
+        pr.perturb(1, 0.1, 0.05)
+        mask_pin = torch.tensor([1, 0, 1, 0, 1], dtype=torch.uint8).pin_memory()
+        busy = torch.empty(1 << 28, device=pr.device)
+        for _ in range(20):
+            busy.add_(1.0)
+        pr.g.sync_round(1, mask_pin.numpy())
+        mask_pin.fill_(1)                                # the caller's array changes at once
+        for sh, st in zip(pr.shards, pr.states):
+            nbr = oracle.sample_neighbors(case.seed, 1, case.K, sh.m, case.p, case.q)
+            oracle.sync_round(st, sh.offsets, nbr, case.eta, case.zeta, sync=[1, 0, 1, 0, 1])
+        pr.compare("pinned mask")
+    finally:
+        pr.close()
+
+
+def test_mask_is_refused_inside_a_stream_capture():
+    w = workloads.get("tiny")
+    pr = Pair(case_of(w), workloads.theta0_numpy(w))
+    try:
+        pr.sync(1)
+        pr.compare("before capture")
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            graph.capture_begin()
+            with pytest.raises(binding.GbmufError) as e:
+                pr.g.sync_round(2, [1, 1, 0, 1], stream=side)
+            pr.g.sync_round(2, stream=side)               # without a mask the round is recorded
+            graph.capture_end()
+        assert e.value.status == binding.ERR_BAD_STATE
+        torch.cuda.current_stream().wait_stream(side)
+        graph.replay()
+        torch.cuda.synchronize()
+        for sh, st in zip(pr.shards, pr.states):
+            nbr = oracle.sample_neighbors(w.seed, 2, w.K, sh.m, w.p, w.q)
+            oracle.sync_round(st, sh.offsets, nbr, w.eta, w.zeta)
+        pr.compare("after replay")
+    finally:
+        pr.close()
+
+
 def test_random_shapes_property():
     """Random K, p, q, component edges (unaligned, tiny and large), eta, zeta, dtype, mode, and
     launch shapes of both variants of the fused kernel (several tiles per CTA included)."""
