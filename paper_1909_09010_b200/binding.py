@@ -331,7 +331,8 @@ class Gbmuf:
                                                 ctypes.byref(st)))
         return {"tiles": tiles.value, "grid": g.value, "block": b.value, "smem_bytes": s.value,
                 "tile_elems": t.value, "stages": st.value,
-                "variant": "tmem" if st.value == 0 else "tmem-window" if st.value < 0 else "smem"}
+                "variant": "tmem" if st.value == 0 else "tmem-window" if st.value < 0
+                else "smem-window" if st.value >= 1000 else "smem"}
 
     def last_error(self) -> str:
         return lib().gbmuf_last_error(self._h).decode()

@@ -11,6 +11,8 @@
 //   sync_fused_tmem.cuh  sync_fused_tmem_kernel: the same with the theta tile in tensor memory and
 //                        bulk stores (the default in gossip-BMUF mode); with many workers only a
 //                        window of rows along the ring is resident; device self-tests
+//   sync_ma_window.cuh   sync_ma_window_kernel: gossip-MA with many workers, a window of rows
+//                        along the ring in shared memory
 //   local_step.cuh       perturb_kernel (synthetic local steps), the Adagrad local step,
 //                        init_stream_kernel (theta^k <- theta_0, omega^k <- theta_0, Delta^k <- 0),
 //                        final_average_kernel (theta = (1/K) sum_k theta^k)
@@ -41,6 +43,7 @@
 #include "primitives.cuh"
 #include "sync_fused.cuh"
 #include "sync_fused_tmem.cuh"
+#include "sync_ma_window.cuh"
 #include "local_step.cuh"
 #include "peer.cuh"
 
@@ -63,6 +66,10 @@ struct Launch {
   // TMEM variant, which rows of a tile are resident: all K (win_rows = cell_rows = npos = K,
   // lead = K, pshift = 0) or a window along the ring plus the kept first p rows
   int win_rows, cell_rows, npos, lead, pshift, keep_lo;
+  // gossip-MA ring window in shared memory (sync_ma_window_kernel): ring slots (0 = not in use),
+  // offsets of the two kept-row sets and of the ring
+  int ma_ring;
+  uint32_t kept_off;
 };
 
 int host_candidates(int K, int p) {
@@ -194,6 +201,7 @@ cudaError_t ensure_kernel_attributes(int device, int max_smem) {
       (const void*)sync_fused_tmem_kernel<__nv_bfloat16, true, true>, (const void*)sync_fused_tmem_kernel<__nv_bfloat16, true, false>,
       (const void*)sync_fused_tmem_kernel<__nv_bfloat16, false, true>, (const void*)sync_fused_tmem_kernel<__nv_bfloat16, false, false>,
       (const void*)sync_fused_kernel<float>, (const void*)sync_fused_kernel<__nv_bfloat16>,
+      (const void*)sync_ma_window_kernel<float>, (const void*)sync_ma_window_kernel<__nv_bfloat16>,
       (const void*)init_stream_kernel<float>, (const void*)init_stream_kernel<__nv_bfloat16>,
       (const void*)adagrad_stream_kernel<float>, (const void*)adagrad_stream_kernel<__nv_bfloat16>,
       (const void*)peer_round_kernel<float>, (const void*)peer_round_kernel<__nv_bfloat16>};
@@ -212,7 +220,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 // Tensor map for boxes of K rows x BW columns over the [K][ld] theta array.
 gbmuf_status build_tensor_maps(gbmuf_ctx* ctx, const Launch& L) {
-  if (L.tmem_cols > 0) return GBMUF_OK;      // the tensor-memory variant stages rows by 1-D copies
+  if (L.tmem_cols > 0 || L.ma_ring > 0) return GBMUF_OK;   // these variants stage rows by 1-D copies
   static EncodeTiledFn encode = nullptr;
   if (!encode) {
     void* fn = nullptr;
@@ -251,6 +259,7 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
   L.flags = t.flags;
   L.tmem_cols = 0; L.meta_off = 0; L.meta_stride = 0;
   L.win_rows = 0; L.cell_rows = 0; L.npos = 0; L.lead = 0; L.pshift = 0; L.keep_lo = 0;
+  L.ma_ring = 0; L.kept_off = 0;
   const long long cap = ctx->max_smem < ctx->smem_per_sm - 1024 ? ctx->max_smem : ctx->smem_per_sm - 1024;
   // Variant: flags bit 3 forces the shared-memory theta tile, bit 1 forces the tensor-memory tile
   // (bit 2: with bulk stores); with neither, the tensor-memory tile with bulk stores is used
@@ -293,8 +302,8 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
   };
   if ((t.flags & 16) && (t.flags & 32))
     return fail(ctx, GBMUF_ERR_INVALID_ARG, "flags bits 4 and 5 (force / forbid the ring window) exclude each other");
-  if ((t.flags & 16) && !(win_possible && bmuf))
-    return fail(ctx, GBMUF_ERR_UNSUPPORTED, "the ring window needs gossip-BMUF mode and 2p + rows per load item < K");
+  if ((t.flags & 16) && bmuf && !win_possible)
+    return fail(ctx, GBMUF_ERR_UNSUPPORTED, "the ring window needs 2p + rows per load item < K");
   bool use_win = false;
   if (win_possible && !(t.flags & 32)) {
     if (t.flags & 16) use_win = true;
@@ -307,11 +316,11 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
   // shared-memory tile: consumer threads, theta stages, or a tile width it cannot have)
   const bool auto_tmem = !(t.flags & 8) && tmem_ok && t.ncons == 0 && t.stages == 0 &&
                          (t.T == 0 || fits_cols(t.T, cells));
-  const bool want_tmem = (t.flags & (2 | 16)) || auto_tmem;
-  if ((t.flags & (2 | 16)) && !tmem_ok)
+  const bool want_tmem = (t.flags & 2) || (bmuf && (t.flags & 16)) || auto_tmem;
+  if (((t.flags & 2) || (bmuf && (t.flags & 16))) && !tmem_ok)
     return fail(ctx, GBMUF_ERR_UNSUPPORTED, "the tensor-memory variant needs gossip-BMUF mode and resident rows that fit 512 columns (K <= 128, or a ring window)");
   if (want_tmem) {
-    const bool forced = (t.flags & (2 | 16)) != 0;
+    const bool forced = (t.flags & 2) != 0 || (bmuf && (t.flags & 16) != 0);
     const bool bulk = (t.flags & 2) ? (t.flags & 4) != 0 : true;
     // theta tile in tensor memory: cells * (T/512) * cw <= 512 columns; T a multiple of 512
     // default width: measured best with 16 replicas (fp32: 3584 x 4 slots; bf16: 3072 x 6 slots)
@@ -361,6 +370,54 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
     }
   }
   L.flags = t.flags & 1;
+  // gossip-MA with many workers: the ring window in shared memory (sync_ma_window_kernel).  Rows
+  // of 8, 6, 4, 2 KB; two sets of p kept rows; a ring of 2p + 1 live rows plus at least two (by
+  // preference four and more) rows of prefetch.  Taken when all K rows of a tile would be
+  // narrower than that (from 48 workers on), on request (flags bit 4), never with bit 5.
+  if (!bmuf && !(t.flags & (8 | 32)) && K >= 2 * p + 2 && t.ncons == 0 && t.stages == 0 &&
+      ((t.flags & 16) || K >= 48)) {
+    const int mv = 16 / esz;                                 // elements per 16 bytes
+    const long long meta_stride = ((long long)sizeof(TileDesc) + (long long)K * q * 4 + 127) / 128 * 128;
+    const long long fixed = (long long)kMwBarBytes + 2 * meta_stride;
+    auto ring_for_rows = [&](int T) {                        // ring slots that fit beside the kept rows
+      const long long rows = (cap - fixed) / ((long long)T * esz);
+      long long R = rows - 2LL * p;
+      if (R > kMaWinMaxRing) R = kMaWinMaxRing;
+      return (int)R;
+    };
+    int T = 0, R = 0;
+    if (t.T) {
+      T = t.T;
+      R = t.ring ? t.ring : ring_for_rows(T);
+    } else {
+      static const int kRowBytes[] = {8192, 6144, 4096, 2048};
+      for (int pass = 0; pass < 2 && !T; ++pass)             // first with 4+ rows of prefetch, then 2
+        for (int i = 0; i < 4 && !T; ++i) {
+          const int Tc = kRowBytes[i] / esz, Rc = t.ring ? t.ring : ring_for_rows(Tc);
+          if (Rc >= 2 * p + 1 + (pass == 0 ? 4 : 2)) { T = Tc; R = Rc; }
+        }
+    }
+    const bool shape_ok = T > 0 && T % (mv * 32) == 0 && T / mv <= 992 && R >= 2 * p + 3 && R <= kMaWinMaxRing &&
+                          fixed + (2LL * p + R) * T * esz <= cap;
+    if (!shape_ok && ((t.flags & 16) || t.T))
+      return fail(ctx, GBMUF_ERR_UNSUPPORTED, "gossip-MA ring window: tile_elems must be a multiple of 32 16-byte vectors, "
+                                              "at most 992 of them, with 2p kept rows and a ring of 2p + 3 .. 32 rows in shared memory");
+    if (shape_ok) {
+      L.T = T; L.BW = 256; L.stages = 1; L.ring = 0; L.ncons = T / mv;
+      L.flags = (t.flags & 1) | 16;
+      L.ma_ring = R;
+      L.meta_off = kMwBarBytes; L.meta_stride = (uint32_t)meta_stride;
+      L.kept_off = (uint32_t)fixed;
+      L.ring_off = (uint32_t)(fixed + 2LL * p * T * esz);
+      L.slot_stride = (uint32_t)(T * esz);
+      L.smem = (uint32_t)(L.ring_off + (long long)R * T * esz);
+      L.stage_stride = 0; L.nbr_off = 0; L.desc_off = 0;
+      *out = L;
+      return GBMUF_OK;
+    }
+  } else if ((t.flags & 16) && !bmuf) {
+    return fail(ctx, GBMUF_ERR_UNSUPPORTED, "the gossip-MA ring window needs K >= 2p + 2 and no consumer_threads / theta_stages setting");
+  }
   auto stage_bytes = [&](int T, Launch* l) {
     long long at = ((long long)K * T * esz + 15) / 16 * 16;
     if (l) l->nbr_off = (uint32_t)at;
@@ -463,6 +520,18 @@ gbmuf_status launch_round(gbmuf_ctx* ctx, const gbmuf_config& cfg, const Launch&
   const int grid = (int)(total < ctx->num_sms ? total : ctx->num_sms);   // one persistent CTA per SM
   SyncParams P;
   fill_sync_params(cfg, L, theta, omega, delta, ld, m, off, prefix, nbr, status, &P);
+  // Programmatic dependent launch: the kernel may start while the round set-up kernel before it
+  // in the stream still runs; it waits for that kernel (grid_dependency_wait) before it reads the
+  // tables.
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3((unsigned)grid, 1, 1);
+  lc.dynamicSmemBytes = L.smem;
+  lc.stream = st;
+  lc.attrs = attr;
+  lc.numAttrs = 1;
   cudaError_t e;
   if (L.tmem_cols > 0) {
     TmemParams Q;
@@ -481,12 +550,26 @@ gbmuf_status launch_round(gbmuf_ctx* ctx, const gbmuf_config& cfg, const Launch&
     else
       kern = bulk ? (win ? sync_fused_tmem_kernel<float, true, true> : sync_fused_tmem_kernel<float, true, false>)
                   : (win ? sync_fused_tmem_kernel<float, false, true> : sync_fused_tmem_kernel<float, false, false>);
-    kern<<<grid, 544, L.smem, st>>>(Q);
+    lc.blockDim = dim3(544, 1, 1);
+    e = cudaLaunchKernelEx(&lc, kern, Q);
+  } else if (L.ma_ring > 0) {
+    MaWinParams M;
+    M.theta = theta; M.off = off; M.tile_prefix = prefix; M.nbr = nbr; M.status = status;
+    M.ld = ld; M.K = cfg.K; M.m = m; M.q = cfg.q; M.p = cfg.p;
+    M.qp1 = P.qp1; M.inv_qp1 = P.inv_qp1; M.inv_exact = P.inv_exact;
+    M.T = L.T; M.R = L.ma_ring; M.ncons = L.ncons; M.row_bytes = L.slot_stride;
+    M.meta_off = L.meta_off; M.meta_stride = L.meta_stride; M.kept_off = L.kept_off; M.ring_off = L.ring_off;
+    lc.blockDim = dim3((unsigned)(32 + L.ncons), 1, 1);
+    if (cfg.theta_dtype == GBMUF_F32) e = cudaLaunchKernelEx(&lc, sync_ma_window_kernel<float>, M);
+    else e = cudaLaunchKernelEx(&lc, sync_ma_window_kernel<__nv_bfloat16>, M);
   } else if (cfg.theta_dtype == GBMUF_F32) {
-    sync_fused_kernel<float><<<grid, 32 + L.ncons, L.smem, st>>>(P, ctx->map_theta);
+    lc.blockDim = dim3((unsigned)(32 + L.ncons), 1, 1);
+    e = cudaLaunchKernelEx(&lc, sync_fused_kernel<float>, P, ctx->map_theta);
   } else {
-    sync_fused_kernel<__nv_bfloat16><<<grid, 32 + L.ncons, L.smem, st>>>(P, ctx->map_theta);
+    lc.blockDim = dim3((unsigned)(32 + L.ncons), 1, 1);
+    e = cudaLaunchKernelEx(&lc, sync_fused_kernel<__nv_bfloat16>, P, ctx->map_theta);
   }
+  if (e != cudaSuccess) return cuda_fail(ctx, "launch of the fused round kernel", e);
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, "launch of the fused round kernel", e);
   return GBMUF_OK;
@@ -686,7 +769,8 @@ gbmuf_status gbmuf_get_launch_info(gbmuf_ctx* ctx, int64_t* tiles, int32_t* grid
   if (smem) *smem = (int32_t)ctx->launch.smem;
   if (tile_elems) *tile_elems = ctx->launch.T;
   if (stages)
-    *stages = ctx->launch.tmem_cols == 0 ? ctx->launch.stages
+    *stages = ctx->launch.ma_ring > 0 ? 1000 + ctx->launch.ma_ring
+              : ctx->launch.tmem_cols == 0 ? ctx->launch.stages
               : ctx->launch.pshift > 0 || ctx->launch.cell_rows < ctx->cfg.K ? -ctx->launch.cell_rows : 0;
   return GBMUF_OK;
 }

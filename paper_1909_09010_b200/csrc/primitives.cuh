@@ -37,6 +37,18 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
   return t;
 }
+// Programmatic dependent launch.  The fused round kernel is launched with the "programmatic
+// stream serialization" attribute: it may start while the kernel before it in the stream (the
+// round set-up kernel) is still running, so that its prologue -- barrier initialisation, the
+// tensor-memory allocation -- overlaps that kernel.  grid_dependency_wait() returns once the
+// preceding kernel has completed and its writes are visible; nothing that kernel writes (the
+// neighbour table, the work-list) and nothing the kernels before it wrote is read earlier.
+// (The set-up kernel says "griddepcontrol.launch_dependents" at its start.)  Launched without
+// the attribute, the instruction does nothing.
+__device__ __forceinline__ void grid_dependency_wait() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // two seconds
 // Wait for the phase with the given parity to complete.  Bounded in wall-clock time: after
 // kWaitLimitNs it records GBMUF_ERR_TIMEOUT in the device status word and returns false; the

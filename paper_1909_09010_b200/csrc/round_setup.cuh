@@ -45,6 +45,9 @@ __device__ __forceinline__ int tiles_of_component(int64_t lo, int64_t hi, int T)
 }
 
 __global__ void __launch_bounds__(256) round_setup_kernel(SetupParams P) {
+  // the round kernel that follows may begin its prologue now; it waits for this grid to finish
+  // before it reads the tables written below
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (g < (int64_t)P.K * P.m && P.q > 0) {
     const int i = (int)(g / P.K), k = (int)(g % P.K);

@@ -123,10 +123,8 @@ sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_th
   const uint32_t bars = smem_u32(smem);
   unsigned char* stage0 = smem + kBarBytes;
   unsigned char* ring0 = smem + P.ring_off;
-  const int total = P.tile_prefix[P.m];
   const int S = P.stages, R = P.ring;
   const bool bmuf = P.mode == GBMUF_MODE_BMUF;
-  const int my_tiles = (int)blockIdx.x < total ? (total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < S; ++s) {
@@ -142,6 +140,10 @@ sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_th
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   __syncthreads();
+  // everything above overlapped the round set-up kernel; its tables are read from here on
+  grid_dependency_wait();
+  const int total = P.tile_prefix[P.m];
+  const int my_tiles = (int)blockIdx.x < total ? (total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
 
   if (threadIdx.x < 32) {
     // ------------------------------------------------------------------ producer warp

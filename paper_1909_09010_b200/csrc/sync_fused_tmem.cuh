@@ -95,6 +95,25 @@ template <> struct TmemCell<float> {
         : "memory");
     x[0] = __uint_as_float(a); x[1] = __uint_as_float(b); x[2] = __uint_as_float(c); x[3] = __uint_as_float(d);
   }
+  // four cells with one wait (used when a worker has many neighbours: the round trips overlap)
+  static __device__ __forceinline__ void fetch4(uint32_t t0, uint32_t t1, uint32_t t2, uint32_t t3,
+                                                float (&x)[4][4]) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%16];\n\t"
+        "tcgen05.ld.sync.aligned.32x32b.x4.b32 {%4, %5, %6, %7}, [%17];\n\t"
+        "tcgen05.ld.sync.aligned.32x32b.x4.b32 {%8, %9, %10, %11}, [%18];\n\t"
+        "tcgen05.ld.sync.aligned.32x32b.x4.b32 {%12, %13, %14, %15}, [%19];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(t0), "r"(t1), "r"(t2), "r"(t3)
+        : "memory");
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) x[i][c] = __uint_as_float(r[i * 4 + c]);
+  }
 };
 template <> struct TmemCell<__nv_bfloat16> {
   static constexpr int COLS = 2;
@@ -114,7 +133,29 @@ template <> struct TmemCell<__nv_bfloat16> {
     x[0] = __uint_as_float(a << 16); x[1] = __uint_as_float(a & 0xFFFF0000u);
     x[2] = __uint_as_float(b << 16); x[3] = __uint_as_float(b & 0xFFFF0000u);
   }
+  static __device__ __forceinline__ void fetch4(uint32_t t0, uint32_t t1, uint32_t t2, uint32_t t3,
+                                                float (&x)[4][4]) {
+    uint32_t r[8];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x2.b32 {%0, %1}, [%8];\n\t"
+        "tcgen05.ld.sync.aligned.32x32b.x2.b32 {%2, %3}, [%9];\n\t"
+        "tcgen05.ld.sync.aligned.32x32b.x2.b32 {%4, %5}, [%10];\n\t"
+        "tcgen05.ld.sync.aligned.32x32b.x2.b32 {%6, %7}, [%11];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+        : "r"(t0), "r"(t1), "r"(t2), "r"(t3)
+        : "memory");
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      x[i][0] = __uint_as_float(r[2 * i] << 16); x[i][1] = __uint_as_float(r[2 * i] & 0xFFFF0000u);
+      x[i][2] = __uint_as_float(r[2 * i + 1] << 16); x[i][3] = __uint_as_float(r[2 * i + 1] & 0xFFFF0000u);
+    }
+  }
 };
+
+// From this many neighbours on, their cells are fetched four per wait.  (With 2 and 4 neighbours
+// several loads per wait measured slower; with a chain of 7 and more round trips they pay.)
+constexpr int kGatherBatchFrom = 8;
 
 // Sum of a worker's own cell (cell row `own`) and its q drawn neighbours' cells (cell rows nb[])
 // of element group `cell0` (the TMEM address of cell row 0), own first, then draw order, each
@@ -123,7 +164,20 @@ template <typename TH>
 __device__ __forceinline__ void tmem_gather(uint32_t cell0, int own, const int* nb, int q, float (&a)[4]) {
   constexpr int CW = TmemCell<TH>::COLS;
   TmemCell<TH>::fetch(cell0 + (uint32_t)(own * CW), a);
-  for (int j = 0; j < q; ++j) {
+  int j = 0;
+  if (q >= kGatherBatchFrom) {
+    // many neighbours: four cells per wait; the additions keep the draw order
+    for (; j + 4 <= q; j += 4) {
+      float t[4][4];
+      TmemCell<TH>::fetch4(cell0 + (uint32_t)(nb[j] * CW), cell0 + (uint32_t)(nb[j + 1] * CW),
+                           cell0 + (uint32_t)(nb[j + 2] * CW), cell0 + (uint32_t)(nb[j + 3] * CW), t);
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int x = 0; x < 4; ++x) a[x] = __fadd_rn(a[x], t[i][x]);
+    }
+  }
+  for (; j < q; ++j) {
     float t[4];
     TmemCell<TH>::fetch(cell0 + (uint32_t)(nb[j] * CW), t);
 #pragma unroll
@@ -156,10 +210,8 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
   unsigned char* meta0 = smem + P.meta_off;
   TH* const theta = reinterpret_cast<TH*>(P.theta);
   const TH* const theta_in = reinterpret_cast<const TH*>(P.theta_in);
-  const int total = P.tile_prefix[P.m];
   const int R = P.ring, K = P.K, q = P.q, T = P.T;
   const int W = WIN ? P.W : K, wtot = WIN ? P.wtot : K, npos = WIN ? P.npos : K, pshift = WIN ? P.pshift : 0;
-  const int my_tiles = (int)blockIdx.x < total ? (total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
   // Items of a tile, in the order both sides generate them: with `s` positions requested and `k`
   // workers put out, the next item is a load item (positions s .. s + IN_ROWS - 1) while
   // s < npos and s <= k + lead, else worker k's output item.
@@ -183,6 +235,10 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
+  // everything above overlapped the round set-up kernel; its tables are read from here on
+  grid_dependency_wait();
+  const int total = P.tile_prefix[P.m];
+  const int my_tiles = (int)blockIdx.x < total ? (total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ producer warp

@@ -591,6 +591,31 @@ def test_which_rows_are_resident_follows_the_ring(K, p, q, dtype, expect):
         g.destroy()
 
 
+@pytest.mark.parametrize("K,p,q,dtype,tuning,expect", [
+    (64, 5, 3, 0, None, "smem-window"), (64, 5, 3, 1, None, "smem-window"), (130, 6, 2, 1, None, "smem-window"),
+    (256, 7, 2, 0, None, "smem-window"), (48, 3, 6, 0, None, "smem-window"), (200, 32, 64, 0, None, "smem"),
+    (9, 2, 4, 0, dict(flags=16), "smem-window"), (12, 1, 2, 1, dict(flags=16, tile_elems=512), "smem-window"),
+    (6, 2, 3, 0, dict(flags=16, tile_elems=128), "smem-window"), (64, 5, 10, 0, dict(tile_elems=256), "smem-window"),
+    (64, 5, 3, 0, dict(flags=32), "smem"), (20, 0, 0, 0, dict(flags=16), "smem-window")])
+def test_gossip_ma_ring_window(K, p, q, dtype, tuning, expect):
+    """gossip-MA with many workers streams a window of rows along the ring through shared memory
+    (from 48 workers on, or on request): several tiles per CTA, ragged component edges, kept first
+    rows, last rows read twice, both theta types, and the settings where it is not taken."""
+    offsets = (0, 5, 4099, 4100, 30_001, 70_003)
+    case = Case(K=K, offsets=offsets, p=p, q=q, eta=0.9, zeta=1.0, dtype=dtype, seed=K + q,
+                mode=binding.MODE_MA)
+    pr = Pair(case, random_theta0(case.N, seed=K, dtype=dtype), tuning=tuning)
+    try:
+        assert pr.g.launch_info()["variant"] == expect
+        for r in (1, 2, 3):
+            pr.perturb(step=r, lr=0.1, sigma=5e-2)
+            mask = None if r != 2 else [1, 0, 1, 1, 0]
+            pr.sync(r, mask)
+            pr.compare(f"round {r}")
+    finally:
+        pr.close()
+
+
 def test_averaging_division_equals_the_ieee_division_for_every_dividend():
     """The kernels divide the gossip sum by q+1 through a multiply and a residual correction;
     for every divisor they can meet (q+1 <= 65) and some beyond, all 2^32 dividends -- zeros,
