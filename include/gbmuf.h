@@ -202,18 +202,24 @@ gbmuf_status gbmuf_selftest_divide(gbmuf_ctx* ctx, int32_t divisor, void* stream
  * streams through.  (b) theta tile in shared memory: everything else, and whenever
  * consumer_threads or theta_stages is given or flags bit 3 is set; consumer_threads: multiple of
  * 32 in 32..992 (one more warp issues the copies); tile_elems: a multiple of 8 and, above 256, of
- * 256; theta_stages: 1..4; ring_slots: 2..8 rows of omega/Delta in flight.  flags: bit 0 =
- * 256-byte L2 promotion for the theta loads of (b); bit 1 = force (a), bit 2 (with bit 1) = with
- * bulk stores (without: stores from registers); bit 3 = force (b); bit 4 = force the ring window
- * of (a), bit 5 = never use it, bit 6 = window with every row read once.  All choices give the
- * same bits.
+ * 256; theta_stages: 1..4; ring_slots: 2..8 rows of omega/Delta in flight.  (c) On request
+ * (flags bit 4; by itself only for fp32 theta with 192 or more workers) and with K >= 2p + 2,
+ * gossip-MA streams a window of rows along the ring
+ * through shared memory instead of holding all K rows of a tile: rows 0 .. p-1 are kept (two sets,
+ * for alternate tiles), the other rows pass through a ring of 2p + 6 .. 64 row slots, the last p
+ * rows are read twice; tile_elems (a row slot) must be a multiple of 128 for fp32 theta, 256 for
+ * bf16, at most 512 16-byte vectors.  flags: bit 0 = 256-byte L2 promotion for the theta loads of
+ * (b); bit 1 = force (a), bit 2 (with bit 1) = with bulk stores (without: stores from registers);
+ * bit 3 = force (b); bit 4 = force the ring window of (a) / of gossip-MA, bit 5 = never use it,
+ * bit 6 = window of (a) with every row read once.  All choices give the same bits.
  * Errors: INVALID_ARG, UNSUPPORTED (does not fit, or (a) forced where it does not apply). */
 gbmuf_status gbmuf_set_tuning(gbmuf_ctx* ctx, int32_t consumer_threads, int32_t tile_elems,
                               int32_t theta_stages, int32_t ring_slots, int32_t flags);
 
 /* What the next full round would launch: tiles (work items), grid and block size, dynamic shared
  * memory in bytes, elements per tile, theta stages in shared memory (0 = the theta tile is kept in
- * tensor memory, all K rows; -r = in tensor memory as a ring window, r resident rows).  Any out
+ * tensor memory, all K rows; -r = in tensor memory as a ring window, r resident rows; 1000 + r =
+ * gossip-MA ring window in shared memory with r ring slots).  Any out
  * pointer may be NULL.  Requires set_partition. */
 gbmuf_status gbmuf_get_launch_info(gbmuf_ctx* ctx, int64_t* tiles, int32_t* grid, int32_t* block,
                                    int32_t* smem_bytes, int32_t* tile_elems, int32_t* stages);

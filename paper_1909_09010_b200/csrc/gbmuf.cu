@@ -201,7 +201,7 @@ cudaError_t ensure_kernel_attributes(int device, int max_smem) {
       (const void*)sync_fused_tmem_kernel<__nv_bfloat16, true, true>, (const void*)sync_fused_tmem_kernel<__nv_bfloat16, true, false>,
       (const void*)sync_fused_tmem_kernel<__nv_bfloat16, false, true>, (const void*)sync_fused_tmem_kernel<__nv_bfloat16, false, false>,
       (const void*)sync_fused_kernel<float>, (const void*)sync_fused_kernel<__nv_bfloat16>,
-      (const void*)sync_ma_window_kernel<float>, (const void*)sync_ma_window_kernel<__nv_bfloat16>,
+      (const void*)sync_ma_window_kernel<float, 1>, (const void*)sync_ma_window_kernel<__nv_bfloat16, 1>,
       (const void*)init_stream_kernel<float>, (const void*)init_stream_kernel<__nv_bfloat16>,
       (const void*)adagrad_stream_kernel<float>, (const void*)adagrad_stream_kernel<__nv_bfloat16>,
       (const void*)peer_round_kernel<float>, (const void*)peer_round_kernel<__nv_bfloat16>};
@@ -293,7 +293,9 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
                           window_shape(cells_once, nullptr) > 0);
   const int win_cells = keep_both ? cells_once : cells_twice;
   const bool win_possible = win_w < K;
-  const int T_default = esz == 4 ? 3584 : 3072;          // measured best with 16 replicas
+  // measured with 16 replicas: fp32 3584 x 4 slots; bf16 4096 x 4 slots (3072 x 6 is as fast when
+  // rounds are far apart but 4 % slower when they run back to back under the power cap)
+  const int T_default = esz == 4 ? 3584 : 4096;
   auto fits_cols = [&](int T, int rows) { return T >= 512 && T % 512 == 0 && (T / 512) * rows * cw <= 512; };
   auto widest = [&](int rows) {                          // widest tile up to the default, 0 = none
     int T = T_default;
@@ -323,7 +325,6 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
     const bool forced = (t.flags & 2) != 0 || (bmuf && (t.flags & 16) != 0);
     const bool bulk = (t.flags & 2) ? (t.flags & 4) != 0 : true;
     // theta tile in tensor memory: cells * (T/512) * cw <= 512 columns; T a multiple of 512
-    // default width: measured best with 16 replicas (fp32: 3584 x 4 slots; bf16: 3072 x 6 slots)
     int T = t.T ? t.T : widest(cells), ring_pref = 0;
     if (use_win && !t.T && bulk) {
       const int Tw = window_shape(cells, &ring_pref);
@@ -371,11 +372,13 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
   }
   L.flags = t.flags & 1;
   // gossip-MA with many workers: the ring window in shared memory (sync_ma_window_kernel).  Rows
-  // of 8, 6, 4, 2 KB; two sets of p kept rows; a ring of 2p + 1 live rows plus at least two (by
-  // preference four and more) rows of prefetch.  Taken when all K rows of a tile would be
-  // narrower than that (from 48 workers on), on request (flags bit 4), never with bit 5.
+  // of 8, 6, 4, 2 KB; two sets of p kept rows; a ring of 2p + 4 live rows (four workers are computed
+  // at a time) plus rows in flight ahead of them.  Taken for fp32 theta from 192 workers on (the
+  // only place where it measured faster than all K rows of a narrow tile: 3.3 against 2.6 TB/s
+  // at K = 256; its consumers are bound by instruction latency), on request (flags bit 4),
+  // never with bit 5.
   if (!bmuf && !(t.flags & (8 | 32)) && K >= 2 * p + 2 && t.ncons == 0 && t.stages == 0 &&
-      ((t.flags & 16) || K >= 48)) {
+      ((t.flags & 16) || (K >= 192 && esz == 4))) {
     const int mv = 16 / esz;                                 // elements per 16 bytes
     const long long meta_stride = ((long long)sizeof(TileDesc) + (long long)K * q * 4 + 127) / 128 * 128;
     const long long fixed = (long long)kMwBarBytes + 2 * meta_stride;
@@ -390,20 +393,22 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
       T = t.T;
       R = t.ring ? t.ring : ring_for_rows(T);
     } else {
+      // The widest row whose ring still has two slots beyond the live ones: the round's time
+      // turned out proportional to the number of rows, not to what is in flight (measured with
+      // 64 workers: 8 KB rows with 4 rows ahead 4.3 TB/s, 4 KB rows with 31 ahead 2.5 TB/s).
       static const int kRowBytes[] = {8192, 6144, 4096, 2048};
-      for (int pass = 0; pass < 2 && !T; ++pass)             // first with 4+ rows of prefetch, then 2
-        for (int i = 0; i < 4 && !T; ++i) {
-          const int Tc = kRowBytes[i] / esz, Rc = t.ring ? t.ring : ring_for_rows(Tc);
-          if (Rc >= 2 * p + 1 + (pass == 0 ? 4 : 2)) { T = Tc; R = Rc; }
-        }
+      for (int i = 0; i < 4 && !T; ++i) {
+        const int Tc = kRowBytes[i] / esz, Rc = t.ring ? t.ring : ring_for_rows(Tc);
+        if (Rc >= 2 * p + kMwUnroll + 2) { T = Tc; R = Rc; }
+      }
     }
-    const bool shape_ok = T > 0 && T % (mv * 32) == 0 && T / mv <= 992 && R >= 2 * p + 3 && R <= kMaWinMaxRing &&
+    const bool shape_ok = T > 0 && T % (mv * 32) == 0 && T / mv <= 512 && R >= 2 * p + kMwUnroll + 2 && R <= kMaWinMaxRing &&
                           fixed + (2LL * p + R) * T * esz <= cap;
     if (!shape_ok && ((t.flags & 16) || t.T))
       return fail(ctx, GBMUF_ERR_UNSUPPORTED, "gossip-MA ring window: tile_elems must be a multiple of 32 16-byte vectors, "
-                                              "at most 992 of them, with 2p kept rows and a ring of 2p + 3 .. 32 rows in shared memory");
+                                              "at most 512 of them, with 2p kept rows and a ring of 2p + 6 .. 64 rows in shared memory");
     if (shape_ok) {
-      L.T = T; L.BW = 256; L.stages = 1; L.ring = 0; L.ncons = T / mv;
+      L.T = T; L.BW = 256; L.stages = 1; L.ring = 0; L.ncons = T / mv;   // one 16-byte piece per thread and row
       L.flags = (t.flags & 1) | 16;
       L.ma_ring = R;
       L.meta_off = kMwBarBytes; L.meta_stride = (uint32_t)meta_stride;
@@ -560,8 +565,8 @@ gbmuf_status launch_round(gbmuf_ctx* ctx, const gbmuf_config& cfg, const Launch&
     M.T = L.T; M.R = L.ma_ring; M.ncons = L.ncons; M.row_bytes = L.slot_stride;
     M.meta_off = L.meta_off; M.meta_stride = L.meta_stride; M.kept_off = L.kept_off; M.ring_off = L.ring_off;
     lc.blockDim = dim3((unsigned)(32 + L.ncons), 1, 1);
-    if (cfg.theta_dtype == GBMUF_F32) e = cudaLaunchKernelEx(&lc, sync_ma_window_kernel<float>, M);
-    else e = cudaLaunchKernelEx(&lc, sync_ma_window_kernel<__nv_bfloat16>, M);
+    if (cfg.theta_dtype == GBMUF_F32) e = cudaLaunchKernelEx(&lc, sync_ma_window_kernel<float, 1>, M);
+    else e = cudaLaunchKernelEx(&lc, sync_ma_window_kernel<__nv_bfloat16, 1>, M);
   } else if (cfg.theta_dtype == GBMUF_F32) {
     lc.blockDim = dim3((unsigned)(32 + L.ncons), 1, 1);
     e = cudaLaunchKernelEx(&lc, sync_fused_kernel<float>, P, ctx->map_theta);

@@ -95,6 +95,19 @@ template <> struct TmemCell<float> {
         : "memory");
     x[0] = __uint_as_float(a); x[1] = __uint_as_float(b); x[2] = __uint_as_float(c); x[3] = __uint_as_float(d);
   }
+  // the same cell row of two element groups with one wait
+  static __device__ __forceinline__ void fetch2(uint32_t t0, uint32_t t1, float (&x)[4], float (&y)[4]) {
+    uint32_t r[8];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%8];\n\t"
+        "tcgen05.ld.sync.aligned.32x32b.x4.b32 {%4, %5, %6, %7}, [%9];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+        : "r"(t0), "r"(t1)
+        : "memory");
+#pragma unroll
+    for (int c = 0; c < 4; ++c) { x[c] = __uint_as_float(r[c]); y[c] = __uint_as_float(r[4 + c]); }
+  }
   // four cells with one wait (used when a worker has many neighbours: the round trips overlap)
   static __device__ __forceinline__ void fetch4(uint32_t t0, uint32_t t1, uint32_t t2, uint32_t t3,
                                                 float (&x)[4][4]) {
@@ -132,6 +145,20 @@ template <> struct TmemCell<__nv_bfloat16> {
         : "memory");
     x[0] = __uint_as_float(a << 16); x[1] = __uint_as_float(a & 0xFFFF0000u);
     x[2] = __uint_as_float(b << 16); x[3] = __uint_as_float(b & 0xFFFF0000u);
+  }
+  static __device__ __forceinline__ void fetch2(uint32_t t0, uint32_t t1, float (&x)[4], float (&y)[4]) {
+    uint32_t a, b, c, d;
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x2.b32 {%0, %1}, [%4];\n\t"
+        "tcgen05.ld.sync.aligned.32x32b.x2.b32 {%2, %3}, [%5];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(a), "=r"(b), "=r"(c), "=r"(d)
+        : "r"(t0), "r"(t1)
+        : "memory");
+    x[0] = __uint_as_float(a << 16); x[1] = __uint_as_float(a & 0xFFFF0000u);
+    x[2] = __uint_as_float(b << 16); x[3] = __uint_as_float(b & 0xFFFF0000u);
+    y[0] = __uint_as_float(c << 16); y[1] = __uint_as_float(c & 0xFFFF0000u);
+    y[2] = __uint_as_float(d << 16); y[3] = __uint_as_float(d & 0xFFFF0000u);
   }
   static __device__ __forceinline__ void fetch4(uint32_t t0, uint32_t t1, uint32_t t2, uint32_t t3,
                                                 float (&x)[4][4]) {
@@ -185,6 +212,25 @@ __device__ __forceinline__ void tmem_gather(uint32_t cell0, int own, const int* 
   }
 }
 
+// The same sums for two element groups of the thread at once (cell row 0 at cellA and cellB): one
+// wait per pair of loads, so the two groups' tensor-memory round trips overlap.
+template <typename TH>
+__device__ __forceinline__ void tmem_gather2(uint32_t cellA, uint32_t cellB, int own, const int* nb, int q,
+                                             float (&a)[4], float (&b)[4]) {
+  constexpr int CW = TmemCell<TH>::COLS;
+  TmemCell<TH>::fetch2(cellA + (uint32_t)(own * CW), cellB + (uint32_t)(own * CW), a, b);
+  for (int j = 0; j < q; ++j) {
+    float t[4], u[4];
+    const uint32_t o = (uint32_t)(nb[j] * CW);
+    TmemCell<TH>::fetch2(cellA + o, cellB + o, t, u);
+#pragma unroll
+    for (int x = 0; x < 4; ++x) { a[x] = __fadd_rn(a[x], t[x]); b[x] = __fadd_rn(b[x], u[x]); }
+  }
+}
+// A thread's element groups are taken two at a time when the worker has few neighbours (with
+// many, the four-cells-per-wait path of tmem_gather already overlaps the round trips).
+constexpr bool kPairGroups = true;
+
 // What the producer must know to send a finished slot out: the staged range starts at e0, whole
 // 16-byte pieces of the rows cover [sb, se); k < 0: a load item, nothing to send.
 struct SlotInfo { long long e0, sb, se; int k; int pad; };
@@ -220,7 +266,7 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
   if (threadIdx.x == 0) {
     for (int r = 0; r < R; ++r) {
       mbar_init(bars + 8 * r, 1);
-      mbar_init(bars + 64 + 8 * r, 512);                 // every consumer thread arrives
+      mbar_init(bars + 64 + 8 * r, 16);                  // every consumer warp arrives (through lane 0)
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -433,13 +479,12 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
           float* row0 = reinterpret_cast<float*>(sbase);
           float* row1 = row0 + T;
           TH* row2 = reinterpret_cast<TH*>(row1 + T);      // BULK: the new theta
-          for (int g = sub; g < ngroups; g += 4) {
+          // one element group of this worker: average, filter, outputs (into the slot or to memory)
+          auto finish_group = [&](int g, float (&a)[4]) {
             const int col = (g * 128 + quarter * 32 + lane) * 4;
             const long long e = e0 + col;
-            float a[4], t[4];
-            __syncwarp();                          // lanes that left the last group early rejoin
-            tmem_gather<TH>(tlane + (uint32_t)(g * wtot * CW), own, snb + k * q, q, a);
-            if (e >= hi || e + 4 <= lo) continue;
+            if (e >= hi || e + 4 <= lo) return;
+            float t[4];
             average_divide(a, P.qp1, P.inv_qp1, P.inv_exact);
             const float4 Wv = *reinterpret_cast<const float4*>(row0 + col);
             const float4 Dv = *reinterpret_cast<const float4*>(row1 + col);
@@ -464,10 +509,27 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
                 }
               }
             }
+          };
+          const bool pairs = kPairGroups && q < kGatherBatchFrom;
+          for (int g = sub; g < ngroups; g += pairs ? 8 : 4) {
+            float a[4], b[4];
+            __syncwarp();                          // lanes that left the last group early rejoin
+            if (pairs && g + 4 < ngroups) {
+              tmem_gather2<TH>(tlane + (uint32_t)(g * wtot * CW), tlane + (uint32_t)((g + 4) * wtot * CW), own,
+                               snb + k * q, q, a, b);
+              finish_group(g, a);
+              finish_group(g + 4, b);
+            } else {
+              tmem_gather<TH>(tlane + (uint32_t)(g * wtot * CW), own, snb + k * q, q, a);
+              finish_group(g, a);
+            }
           }
         }
+        // every thread makes its own writes to the slot visible to the copy engine; then the warp
+        // arrives once (16 arrivals per item instead of 512 on one barrier)
         if (BULK && !is_load) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        mbar_arrive(bars + 64 + 8 * slot);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bars + 64 + 8 * slot);
         if (is_load) s += IN_ROWS; else ++k;
       }
     }

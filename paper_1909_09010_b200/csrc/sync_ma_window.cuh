@@ -47,22 +47,43 @@ struct MaWinParams {
   int K, m, q, p;
   float qp1, inv_qp1;
   int inv_exact;
-  int T, R, ncons;         // elements per row slot, ring slots, consumer threads (T / elements per 16 B)
+  int T, R, ncons;         // elements per row slot, ring slots, consumer threads: T / (V * elements per 16 B)
   uint32_t row_bytes;      // T * element size
   uint32_t meta_off, meta_stride;   // two entries: [TileDesc | codes K*q ints]
   uint32_t kept_off;       // 2 sets of p row slots
   uint32_t ring_off;       // R row slots
 };
 
-constexpr int kMaWinMaxRing = 32;
-// barrier block: ring full [0, 256), ring empty [256, 512), kept full [512, 528), kept empty [528, 544)
-constexpr uint32_t kMwRingFull = 0, kMwRingEmpty = 256, kMwKeptFull = 512, kMwKeptEmpty = 528;
-constexpr uint32_t kMwBarBytes = 640;
-constexpr int kMwKeptFlag = 0x40000000;   // slot code: a kept row (low bits: which); else a signed ring offset + bias
-constexpr int kMwBias = 1 << 20;
+constexpr int kMaWinMaxRing = 64;
+constexpr int kMwUnroll = 4;     // workers per consumer iteration
+// barrier block: ring full [0, 512), ring empty [512, 1024), kept full [1024, 1040), kept empty [1040, 1056)
+constexpr uint32_t kMwRingFull = 0, kMwRingEmpty = 512, kMwKeptFull = 1024, kMwKeptEmpty = 1040;
+constexpr uint32_t kMwBarBytes = 1152;
 
-template <typename TH>
-__global__ void __launch_bounds__(1024, 1) sync_ma_window_kernel(const MaWinParams P) {
+// 16 bytes from shared memory by 32-bit shared address (the consumers' inner loop works on plain
+// 32-bit offsets: 64-bit generic pointers cost several instructions per access)
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+template <typename TH> struct Row16;          // the elements in 16 bytes of a row, widened to fp32
+template <> struct Row16<float> {
+  static __device__ __forceinline__ void widen(const uint4& v, float (&x)[4]) {
+    x[0] = __uint_as_float(v.x); x[1] = __uint_as_float(v.y); x[2] = __uint_as_float(v.z); x[3] = __uint_as_float(v.w);
+  }
+};
+template <> struct Row16<__nv_bfloat16> {
+  static __device__ __forceinline__ void widen(const uint4& v, float (&x)[8]) {
+    x[0] = __uint_as_float(v.x << 16); x[1] = __uint_as_float(v.x & 0xFFFF0000u);
+    x[2] = __uint_as_float(v.y << 16); x[3] = __uint_as_float(v.y & 0xFFFF0000u);
+    x[4] = __uint_as_float(v.z << 16); x[5] = __uint_as_float(v.z & 0xFFFF0000u);
+    x[6] = __uint_as_float(v.w << 16); x[7] = __uint_as_float(v.w & 0xFFFF0000u);
+  }
+};
+
+template <typename TH, int V>
+__global__ void __launch_bounds__(544, 1) sync_ma_window_kernel(const MaWinParams P) {
   constexpr int MV = ThetaTraits<TH>::VEC;      // elements per 16 bytes
   extern __shared__ __align__(128) unsigned char smem[];
   const uint32_t bars = smem_u32(smem);
@@ -75,11 +96,11 @@ __global__ void __launch_bounds__(1024, 1) sync_ma_window_kernel(const MaWinPara
   if (threadIdx.x == 0) {
     for (int r = 0; r < R; ++r) {
       mbar_init(bars + kMwRingFull + 8 * r, 1);
-      mbar_init(bars + kMwRingEmpty + 8 * r, P.ncons);
+      mbar_init(bars + kMwRingEmpty + 8 * r, P.ncons / 32);   // one arrival per consumer warp
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(bars + kMwKeptFull + 8 * s, 1);
-      mbar_init(bars + kMwKeptEmpty + 8 * s, P.ncons);
+      mbar_init(bars + kMwKeptEmpty + 8 * s, P.ncons / 32);
     }
     for (int s = 0; s < 2; ++s) reinterpret_cast<TileDesc*>(meta0 + (size_t)s * P.meta_stride)->comp = -1;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -109,8 +130,13 @@ __global__ void __launch_bounds__(1024, 1) sync_ma_window_kernel(const MaWinPara
       cb = __ldg(P.off + comp);
       ce = __ldg(P.off + comp + 1);
     }
-    long long gi = 0;          // ring rows requested so far, over all tiles of this CTA
-    int meta_comp[2] = {-1, -1};
+    // ring rows are requested in one running sequence over all tiles of this CTA; the next one
+    // goes to `slot`, whose barriers are in phase `slot_par`.  (Kept incremental: this loop runs
+    // once per row and a division in it would cost more than the copy it issues.)
+    int slot = 0;
+    uint32_t slot_par = 0;
+    bool wrapped = false;      // the ring has been filled once: a slot must be released before re-use
+    int meta_comp0 = -1, meta_comp1 = -1;   // which component's codes each meta entry holds
     for (int it = 0; it < my_tiles && ok; ++it) {
       const int w = (int)blockIdx.x + it * (int)gridDim.x;
       if (w >= pfx_hi) {
@@ -137,7 +163,7 @@ __global__ void __launch_bounds__(1024, 1) sync_ma_window_kernel(const MaWinPara
       unsigned char* meta = meta0 + (size_t)set * P.meta_stride;
       TileDesc* d = reinterpret_cast<TileDesc*>(meta);
       int* codes = reinterpret_cast<int*>(meta + sizeof(TileDesc));
-      if (meta_comp[set] != comp) {
+      if ((set ? meta_comp1 : meta_comp0) != comp) {
         // the drawn neighbours as slot codes: kept row v (or v - K), else the signed ring offset
         // from the worker's own ring index (v - k, or v + p - k for the first read of a last row)
         const int32_t* gnb = P.nbr + (size_t)comp * K * q;
@@ -148,14 +174,17 @@ __global__ void __launch_bounds__(1024, 1) sync_ma_window_kernel(const MaWinPara
           if (dist > p) dist -= K;
           if (dist < -p) dist += K;
           const int v = k + dist;
+          // (kept row: its byte offset in the kept set, flagged by bit 0; else the signed byte
+          // offset from the worker's own ring slot)
           int code;
-          if (v < 0) code = kMwBias + dist + p;
-          else if (v < p) code = kMwKeptFlag | v;
-          else if (v < K) code = kMwBias + dist;
-          else code = kMwKeptFlag | (v - K);
+          const int rb = (int)P.row_bytes;
+          if (v < 0) code = ((dist + p) * rb) * 2;
+          else if (v < p) code = (v * rb) * 2 + 1;
+          else if (v < K) code = (dist * rb) * 2;
+          else code = ((v - K) * rb) * 2 + 1;
           codes[x] = code;
         }
-        meta_comp[set] = comp;
+        if (set) meta_comp1 = comp; else meta_comp0 = comp;
       }
       __syncwarp();
       if (lane == 0) {
@@ -174,33 +203,54 @@ __global__ void __launch_bounds__(1024, 1) sync_ma_window_kernel(const MaWinPara
           bulk_load_row(dst + (uint32_t)r * P.row_bytes, theta + (long long)r * P.ld + e0, bytes, full);
       }
       // ring rows
-      for (int i = 0; i < K && ok; ++i, ++gi) {
-        const int slot = (int)(gi % R);
-        if (gi >= R) {
-          bool fine = mbar_wait_bounded(bars + kMwRingEmpty + 8 * slot, (uint32_t)((gi / R) - 1) & 1, P.status);
+      const TH* src = theta + (long long)(K - p) * P.ld + e0;      // ring index 0 is row K - p
+      for (int i = 0; i < K && ok; ++i) {
+        if (i == p) src = theta + (long long)p * P.ld + e0;        // ring index i >= p is row i
+        if (wrapped) {
+          // the slot's previous occupant was released in the phase before the current one
+          bool fine = mbar_wait_bounded(bars + kMwRingEmpty + 8 * slot, slot_par ^ 1, P.status);
           ok = __all_sync(0xffffffffu, fine);
           if (!ok) break;
         }
         if (lane == 0) {
-          const int row = i < p ? K - p + i : i;
           const uint32_t full = bars + kMwRingFull + 8 * slot;
           mbar_arrive_expect_tx(full, bytes);
-          bulk_load_row(smem_u32(ring0 + (size_t)slot * P.row_bytes), theta + (long long)row * P.ld + e0, bytes, full);
+          bulk_load_row(smem_u32(ring0 + (size_t)slot * P.row_bytes), src, bytes, full);
         }
+        src += P.ld;
+        if (++slot == R) { slot = 0; slot_par ^= 1; wrapped = true; }
       }
     }
     if (!ok) {
-      // leave only after the copies already requested into this CTA's shared memory have landed
-      for (long long j = gi > R ? gi - R : 0; j < gi; ++j)
-        mbar_wait_bounded(bars + kMwRingFull + 8 * (int)(j % R), (uint32_t)(j / R) & 1, P.status);
+      // leave only after the copies already requested into this CTA's shared memory have landed:
+      // every slot's newest request is in phase slot_par (slots before `slot`) or the one before
+      for (int j = 0; j < R; ++j) {
+        const bool cur_phase = j < slot;
+        if (!cur_phase && !wrapped) continue;                      // never requested
+        mbar_wait_bounded(bars + kMwRingFull + 8 * j, cur_phase ? slot_par : slot_par ^ 1, P.status);
+      }
     }
     return;
   }
 
   // -------------------------------------------------------------------- consumer warps
+  // A row is 8 KB at most, so a worker takes well under a microsecond: the loop over the workers
+  // has to be lean.  A thread owns V pieces of 16 bytes of every row (columns (c + v * ncons) *
+  // MV; V = 1 is what is launched: with 2 and 4 pieces and a half or a quarter of the warps the
+  // round ran slower, the warps' instruction streams being latency-bound); workers are taken
+  // four at a time, stage by stage, so that the shared-memory round trips of one overlap the
+  // arithmetic of the others; addresses are 32-bit shared addresses, slot and phase are carried
+  // along instead of recomputed, and a warp arrives on a barrier once, through lane 0, after
+  // all its lanes have finished reading.
   const int c = threadIdx.x - 32;
-  const int col = c * MV;                 // this thread's 16 bytes of every row
-  long long gi = 0;                       // ring index of worker 0 of the current tile, running
+  const bool lane0 = (threadIdx.x & 31) == 0;
+  const uint32_t rb = P.row_bytes;
+  const int ring_bytes = R * (int)rb;
+  const uint32_t ring_b = smem_u32(ring0) + (uint32_t)c * 16u;
+  const uint32_t vstep = (uint32_t)P.ncons * 16u;          // bytes between a thread's pieces
+  int cur = 0;                            // slot of the current worker's ring index, running over tiles
+  int cur_off = 0;                        // cur * row bytes
+  uint32_t cur_par = 0;                   // and the phase of that slot's barriers
   for (int it = 0; it < my_tiles; ++it) {
     const int set = it & 1;
     if (!mbar_wait_bounded(bars + kMwKeptFull + 8 * set, (uint32_t)(it >> 1) & 1, P.status)) return;
@@ -208,79 +258,133 @@ __global__ void __launch_bounds__(1024, 1) sync_ma_window_kernel(const MaWinPara
     const TileDesc* d = reinterpret_cast<const TileDesc*>(meta);
     const int* codes = reinterpret_cast<const int*>(meta + sizeof(TileDesc));
     const long long e0 = d->e0, lo = d->lo, hi = d->hi;
-    const TH* kept = reinterpret_cast<const TH*>(kept0 + (size_t)set * p * P.row_bytes);
-    const long long e = e0 + col;
-    const bool mine = col < P.T && e < hi && e + MV > lo;
-    const bool whole = e >= lo && e + MV <= hi;
-    int cur = (int)(gi % R);              // slot of ring index k
+    const uint32_t kept_b = smem_u32(kept0 + (size_t)set * p * rb) + (uint32_t)c * 16u;
+    bool mine[V], whole[V];
+    bool any = false;
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+      const long long e = e0 + (long long)(c + v * P.ncons) * MV;
+      mine[v] = e < hi && e + MV > lo;
+      whole[v] = e >= lo && e + MV <= hi;
+      any |= mine[v];
+    }
+    TH* gp = theta + e0 + (long long)c * MV;   // this thread's first piece of worker k's row
     // the newest ring index the next worker needs, min(k + p, K - 1): slot and barrier phase
     int ahead = cur;
-    uint32_t ahead_par = (uint32_t)(gi / R) & 1;
+    uint32_t ahead_par = cur_par;
     if (!mbar_wait_bounded(bars + kMwRingFull + 8 * ahead, ahead_par, P.status)) return;
     for (int i = 1; i <= p && i < K; ++i) {          // before worker 0: ring indices 0 .. min(p, K-1)
       if (++ahead == R) { ahead = 0; ahead_par ^= 1; }
       if (!mbar_wait_bounded(bars + kMwRingFull + 8 * ahead, ahead_par, P.status)) return;
     }
-    for (int k = 0; k < K; ++k) {
-      if (k > 0 && k + p < K) {
-        // one more ring index becomes needed with every worker
+    int ahead_idx = p < K ? p : K - 1;     // the ring index `ahead` stands for
+    for (int k = 0; k < K; k += kMwUnroll) {
+      const int nu = K - k < kMwUnroll ? K - k : kMwUnroll;
+      const int need = k + nu - 1 + p < K - 1 ? k + nu - 1 + p : K - 1;
+      while (ahead_idx < need) {            // ring indices that become needed with these workers
+        ++ahead_idx;
         if (++ahead == R) { ahead = 0; ahead_par ^= 1; }
-        if (!mbar_wait_bounded(bars + kMwRingFull + 8 * ahead, ahead_par, P.status)) return;
+        const uint32_t bar = bars + kMwRingFull + 8 * ahead;
+        if (!mbar_try_wait(bar, ahead_par) && !mbar_wait_bounded(bar, ahead_par, P.status)) return;
       }
-      if (mine) {
-        float a[MV], t[MV];
-        const TH* own = k < p ? kept + (size_t)k * P.T : reinterpret_cast<const TH*>(ring0 + (size_t)cur * P.row_bytes);
-        ThetaTraits<TH>::lds(own + col, a);
+      if (any) {
+        float a[kMwUnroll][V][MV];
+        int off[kMwUnroll];                 // byte offset of worker k + u's own ring slot
+#pragma unroll
+        for (int u = 0; u < kMwUnroll; ++u) {
+          int o = cur_off + u * (int)rb;
+          o -= o >= ring_bytes ? ring_bytes : 0;
+          off[u] = o;
+          if (u < nu) {
+            const uint32_t src = k + u < p ? kept_b + (uint32_t)(k + u) * rb : ring_b + (uint32_t)o;
+#pragma unroll
+            for (int v = 0; v < V; ++v) Row16<TH>::widen(lds128(src + (uint32_t)v * vstep), a[u][v]);
+          }
+        }
         for (int j = 0; j < q; ++j) {
-          const int code = codes[k * q + j];
-          const TH* src;
-          if (code & kMwKeptFlag) {
-            src = kept + (size_t)(code & 0xFFFF) * P.T;
-          } else {
-            int s = cur + (code - kMwBias);
-            if (s < 0) s += R;
-            if (s >= R) s -= R;
-            src = reinterpret_cast<const TH*>(ring0 + (size_t)s * P.row_bytes);
-          }
-          ThetaTraits<TH>::lds(src + col, t);
 #pragma unroll
-          for (int x = 0; x < MV; ++x) a[x] = __fadd_rn(a[x], t[x]);
-        }
-        if (P.inv_exact) {
+          for (int u = 0; u < kMwUnroll; ++u) {
+            if (u < nu) {
+              const int code = codes[(k + u) * q + j];
+              const int off_n = code >> 1;               // byte offset (signed for ring rows)
+              int o = off[u] + off_n;
+              o += o < 0 ? ring_bytes : 0;
+              o -= o >= ring_bytes ? ring_bytes : 0;
+              const uint32_t src = (code & 1) ? kept_b + (uint32_t)off_n : ring_b + (uint32_t)o;
+              uint4 raw[V];
 #pragma unroll
-          for (int x = 0; x < MV; ++x) a[x] = __fmul_rn(a[x], P.inv_qp1);
-        } else {
-          uint32_t mid = 0xFFFFFFFFu;
+              for (int v = 0; v < V; ++v) raw[v] = lds128(src + (uint32_t)v * vstep);
 #pragma unroll
-          for (int x = 0; x < MV; ++x) mid &= mid_range_bit(a[x]);
-          if (mid & kMidRange) {
+              for (int v = 0; v < V; ++v) {
+                float t[MV];
+                Row16<TH>::widen(raw[v], t);
 #pragma unroll
-            for (int x = 0; x < MV; ++x) a[x] = divide_corrected(a[x], P.qp1, P.inv_qp1);
-          } else {
-#pragma unroll
-            for (int x = 0; x < MV; ++x) a[x] = __fdiv_rn(a[x], P.qp1);
+                for (int x = 0; x < MV; ++x) a[u][v][x] = __fadd_rn(a[u][v][x], t[x]);
+              }
+            }
           }
         }
-        const long long at = (long long)k * P.ld + e;
-        if (whole) {
-          ThetaTraits<TH>::stg(theta + at, a);
-        } else {
-          for (int x = 0; x < MV; ++x)
-            if (e + x >= lo && e + x < hi) theta[at + x] = ThetaTraits<TH>::narrow(a[x]);
+#pragma unroll
+        for (int u = 0; u < kMwUnroll; ++u) {
+          if (u < nu) {
+            TH* out = gp + (long long)u * P.ld;
+#pragma unroll
+            for (int v = 0; v < V; ++v) {
+              if (P.inv_exact) {
+#pragma unroll
+                for (int x = 0; x < MV; ++x) a[u][v][x] = __fmul_rn(a[u][v][x], P.inv_qp1);
+              } else {
+                uint32_t mid = 0xFFFFFFFFu;
+#pragma unroll
+                for (int x = 0; x < MV; ++x) mid &= mid_range_bit(a[u][v][x]);
+                if (mid & kMidRange) {
+#pragma unroll
+                  for (int x = 0; x < MV; ++x) a[u][v][x] = divide_corrected(a[u][v][x], P.qp1, P.inv_qp1);
+                } else {
+#pragma unroll
+                  for (int x = 0; x < MV; ++x) a[u][v][x] = __fdiv_rn(a[u][v][x], P.qp1);
+                }
+              }
+              TH* ov = out + (long long)v * P.ncons * MV;
+              if (whole[v]) {
+                ThetaTraits<TH>::stg(ov, a[u][v]);
+              } else if (mine[v]) {
+                const long long e = e0 + (long long)(c + v * P.ncons) * MV;
+                for (int x = 0; x < MV; ++x)
+                  if (e + x >= lo && e + x < hi) ov[x] = ThetaTraits<TH>::narrow(a[u][v][x]);
+              }
+            }
+          }
         }
       }
-      // ring index k - p is not needed by any later worker
-      if (k >= p) {
-        int s = cur - p;
-        if (s < 0) s += R;
+      gp += (long long)nu * P.ld;
+      // ring indices up to k + nu - 1 - p are not needed by any later worker
+      __syncwarp();
+      if (lane0) {
+        for (int u = 0; u < nu; ++u) {
+          if (k + u >= p) {
+            int s2 = cur + u - p;
+            s2 += s2 < 0 ? R : 0;
+            s2 -= s2 >= R ? R : 0;
+            mbar_arrive(bars + kMwRingEmpty + 8 * s2);
+          }
+        }
+      }
+      cur += nu;
+      cur_off += nu * (int)rb;
+      if (cur >= R) { cur -= R; cur_off -= ring_bytes; cur_par ^= 1; }
+    }
+    // after the last worker (cur is now the slot of the next tile's ring index 0): the last
+    // min(p, K) ring indices, which nobody released yet, and the kept rows / meta entry
+    __syncwarp();
+    if (lane0) {
+      int s = cur;
+      for (int i = 0; i < p && i < K; ++i) {
+        if (--s < 0) s = R - 1;
         mbar_arrive(bars + kMwRingEmpty + 8 * s);
       }
-      if (++cur == R) cur = 0;
+      mbar_arrive(bars + kMwKeptEmpty + 8 * set);
     }
-    // after the last worker: the ring indices nobody released yet, and the kept rows / meta entry
-    for (int i = (K - p > 0 ? K - p : 0); i < K; ++i) mbar_arrive(bars + kMwRingEmpty + 8 * (int)((gi + i) % R));
-    mbar_arrive(bars + kMwKeptEmpty + 8 * set);
-    gi += K;
   }
 }
 

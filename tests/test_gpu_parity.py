@@ -117,6 +117,18 @@ def test_gossip_ma_mode(dtype):
     run(case, random_theta0(case.N, seed=8, dtype=dtype), rounds=3, sigma=5e-2)
 
 
+@pytest.mark.parametrize("K,p,q", [(16, 8, 15), (16, 3, 6), (8, 3, 6), (12, 4, 5), (7, 3, 6), (6, 3, 5)])
+@pytest.mark.parametrize("dtype", [0, 1])
+def test_gossip_ma_many_neighbours(K, p, q, dtype):
+    """gossip-MA with many neighbours per draw (local-MA q = 2p, the full average q = K - 1)."""
+    offsets = (0, 3, 1001, 5000, 5004, 70_011)
+    case = Case(K=K, offsets=offsets, p=p, q=q, dtype=dtype, seed=3 * K + q, mode=binding.MODE_MA)
+    run(case, random_theta0(case.N, seed=K + q, dtype=dtype), rounds=3, sigma=5e-2,
+        masks=[None, [1, 1, 0, 1, 1], None])
+    run(case, random_theta0(case.N, seed=K + q, dtype=dtype), rounds=2, sigma=5e-2,
+        tuning=dict(tile_elems=256, theta_stages=2), check_nbr=False)
+
+
 def test_component_masks_and_periods():
     offsets = (0, 3000, 3001, 9000, 20000, 40001)
     masks = [[1, 0, 1, 0, 1], [0, 1, 0, 0, 0], [0, 0, 0, 0, 0], [1, 1, 1, 1, 1]]
@@ -592,14 +604,15 @@ def test_which_rows_are_resident_follows_the_ring(K, p, q, dtype, expect):
 
 
 @pytest.mark.parametrize("K,p,q,dtype,tuning,expect", [
-    (64, 5, 3, 0, None, "smem-window"), (64, 5, 3, 1, None, "smem-window"), (130, 6, 2, 1, None, "smem-window"),
-    (256, 7, 2, 0, None, "smem-window"), (48, 3, 6, 0, None, "smem-window"), (200, 32, 64, 0, None, "smem"),
+    (64, 5, 3, 0, dict(flags=16), "smem-window"), (64, 5, 3, 1, dict(flags=16), "smem-window"),
+    (130, 6, 2, 1, dict(flags=16), "smem-window"), (256, 7, 2, 0, None, "smem-window"),
+    (200, 6, 6, 0, None, "smem-window"), (200, 32, 64, 0, None, "smem"), (256, 7, 2, 1, None, "smem"),
     (9, 2, 4, 0, dict(flags=16), "smem-window"), (12, 1, 2, 1, dict(flags=16, tile_elems=512), "smem-window"),
-    (6, 2, 3, 0, dict(flags=16, tile_elems=128), "smem-window"), (64, 5, 10, 0, dict(tile_elems=256), "smem-window"),
+    (6, 2, 3, 0, dict(flags=16, tile_elems=128), "smem-window"), (64, 5, 10, 0, dict(flags=16, tile_elems=256), "smem-window"),
     (64, 5, 3, 0, dict(flags=32), "smem"), (20, 0, 0, 0, dict(flags=16), "smem-window")])
 def test_gossip_ma_ring_window(K, p, q, dtype, tuning, expect):
     """gossip-MA with many workers streams a window of rows along the ring through shared memory
-    (from 48 workers on, or on request): several tiles per CTA, ragged component edges, kept first
+    (fp32 theta from 192 workers on, or on request): several tiles per CTA, ragged component edges, kept first
     rows, last rows read twice, both theta types, and the settings where it is not taken."""
     offsets = (0, 5, 4099, 4100, 30_001, 70_003)
     case = Case(K=K, offsets=offsets, p=p, q=q, eta=0.9, zeta=1.0, dtype=dtype, seed=K + q,
@@ -646,8 +659,16 @@ def test_tensor_memory_variant_is_refused_where_it_does_not_apply():
                       mode=binding.MODE_MA)
     with pytest.raises(binding.GbmufError):
         g.set_tuning(flags=6)                      # gossip-MA
-    with pytest.raises(binding.GbmufError):
-        g.set_tuning(flags=16)                     # the ring window belongs to the tensor-memory tile
+    g.set_tuning(flags=16)                         # gossip-MA has a ring window of its own (shared memory)
+    g.set_partition([0, 1024])
+    assert g.launch_info()["variant"] == "smem-window"
+    g.destroy()
+    th = torch.zeros((3, 1024), device=dev)
+    g = binding.Gbmuf(th, th.clone(), th.clone(), K=3, N=1024, ld=1024, p=1, q=1, eta=0.9, zeta=1.0,
+                      mode=binding.MODE_MA)
+    with pytest.raises(binding.GbmufError) as e:
+        g.set_tuning(flags=16)                     # too few workers for a window: K < 2p + 2
+    assert e.value.status == binding.ERR_UNSUPPORTED
     g.destroy()
     th = torch.zeros((24, 1024), device=dev)
     g = binding.Gbmuf(th, th.clone(), th.clone(), K=24, N=1024, ld=1024, p=3, q=2, eta=0.9, zeta=1.0)
