@@ -1,7 +1,10 @@
-"""The multi-GPU plan on CPU: the path shards by column range with no data exchange.  Two gloo
-ranks each take their share from the shard planner, run the round on it alone (here with the
-oracle, since these ranks have no GPU), and the pieces must reassemble to the
-unsharded result; the timing reduction the bench uses is the max over ranks."""
+"""The column-range shard planner on CPU: `workloads.shard_even` cuts the columns between ranks,
+and because the path shards with no data exchange, running the round on each share alone must
+reassemble to the unsharded result.  Two gloo ranks do that here with the oracle as the round
+(these ranks have no GPU): this pins the PLANNER (global component / element indices of a share).
+The ranks of the product are covered elsewhere: `test_bench_ranks.py` drives the bench's own rank
+launching with two gloo ranks on CPU, and `test_gpu_bench_ranks.py` runs the CUDA library inside
+two rank processes and compares the reassembled state with the oracle."""
 import os
 import socket
 
