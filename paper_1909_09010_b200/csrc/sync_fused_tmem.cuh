@@ -108,25 +108,6 @@ template <> struct TmemCell<float> {
 #pragma unroll
     for (int c = 0; c < 4; ++c) { x[c] = __uint_as_float(r[c]); y[c] = __uint_as_float(r[4 + c]); }
   }
-  // four cells with one wait (used when a worker has many neighbours: the round trips overlap)
-  static __device__ __forceinline__ void fetch4(uint32_t t0, uint32_t t1, uint32_t t2, uint32_t t3,
-                                                float (&x)[4][4]) {
-    uint32_t r[16];
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%16];\n\t"
-        "tcgen05.ld.sync.aligned.32x32b.x4.b32 {%4, %5, %6, %7}, [%17];\n\t"
-        "tcgen05.ld.sync.aligned.32x32b.x4.b32 {%8, %9, %10, %11}, [%18];\n\t"
-        "tcgen05.ld.sync.aligned.32x32b.x4.b32 {%12, %13, %14, %15}, [%19];\n\t"
-        "tcgen05.wait::ld.sync.aligned;"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(t0), "r"(t1), "r"(t2), "r"(t3)
-        : "memory");
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-      for (int c = 0; c < 4; ++c) x[i][c] = __uint_as_float(r[i * 4 + c]);
-  }
 };
 template <> struct TmemCell<__nv_bfloat16> {
   static constexpr int COLS = 2;
@@ -160,29 +141,7 @@ template <> struct TmemCell<__nv_bfloat16> {
     y[0] = __uint_as_float(c << 16); y[1] = __uint_as_float(c & 0xFFFF0000u);
     y[2] = __uint_as_float(d << 16); y[3] = __uint_as_float(d & 0xFFFF0000u);
   }
-  static __device__ __forceinline__ void fetch4(uint32_t t0, uint32_t t1, uint32_t t2, uint32_t t3,
-                                                float (&x)[4][4]) {
-    uint32_t r[8];
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x2.b32 {%0, %1}, [%8];\n\t"
-        "tcgen05.ld.sync.aligned.32x32b.x2.b32 {%2, %3}, [%9];\n\t"
-        "tcgen05.ld.sync.aligned.32x32b.x2.b32 {%4, %5}, [%10];\n\t"
-        "tcgen05.ld.sync.aligned.32x32b.x2.b32 {%6, %7}, [%11];\n\t"
-        "tcgen05.wait::ld.sync.aligned;"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-        : "r"(t0), "r"(t1), "r"(t2), "r"(t3)
-        : "memory");
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      x[i][0] = __uint_as_float(r[2 * i] << 16); x[i][1] = __uint_as_float(r[2 * i] & 0xFFFF0000u);
-      x[i][2] = __uint_as_float(r[2 * i + 1] << 16); x[i][3] = __uint_as_float(r[2 * i + 1] & 0xFFFF0000u);
-    }
-  }
 };
-
-// From this many neighbours on, their cells are fetched four per wait.  (With 2 and 4 neighbours
-// several loads per wait measured slower; with a chain of 7 and more round trips they pay.)
-constexpr int kGatherBatchFrom = 8;
 
 // Sum of a worker's own cell (cell row `own`) and its q drawn neighbours' cells (cell rows nb[])
 // of element group `cell0` (the TMEM address of cell row 0), own first, then draw order, each
@@ -191,20 +150,7 @@ template <typename TH>
 __device__ __forceinline__ void tmem_gather(uint32_t cell0, int own, const int* nb, int q, float (&a)[4]) {
   constexpr int CW = TmemCell<TH>::COLS;
   TmemCell<TH>::fetch(cell0 + (uint32_t)(own * CW), a);
-  int j = 0;
-  if (q >= kGatherBatchFrom) {
-    // many neighbours: four cells per wait; the additions keep the draw order
-    for (; j + 4 <= q; j += 4) {
-      float t[4][4];
-      TmemCell<TH>::fetch4(cell0 + (uint32_t)(nb[j] * CW), cell0 + (uint32_t)(nb[j + 1] * CW),
-                           cell0 + (uint32_t)(nb[j + 2] * CW), cell0 + (uint32_t)(nb[j + 3] * CW), t);
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int x = 0; x < 4; ++x) a[x] = __fadd_rn(a[x], t[i][x]);
-    }
-  }
-  for (; j < q; ++j) {
+  for (int j = 0; j < q; ++j) {
     float t[4];
     TmemCell<TH>::fetch(cell0 + (uint32_t)(nb[j] * CW), t);
 #pragma unroll
@@ -227,8 +173,9 @@ __device__ __forceinline__ void tmem_gather2(uint32_t cellA, uint32_t cellB, int
     for (int x = 0; x < 4; ++x) { a[x] = __fadd_rn(a[x], t[x]); b[x] = __fadd_rn(b[x], u[x]); }
   }
 }
-// A thread's element groups are taken two at a time when the worker has few neighbours (with
-// many, the four-cells-per-wait path of tmem_gather already overlaps the round trips).
+// A thread's element groups are taken two at a time.  (Several cell rows of ONE group per wait --
+// two, or four from many neighbours on -- measured slower or no faster; with 15 neighbours the
+// pairs run the round in 16.97 ms against 19.4 ms with four cells of one group per wait.)
 constexpr bool kPairGroups = true;
 
 // What the producer must know to send a finished slot out: the staged range starts at e0, whole
@@ -510,7 +457,7 @@ __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParam
               }
             }
           };
-          const bool pairs = kPairGroups && q < kGatherBatchFrom;
+          const bool pairs = kPairGroups;
           for (int g = sub; g < ngroups; g += pairs ? 8 : 4) {
             float a[4], b[4];
             __syncwarp();                          // lanes that left the last group early rejoin
