@@ -138,3 +138,28 @@ def test_every_element_of_a_ring_window_round():
     w = workloads.get("profile64", offsets=cuts)
     assert w.K * w.N >= 1 << 30
     _full_round_check(w)
+
+
+# ------------------------------------------------------------------------------------------------
+# the whole schedule of a workload at full size, on sampled ranges
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("name,width,interior", [("wikitext103", 4096, 4), ("longrun", 1024, 2)])
+def test_full_size_whole_schedule_sampled(name, width, interior):
+    """All rounds the workload is specified with (wikitext103: 20 rounds, one local step each;
+    long-run: 100 rounds of 8 local steps each, bf16 theta), at full size in the launch
+    configuration the bench times, compared with the oracle after EVERY round on column ranges
+    around every component edge plus interior ones: momentum, global models and restart points
+    after many rounds, not only after the first two."""
+    w = workloads.get(name)
+    dev = torch.device("cuda:0")
+    theta0 = workloads.theta0_torch(w, dev)
+    if w.dtype == 1:
+        theta0 = theta0.to(torch.bfloat16)
+    pr = Pair(case_of(w), theta0, slices=_slices(w, width=width, interior=interior))
+    try:
+        for r in range(1, w.rounds + 1):
+            pr.perturb(step=r * w.local_steps, lr=w.lr, sigma=w.sigma, nsteps=w.local_steps)
+            pr.sync(r)
+            pr.compare(f"{name} round {r}")
+    finally:
+        pr.close()
