@@ -80,8 +80,8 @@ def test_full_size_sampled_parity(name, over, tuning):
 # every element of a full-size launch
 # ------------------------------------------------------------------------------------------------
 def _full_round_check(w, second_round=True):
-    """Round 1 from the state the initialisation line leaves (plus seeded local steps), and, if
-    asked, a second round with some components idle from the state round 1 left (momentum and
+    """The first synchronisation from the state the initialisation line leaves (plus seeded local
+    steps), and, if asked, a second one with some components idle from the state the first left (momentum and
     global models no longer trivial): all K * N elements of theta, omega and Delta against the
     oracle, in the launch configuration the bench times."""
     dev = torch.device("cuda:0")
@@ -104,7 +104,7 @@ def _full_round_check(w, second_round=True):
         torch.cuda.synchronize()
         assert g.device_status() == 0
         n = check_round_every_element(case, 1, (pre_theta, theta0, None), (theta, omega, delta),
-                                      what=f"{w.name} round 1")
+                                      what=f"{w.name} first synchronisation")
         assert n >= K * N // (1 << 26)
         if second_round:
             g.local_perturb(2, w.lr, 10 * w.sigma, w.local_steps)
@@ -114,7 +114,7 @@ def _full_round_check(w, second_round=True):
             torch.cuda.synchronize()
             assert g.device_status() == 0
             check_round_every_element(case, 2, pre, (theta, omega, delta), mask=mask,
-                                      what=f"{w.name} round 2")
+                                      what=f"{w.name} second synchronisation")
     finally:
         g.destroy()
 
