@@ -277,13 +277,14 @@ gbmuf_status plan_launch(gbmuf_ctx* ctx, const Tuning& t, Launch* out) {
   // second form is taken when it costs no tile width (or on request: flags bit 6).
   const int win_w = 2 * p + in_rows, cells_twice = win_w + p, cells_once = win_w + 2 * p;
   // widths whose element groups share out evenly over the consumer warps measured best for the
-  // window (fp32, K = 64..256: 4096 x 4 slots, 3072 x 6, 2048 x 8 ahead of 3584 x 4 and 2560 x 6;
+  // window (fp32, K = 64..256: 4096 x 4 slots, 3072 x 6, 2048 x 8 ahead of 3584 x 4; 2560 x 6 since a
+  // thread's element groups are taken in pairs: 5 groups per row beat 4;
   // bf16: 5120 x 4 and 4096 x 4 ahead of 3584 x 6 and 3072 x 6), the ring as deep as fits
-  static const int kWinF32[][2] = {{4096, 4}, {3072, 6}, {2048, 8}, {1024, 8}, {512, 8}};
+  static const int kWinF32[][2] = {{4096, 4}, {3072, 6}, {2560, 6}, {2048, 8}, {1024, 8}, {512, 8}};
   static const int kWinBf16[][2] = {{5120, 4}, {4096, 4}, {3584, 6}, {3072, 6}, {2048, 8}, {1024, 8}, {512, 8}};
   auto window_shape = [&](int rows, int* ring) {         // widest listed tile for `rows` cell rows
     const int (*tab)[2] = esz == 4 ? kWinF32 : kWinBf16;
-    const int n = esz == 4 ? 5 : 7;
+    const int n = esz == 4 ? 6 : 7;
     for (int i = 0; i < n; ++i)
       if ((tab[i][0] / 512) * rows * cw <= 512) { if (ring) *ring = tab[i][1]; return tab[i][0]; }
     return 0;

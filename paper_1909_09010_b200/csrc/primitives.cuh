@@ -55,12 +55,7 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // two seconds
 // caller then leaves its loop.  (try_wait may itself suspend the thread for a while, so the bound
 // is on the timer, not on the number of tries.)
 __device__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, int32_t* status) {
-  // The first tries go without the clock: reading %globaltimer costs a few hundred nanoseconds,
-  // which a producer that waits once per 4 KB row cannot afford on every wait, and a try that
-  // finds the phase incomplete suspends the thread for a bounded time by itself.
-#pragma unroll 1
-  for (int i = 0; i < 16; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
+  if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_timer_ns();
   for (uint32_t spin = 0;; ++spin) {
     if (mbar_try_wait(bar, parity)) return true;
