@@ -50,10 +50,10 @@ NVLINK_GBS_PER_DIRECTION = 770.0     # measured peer copy on this machine, per dire
 # theta dtype it was taken with: key = (variant, dtype); 0 fp32 from workload profile16, 1 bf16
 # from profile16bf (all K rows in tensor memory); the ring-window figure is from profile64 and
 # holds for that ring only (K = 64, p = 5: p / K extra theta row reads).
-NCU_TRAFFIC = {"source_sha": "0748bf3e860f",
-               "bytes_per_replica_param": {("tmem", 0): (3.221729e9 + 3.161231e9) / 268435536,
-                                           ("tmem", 1): (2.684594e9 + 2.625002e9) / 268435536,
-                                           ("tmem-window", 0): (3.310324e9 + 3.160895e9) / 268435776},
+NCU_TRAFFIC = {"source_sha": "eef893168e51",
+               "bytes_per_replica_param": {("tmem", 0): (3.221349e9 + 3.161665e9) / 268435536,
+                                           ("tmem", 1): (2.684770e9 + 2.625498e9) / 268435536,
+                                           ("tmem-window", 0): (3.311525e9 + 3.161882e9) / 268435776},
                "window_ring": (64, 5)}
 
 

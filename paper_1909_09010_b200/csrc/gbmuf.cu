@@ -581,6 +581,24 @@ gbmuf_status launch_round(gbmuf_ctx* ctx, const gbmuf_config& cfg, const Launch&
   return GBMUF_OK;
 }
 
+// Launches the round set-up kernel as a programmatic dependent of whatever kernel precedes it in
+// the stream: it may become resident early and waits (griddepcontrol.wait, its first
+// instruction) for that kernel to finish before it touches anything.
+cudaError_t launch_setup(const SetupParams& S, cudaStream_t st) {
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t lc = {};
+  const long long items = (long long)S.K * S.m;
+  lc.gridDim = dim3((unsigned)((items + 255) / 256), 1, 1);
+  lc.blockDim = dim3(256, 1, 1);
+  lc.dynamicSmemBytes = 0;
+  lc.stream = st;
+  lc.attrs = attr;
+  lc.numAttrs = 1;
+  return cudaLaunchKernelEx(&lc, round_setup_kernel, S);
+}
+
 void fill_setup(const gbmuf_ctx* ctx, uint64_t round, bool use_mask, bool plan, int32_t* nbr,
                 SetupParams* S) {
   S->K = ctx->cfg.K; S->m = ctx->m; S->p = ctx->cfg.p; S->q = ctx->cfg.q;
@@ -932,9 +950,7 @@ gbmuf_status gbmuf_sync_round(gbmuf_ctx* ctx, uint64_t round, const uint8_t* com
   }
   SetupParams S;
   fill_setup(ctx, round, comp_mask != nullptr, true, ctx->d_nbr, &S);
-  const long long items = (long long)ctx->cfg.K * ctx->m;
-  round_setup_kernel<<<(int)((items + 255) / 256), 256, 0, st>>>(S);
-  e = cudaGetLastError();
+  e = launch_setup(S, st);
   if (e != cudaSuccess) return cuda_fail(ctx, "launch of the round set-up kernel", e);
 
   const gbmuf_status rc = launch_round(ctx, ctx->cfg, L, ctx->theta, ctx->omega, ctx->delta, ctx->cfg.ld, ctx->m,
@@ -1222,9 +1238,7 @@ gbmuf_status gbmuf_sync_round_noalloc(const gbmuf_config* cfg, void* theta, floa
     S.mask = scratch + kNaMaskOff;
     S.nbr = reinterpret_cast<int32_t*>(scratch + kNaNbrOff);
     S.tile_prefix = reinterpret_cast<int32_t*>(scratch + kNaPrefixOff);
-    const long long items = (long long)cfg->K * m;
-    round_setup_kernel<<<(int)((items + 255) / 256), 256, 0, cs>>>(S);
-    e = cudaGetLastError();
+    e = launch_setup(S, cs);
     if (e != cudaSuccess) return cuda_fail(nullptr, "launch of the round set-up kernel", e);
 
     st = launch_round(&tmp, *cfg, L, theta, omega, delta, cfg->ld, m, S.off, S.tile_prefix, S.nbr, d_status,
@@ -1469,8 +1483,7 @@ gbmuf_status gbmuf_host_sync_round(gbmuf_host* h, void* theta, float* omega, flo
     S.mask = hs.tables + h->t_mask;
     S.nbr = reinterpret_cast<int32_t*>(hs.tables + h->t_nbr);
     S.tile_prefix = reinterpret_cast<int32_t*>(hs.tables);
-    round_setup_kernel<<<(int)(((long long)K * c.mc + 255) / 256), 256, 0, cs>>>(S);
-    e = cudaGetLastError();
+    e = launch_setup(S, cs);
     if (e != cudaSuccess) { st = cuda_fail(nullptr, "launch of the round set-up kernel", e); break; }
     st = launch_round(&hs.ctx, cfg, hs.ctx.launch, hs.ctx.theta, hs.ctx.omega, hs.ctx.delta, chunk_cols, c.mc,
                       S.off, S.tile_prefix, S.nbr, reinterpret_cast<int32_t*>(hs.tables + h->t_status), total, cs);

@@ -19,6 +19,7 @@ __global__ void __launch_bounds__(256) perturb_kernel(TH* theta, int K, long lon
                                                       uint32_t key0, uint32_t key1, uint32_t step0,
                                                       int nsteps, float lr, float sigma,
                                                       long long elem_base) {
+  grid_launch_dependents();
   constexpr int VEC = ThetaTraits<TH>::VEC;
   const long long nvec = (N + VEC - 1) / VEC;
   const int k = blockIdx.y;                 // one grid row per worker
@@ -144,6 +145,7 @@ struct AdagradSlot { long long e0, hi, se; int k; int where; float sc; int pad; 
 
 template <typename TH>
 __global__ void __launch_bounds__(544, 1) adagrad_stream_kernel(const AdagradParams P) {
+  grid_launch_dependents();
   constexpr int EB = (int)sizeof(TH);
   constexpr long long ALN = 16 / EB;                 // elements per 16 bytes of theta
   extern __shared__ __align__(128) unsigned char smem[];

@@ -48,6 +48,11 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
 __device__ __forceinline__ void grid_dependency_wait() {
   asm volatile("griddepcontrol.wait;" ::: "memory");
 }
+// Said at the top of the long kernels (the fused round, the local steps): a set-up kernel queued
+// behind them may be made resident early; it waits for their completion before doing anything.
+__device__ __forceinline__ void grid_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
 
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // two seconds
 // Wait for the phase with the given parity to complete.  Bounded in wall-clock time: after

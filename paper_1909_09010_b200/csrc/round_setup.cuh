@@ -45,8 +45,13 @@ __device__ __forceinline__ int tiles_of_component(int64_t lo, int64_t hi, int T)
 }
 
 __global__ void __launch_bounds__(256) round_setup_kernel(SetupParams P) {
-  // the round kernel that follows may begin its prologue now; it waits for this grid to finish
-  // before it reads the tables written below
+  // This kernel is itself launched as a programmatic dependent: it may become resident while the
+  // kernel before it in the stream (a local step, the previous round) still runs, which hides
+  // its launch latency.  It must not touch the tables before that kernel has finished -- the
+  // previous round reads them -- so it waits first.  Then the round kernel that follows may begin
+  // its prologue; it in turn waits for this grid to finish before it reads the tables written
+  // below (and thereby, transitively, for everything before this grid).
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (g < (int64_t)P.K * P.m && P.q > 0) {

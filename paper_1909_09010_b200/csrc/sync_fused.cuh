@@ -118,6 +118,7 @@ __device__ __forceinline__ void bmuf_filter(float avg, float& w, float& d, float
 template <typename TH>
 __global__ void __launch_bounds__(1024, 1)
 sync_fused_kernel(const SyncParams P, const __grid_constant__ CUtensorMap map_theta) {
+  grid_launch_dependents();
   constexpr int VEC = 4;   // elements per thread and row: 16 bytes of omega / Delta, 16 or 8 of theta
   extern __shared__ __align__(128) unsigned char smem[];
   const uint32_t bars = smem_u32(smem);

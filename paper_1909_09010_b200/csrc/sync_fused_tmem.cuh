@@ -189,6 +189,7 @@ struct SlotInfo { long long e0, sb, se; int k; int pad; };
 // WIN: ring window (else all K rows resident; the window's arithmetic then folds away).
 template <typename TH, bool BULK, bool WIN>
 __global__ void __launch_bounds__(544, 1) sync_fused_tmem_kernel(const TmemParams P) {
+  grid_launch_dependents();
   constexpr int EB = (int)sizeof(TH);
   constexpr int CW = TmemCell<TH>::COLS;
   constexpr int IN_ROWS = 8 / EB;                    // theta rows per load item

@@ -84,6 +84,7 @@ template <> struct Row16<__nv_bfloat16> {
 
 template <typename TH, int V>
 __global__ void __launch_bounds__(544, 1) sync_ma_window_kernel(const MaWinParams P) {
+  grid_launch_dependents();
   constexpr int MV = ThetaTraits<TH>::VEC;      // elements per 16 bytes
   extern __shared__ __align__(128) unsigned char smem[];
   const uint32_t bars = smem_u32(smem);
