@@ -163,3 +163,31 @@ def test_full_size_whole_schedule_sampled(name, width, interior):
             pr.compare(f"{name} round {r}")
     finally:
         pr.close()
+
+
+def test_every_point_of_the_granularity_sweep_at_full_size():
+    """All 24 points of the granularity sweep (C in {4, 16, 64, 256} components with non-uniform
+    sizes, 1 / 2 / 4 neighbours, eta 0.5 / 0.9; K = 8 replicas of the 279 M-parameter model) in the
+    launch configuration the bench times: one synchronisation each after seeded local steps,
+    compared with the oracle on column ranges around every component edge (at most 48 of them,
+    evenly picked) plus interior ones."""
+    dev = torch.device("cuda:0")
+    for C, q, eta in workloads.SWEEP_POINTS:
+        w = workloads.get("sweep", C=C, q=q, eta=eta)
+        sl = workloads.edge_slices(w.offsets, 2048, count=48)
+        g = np.random.Generator(np.random.PCG64(1000 + C + q))
+        for _ in range(3):
+            a = int(g.integers(0, w.N - 2048))
+            if all(b <= a or a + 2048 <= c for c, b in sl):
+                sl.append((a, a + 2048))
+        pr = Pair(case_of(w), workloads.theta0_torch(w, dev), slices=sorted(sl))
+        try:
+            assert pr.g.launch_info()["grid"] == torch.cuda.get_device_properties(0).multi_processor_count
+            pr.perturb(step=1, lr=w.lr, sigma=10 * w.sigma, nsteps=1)
+            pr.check_neighbors(1)
+            pr.sync(1)
+            pr.compare(f"sweep C={C} q={q} eta={eta}")
+        finally:
+            pr.close()
+            del pr
+            torch.cuda.empty_cache()
