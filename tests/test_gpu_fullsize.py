@@ -79,21 +79,23 @@ def test_full_size_sampled_parity(name, over, tuning):
 # ------------------------------------------------------------------------------------------------
 # every element of a full-size launch
 # ------------------------------------------------------------------------------------------------
-def _full_round_check(w, second_round=True):
+def _full_round_check(w, second_round=True, tuning=None):
     """The first synchronisation from the state the initialisation line leaves (plus seeded local
     steps), and, if asked, a second one with some components idle from the state the first left (momentum and
     global models no longer trivial): all K * N elements of theta, omega and Delta against the
     oracle, in the launch configuration the bench times."""
     dev = torch.device("cuda:0")
-    case = case_of(w)
+    case = case_of(w, mode=w.mode)
     K, N, ld = w.K, w.N, w.ld
     theta0 = workloads.theta0_torch(w, dev).to(tdtype(w.dtype))
     theta = torch.empty((K, ld), dtype=tdtype(w.dtype), device=dev)
     omega = torch.empty((K, ld), dtype=torch.float32, device=dev)
     delta = torch.empty((K, ld), dtype=torch.float32, device=dev)
     g = binding.Gbmuf(theta, omega, delta, K=K, N=N, ld=ld, p=w.p, q=w.q, eta=w.eta, zeta=w.zeta,
-                      seed=w.seed, theta_dtype=w.dtype)
+                      seed=w.seed, theta_dtype=w.dtype, mode=w.mode)
     try:
+        if tuning:
+            g.set_tuning(**tuning)
         g.set_partition(w.offsets)
         info = g.launch_info()
         assert info["grid"] == torch.cuda.get_device_properties(0).multi_processor_count
@@ -128,6 +130,18 @@ def test_every_element_of_the_headline_launch():
 def test_every_element_of_a_long_run_round():
     """The mixed-precision workload (bf16 theta, K = 16, 238.5 M columns, 64 components)."""
     _full_round_check(workloads.get("longrun"), second_round=False)
+
+
+def test_every_element_of_a_gossip_ma_round():
+    """The other branch of Algorithm 1 (theta <- average) at the wikitext103 size: every element
+    of one round through the gossip-MA schedule of the shared-memory kernel."""
+    _full_round_check(workloads.get("wikitext103", mode=1), second_round=False)
+
+
+def test_every_element_with_the_shared_memory_tile():
+    """The gossip-BMUF round with the theta tile in shared memory (tuning flag bit 3), K = 8
+    replicas of the wikitext103 model: every element of one round."""
+    _full_round_check(workloads.get("sweep", C=16, q=2, eta=0.9), second_round=False, tuning=dict(flags=8))
 
 
 def test_every_element_of_a_ring_window_round():
