@@ -81,6 +81,30 @@ def test_host_handle_over_several_rounds(dtype, mode, row_copies):
         h.destroy()
 
 
+def test_host_handle_many_chunks_of_the_default_size():
+    """Five chunks of the default 2,097,152 columns rotate through the three buffer sets (every
+    set is re-used), two rounds, the second with a mask that leaves whole chunks untouched;
+    every element against the oracle."""
+    K, p, q, eta, zeta, seed = 8, 2, 2, 0.9, 1.0, 77
+    N = (1 << 23) + 5
+    offsets = (0, 1 << 21, (1 << 21) + 3, 3 << 21, (3 << 21) + 1000, N)
+    st = oracle.init(random_theta0(N, seed=4), K)
+    oracle.local_perturb(st, seed, 0, 1.0, 0.05)
+    th = torch.from_numpy(st.theta).clone().pin_memory()
+    om = torch.from_numpy(st.omega).clone().pin_memory()
+    de = torch.from_numpy(st.delta).clone().pin_memory()
+    h = binding.GbmufHost(offsets, K=K, N=N, ld=N, p=p, q=q, eta=eta, zeta=zeta, seed=seed)
+    try:
+        for rnd, mask in ((1, None), (2, [0, 1, 1, 0, 1])):
+            h.sync_round(th, om, de, rnd, mask)
+            nbr = oracle.sample_neighbors(seed, rnd, K, len(offsets) - 1, p, q)
+            oracle.sync_round(st, offsets, nbr, eta, zeta, sync=mask)
+            for name, got, ref in (("theta", th, st.theta), ("omega", om, st.omega), ("delta", de, st.delta)):
+                assert np.array_equal(got.numpy().view(np.uint32), ref.view(np.uint32)), f"{name}, round {rnd}"
+    finally:
+        h.destroy()
+
+
 def test_host_round_argument_errors():
     K, N = 4, 1000
     th = torch.zeros((K, N))
