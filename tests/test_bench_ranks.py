@@ -76,3 +76,31 @@ def test_peer_form_is_parsed_and_needs_ranks():
     assert "one worker per rank x3" in bench.parallelism_text("peer", 3)
     with pytest.raises(SystemExit):
         bench.resolve_workload(bench.build_parser().parse_args(["--workload", "tiny:form=nope"]))
+
+
+def test_clock_sampler_summarises_a_window():
+    """The nvidia-smi sampler's parsing and binning, fed with canned rows (no GPU needed)."""
+    s = bench.ClockSampler(0)
+    s.proc = object()                                    # pretend the query is running
+    row = "{sm}, 1965, {w}, Not Active, Not Active, Not Active, {cap}, 3996"
+    s.rows = [(10.0, row.format(sm=1965, w=700.0, cap="Not Active")),
+              (10.1, row.format(sm=1740, w=995.5, cap="Active")),
+              (10.2, row.format(sm=1725, w=996.0, cap="Active")),
+              (10.3, "garbage"),
+              (99.0, row.format(sm=500, w=100.0, cap="Not Active"))]      # outside the window
+    out = s.window(10.0, 10.25, detail=True)
+    assert out["samples"] == 3 and out["sm_mhz"] == 1740.0 and out["sm_max_mhz"] == 1965.0
+    assert out["reasons"] == ["sw_power_cap"] and out["mem_mhz"] == 3996.0
+    assert out["power_w_max"] == 996.0 and out["samples_by_sm_mhz"] == {"1700-1799": 2, "1900-1999": 1}
+    e = bench._regime_entry(17.0, 24 * 4458028400, 6530.0, out)
+    assert abs(e["gbs"] - 24 * 4458028400 / 17.0e-3 / 1e9) < 1e-6 and abs(e["ms_x_sm_ghz"] - 17.0 * 1.74) < 1e-9
+
+
+def test_traffic_constants_name_a_kernel_fingerprint():
+    """The DRAM-traffic constants are only applied to the kernel source they were measured on."""
+    sha = bench.source_sha()
+    assert len(sha) == 12 and all(c in "0123456789abcdef" for c in sha)
+    assert set(bench.NCU_TRAFFIC["bytes_per_replica_param"]) == {("tmem", 0), ("tmem", 1), ("tmem-window", 0)}
+    for (variant, dtype), b in bench.NCU_TRAFFIC["bytes_per_replica_param"].items():
+        alg = bench.algorithmic_bytes_per_replica_param(dtype)
+        assert 0.97 * alg < b < 1.03 * alg, (variant, dtype, b)      # measured traffic ~ algorithmic bytes
